@@ -1,0 +1,284 @@
+"""CPU oracle for the Pre-hoc Sparsity (PrHS / CIS) sparse decode-attention path.
+
+TEST INFRASTRUCTURE ONLY.  This module is a plain, slow, obviously-correct restatement
+of what the path computes, written from the paper's definitions.  Only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import it.  It shares no code with
+the CUDA library and never imports it; the CUDA library never imports this module.
+
+Precision.  The paper does not fix a precision.  Inputs are bf16 values widened exactly
+to float64; every dot product, softmax sum and mass is formed in float64.  The one place
+where floating point decides an integer -- the top-k ranking -- is taken on the logits
+rounded once to float32, the precision the CUDA path ranks in.
+
+Indexing.  0-based, half-open.  `t` is the number of cached positions visible to the
+current query, the current token (position t-1) included.  The paper is 1-based; its
+three groups (Sec. 4.1 "Selection Criteria") become
+    sinks  = [0, S0)        middle candidates = [S0, t-W)        local = [t-W, t)
+which are pairwise disjoint.
+
+Every function below is pinned by tests/test_oracle_pins.py against closed forms,
+brute-force enumeration, textbook identities and the paper's inequalities, except
+cross-layer reuse (`PrhsOracle` with layer_group > 1), which the paper only motivates
+and does not define: that part is "parity unpinned" beyond structural invariants.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+__all__ = [
+    "dense_scores", "rank_logits", "softmax_full", "logsumexp", "dense_attention",
+    "topk_middle", "dilate", "build_set", "attn_over_set", "retained_mass",
+    "dropped_mass", "delta_from_lse", "mi_bound_g", "coverage", "bf16_round",
+    "Schedule", "PrhsOracle",
+]
+
+
+# --------------------------------------------------------------------------- helpers
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round float values to the nearest bf16 (ties to even); result as float32.
+
+    Used only to compare against the CUDA path's bf16 output tensor.
+    """
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    bits = x32.view(np.uint32).astype(np.uint64)
+    lsb = (bits >> 16) & 1
+    rounded = ((bits + 0x7FFF + lsb) >> 16) << 16
+    out = rounded.astype(np.uint32).view(np.float32)
+    return np.where(np.isfinite(x32), out, x32).astype(np.float32)
+
+
+# ------------------------------------------------------------------ Eq. (2): attention
+def dense_scores(q: np.ndarray, K: np.ndarray, t: int) -> np.ndarray:
+    """Logits a_i = q . k_i / sqrt(d) for every cached position i < t  (Eq. 2), float64."""
+    d = q.shape[-1]
+    return (K[:t].astype(np.float64) @ q.astype(np.float64)) / math.sqrt(d)
+
+
+def rank_logits(a: np.ndarray) -> np.ndarray:
+    """The logits in the precision the ranking decision is taken in (float32)."""
+    return a.astype(np.float32)
+
+
+def logsumexp(a: np.ndarray) -> float:
+    """log sum_i exp(a_i) in float64; -inf for an empty vector."""
+    if a.size == 0:
+        return -math.inf
+    mx = float(np.max(a))
+    return mx + math.log(float(np.sum(np.exp(a.astype(np.float64) - mx))))
+
+
+def softmax_full(a: np.ndarray) -> np.ndarray:
+    """A_i = exp(a_i) / sum_j exp(a_j) over all visible positions (Eq. 2)."""
+    e = np.exp(a.astype(np.float64) - np.max(a))
+    return e / np.sum(e)
+
+
+def dense_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, t: int):
+    """y = sum_i A_i v_i over i < t (Eq. 2).  Returns (y float64 [d], lse float)."""
+    a = dense_scores(q, K, t)
+    A = softmax_full(a)
+    return A @ V[:t].astype(np.float64), logsumexp(a)
+
+
+# ------------------------------------------------- Sec. 4.1: top-k over the middle range
+def topk_middle(a: np.ndarray, t: int, sinks: int, window: int, k: int) -> np.ndarray:
+    """S* = the k positions of largest logit among the middle candidates [S0, t-W).
+
+    Returned in descending-logit order p_1, p_2, ... (Sec. 4.1: "sorted and selected in
+    descending order of attention weight"); equal logits are ordered by lower position
+    first.  Softmax is monotone in the logit, so ranking logits ranks attention weights.
+    The ranking uses the float32-rounded logits (see module docstring).
+    """
+    lo, hi = sinks, t - window
+    if hi <= lo or k <= 0:
+        return np.zeros(0, dtype=np.int64)
+    cand = np.arange(lo, hi, dtype=np.int64)
+    a32 = rank_logits(a[lo:hi])
+    # stable sort on the negated logit: descending logit, ascending position among equals
+    order = np.argsort(-a32.astype(np.float64), kind="stable")
+    return cand[order[: min(k, hi - lo)]]
+
+
+# ------------------------------------------------------------- Eq. (10): neighbour dilation
+def dilate(s_star: np.ndarray, m: int, r: int, t_anchor: int) -> np.ndarray:
+    """S^ = S* ∪ ⋃_{i<m} { p_i + j : -r <= j <= r }, clipped to [0, t_anchor)  (Eq. 10).
+
+    `s_star` is in descending-weight order, so its first m entries are the m highest-
+    weight winners.  Returns a sorted array of unique positions.
+    """
+    out = set(int(p) for p in s_star)
+    for p in s_star[: max(0, min(m, len(s_star)))]:
+        for j in range(-r, r + 1):
+            x = int(p) + j
+            if 0 <= x < t_anchor:
+                out.add(x)
+    return np.array(sorted(out), dtype=np.int64)
+
+
+# ---------------------------------------------------------------- Sec. 4.1: critical set
+def build_set(t: int, sinks: int, window: int, middle: np.ndarray) -> np.ndarray:
+    """C = [0, S0) ∪ M ∪ [t-W, t) at the CURRENT length t; sorted, unique (Sec. 4.1).
+
+    On a sharing step M is the anchor's (dilated) middle set (Def. 3.2); the sink and
+    local groups are positional and follow the current t.
+    """
+    out = set(range(0, min(sinks, t)))
+    out.update(int(x) for x in middle if 0 <= int(x) < t)
+    out.update(range(max(0, t - window), t))
+    return np.array(sorted(out), dtype=np.int64)
+
+
+# ------------------------------------------------------ Def. 3.1: token-sparse attention
+def attn_over_set(q: np.ndarray, K: np.ndarray, V: np.ndarray, C: np.ndarray):
+    """Attention restricted to index set C and renormalised over it (Def. 3.1).
+
+    Returns (y float64 [d], lse_C float) with lse_C = log sum_{i in C} exp(a_i).
+    """
+    d = q.shape[-1]
+    if len(C) == 0:
+        return np.zeros(d, dtype=np.float64), -math.inf
+    a = (K[C].astype(np.float64) @ q.astype(np.float64)) / math.sqrt(d)
+    mx = np.max(a)
+    e = np.exp(a - mx)
+    return (e / np.sum(e)) @ V[C].astype(np.float64), float(mx + math.log(np.sum(e)))
+
+
+# ---------------------------------------------------- Sec. 2.3: retained / dropped mass
+def retained_mass(a: np.ndarray, C: np.ndarray) -> float:
+    """tau_C = sum_{i in C} A_i with A the FULL softmax over all visible positions."""
+    return float(np.sum(softmax_full(a)[C]))
+
+
+def dropped_mass(a: np.ndarray, C: np.ndarray) -> float:
+    """delta_C = 1 - tau_C, summed directly over the complement to avoid cancellation."""
+    A = softmax_full(a)
+    mask = np.ones(a.shape[0], dtype=bool)
+    mask[C] = False
+    return float(np.sum(A[mask]))
+
+
+def delta_from_lse(lse_C: float, lse_full: float) -> float:
+    """delta = 1 - exp(lse_C - lse_full): the same quantity from the two log-sums."""
+    if lse_C == -math.inf:
+        return 1.0
+    return float(-math.expm1(lse_C - lse_full))
+
+
+def mi_bound_g(delta: float, L: int) -> float:
+    """g(delta) = 2 [ h_b(delta) + delta log L ]  (Eq. 4), natural logarithm."""
+    if delta <= 0.0:
+        return 0.0
+    hb = -delta * math.log(delta)
+    if delta < 1.0:
+        hb -= (1.0 - delta) * math.log1p(-delta)
+    return 2.0 * (hb + delta * math.log(L))
+
+
+def coverage(shared: np.ndarray, target: np.ndarray) -> float:
+    """|shared ∩ target| / |target|: the overlap measure of Fig. 4."""
+    if len(target) == 0:
+        return 1.0
+    return len(np.intersect1d(shared, target)) / float(len(target))
+
+
+# ------------------------------------------------------------- the per-step state machine
+@dataclass
+class Schedule:
+    """The knobs of CIS (Sec. 4.1, defaults Sec. 5.1) plus the cross-layer group size."""
+    top_k: int
+    window: int
+    sinks: int
+    refresh_interval: int = 1      # s: block size; the first step of a block retrieves
+    layer_group: int = 1           # G_L: layers sharing one leader's set (not in the paper body)
+    dilate_r: int = 1
+    dilate_m: int = -1             # -1 -> floor(k/3)
+    dilate_anchor: bool = False    # True: the anchor's own attention also uses S^
+    top_k_per_seq: np.ndarray | None = None
+
+    def k_for(self, b: int) -> int:
+        return int(self.top_k_per_seq[b]) if self.top_k_per_seq is not None else self.top_k
+
+    def m_for(self, b: int) -> int:
+        return self.k_for(b) // 3 if self.dilate_m < 0 else self.dilate_m
+
+
+@dataclass
+class _Shared:
+    step: int = -1
+    s_star: dict = field(default_factory=dict)   # (b, h) -> S* (descending weight)
+    s_hat: dict = field(default_factory=dict)    # (b, h) -> S^ (ascending)
+
+
+class PrhsOracle:
+    """Runs the decode-step schedule one (layer, step) at a time.
+
+    A (layer, step) retrieves iff the layer is the first of its group and the step is the
+    first of its block (step % s == 0).  The retrieving call stores S* and its dilation
+    S^ (Eq. 10) per (sequence, query head).  Every other (layer, step) of the same block
+    and group attends over C built from the stored S^ (Def. 3.2) with its own q, K, V.
+    The retrieving call itself attends over C built from the undilated S* unless
+    `dilate_anchor` is set (dilation costs budget "during sharing", Sec. 5.2.2).
+    """
+
+    def __init__(self, sched: Schedule, num_q_heads: int, num_kv_heads: int):
+        self.s = sched
+        self.hq, self.hkv = num_q_heads, num_kv_heads
+        self.gq = num_q_heads // num_kv_heads
+        self.groups: dict[int, _Shared] = {}
+
+    def is_retrieval(self, layer: int, step: int) -> bool:
+        return layer % self.s.layer_group == 0 and step % self.s.refresh_interval == 0
+
+    def index_set(self, layer: int, step: int, b: int, h: int, t: int) -> np.ndarray:
+        g = layer // self.s.layer_group
+        sh = self.groups.get(g)
+        anchor = step - step % self.s.refresh_interval
+        if sh is None or sh.step != anchor:
+            raise RuntimeError("group leader has not retrieved for this block")
+        own = self.is_retrieval(layer, step) and not self.s.dilate_anchor
+        M = sh.s_star[(b, h)] if own else sh.s_hat[(b, h)]
+        return build_set(t, self.s.sinks, self.s.window, M)
+
+    def decode_step(self, layer, step, q, K, V, seq_lens, units=None, want_delta=True):
+        """q [B][Hq][d]; K, V [B][Hkv][cap][d]; seq_lens [B].
+
+        `units` optionally restricts the work to a list of (b, h) pairs (sampled parity).
+        Returns dict with per-unit 'y' (float64), 'lse', 'delta', 'set', and on retrieval
+        steps 's_star', 'lse_full', 'scores32'.
+        """
+        B = q.shape[0]
+        if units is None:
+            units = [(b, h) for b in range(B) for h in range(self.hq)]
+        g = layer // self.s.layer_group
+        retrieve = self.is_retrieval(layer, step)
+        if retrieve:
+            sh = self.groups.setdefault(g, _Shared())
+            if sh.step != step:
+                sh.step, sh.s_star, sh.s_hat = step, {}, {}
+        out = {"y": {}, "lse": {}, "delta": {}, "set": {}, "s_star": {}, "lse_full": {},
+               "scores32": {}}
+        for (b, h) in units:
+            t = int(seq_lens[b])
+            kv = h // self.gq
+            a = None
+            if retrieve:
+                a = dense_scores(q[b, h], K[b, kv], t)
+                s_star = topk_middle(a, t, self.s.sinks, self.s.window, self.s.k_for(b))
+                sh = self.groups[g]
+                sh.s_star[(b, h)] = s_star
+                sh.s_hat[(b, h)] = dilate(s_star, self.s.m_for(b), self.s.dilate_r, t)
+                out["s_star"][(b, h)] = s_star
+                out["scores32"][(b, h)] = rank_logits(a)
+            C = self.index_set(layer, step, b, h, t)
+            y, lse_c = attn_over_set(q[b, h], K[b, kv], V[b, kv], C)
+            out["set"][(b, h)], out["y"][(b, h)], out["lse"][(b, h)] = C, y, lse_c
+            if want_delta:
+                if a is None:
+                    a = dense_scores(q[b, h], K[b, kv], t)
+                lse_full = logsumexp(a)
+                out["lse_full"][(b, h)] = lse_full
+                out["delta"][(b, h)] = delta_from_lse(lse_c, lse_full)
+        return out
