@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the PrHS sparse decode-attention path on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+A step is one pass of the whole hot path over one batch: one decode step of one layer
+(retrieval on the first step of every block of `refresh` steps, then index-set build and
+gathered attention).  The workload is the LLaMA-2-7B-shaped single layer at 32K context
+(batch 8, 32 MHA heads, k = 1024, window 128, 4 sinks, refresh every 4 steps), synthetic.
+
+Prints ONE JSON line.  `value` is attention-only decode throughput in tokens/s (batch tokens
+per step / device time per step) with every input resident in HBM; `e2e` is the same metric
+through the host-buffer entry point with the per-step host<->device copies timed.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_08329_b200 import workloads as W  # noqa: E402
+
+METRIC = "sparse_decode_attn_tokens_per_s_32k_ctx"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 256 << 20
+# DRAM bytes per launch (read + write) of the kernels, from the ncu captures summarised under
+# profiles/ (scaled to a full launch by the units processed); None until captured.
+NCU_TRAFFIC_BYTES = {"score": None, "attn_sparse": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------- clocks sampling
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the bench runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, uuid: str | None = None, period=0.05):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode() if uuid else b"")
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------- multi-rank aggregation (host)
+def reduce_max_ms(local_ms: float, dist, device) -> float:
+    """Max over ranks of a per-rank duration (the job is as slow as its slowest replica)."""
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, batch: int, steps: int, max_ms: float) -> float:
+    """Whole-job tokens/s: every rank decodes `batch` tokens per step (weak scaling)."""
+    return world * batch * steps / (max_ms * 1e-3)
+
+
+# ---------------------------------------------------------------------- the CPU oracle arm
+def oracle_throughput(w: W.Workload, steps: int, warmup: int, heads_per_step: int):
+    """Time the CPU oracle, unmodified, on a bounded sample of the workload.
+
+    One sequence of the batch is generated on the CPU; each step runs `heads_per_step` of its
+    heads through the oracle's decode step (retrieval on the first step of a block), and the
+    step time is scaled to the full batch x heads.  Returns (tokens/s, ms per scaled step,
+    threads, sample description).
+    """
+    from oracle import prhs_oracle as O
+    ws = w.scaled(batch=1, steps=warmup + steps)
+    k, v = W.make_kv(ws, "cpu")
+    q = W.make_queries(ws, "cpu")[0]
+    K, V, Q = k.float().numpy(), v.float().numpy(), q.float().numpy()
+    orc = O.PrhsOracle(O.Schedule(top_k=w.top_k, window=w.window, sinks=w.sinks,
+                                  refresh_interval=w.refresh, dilate_r=w.dilate_r), w.q_heads, w.kv_heads)
+    units = [(0, h) for h in range(min(heads_per_step, w.q_heads))]
+    scale = (w.batch * w.q_heads) / len(units)
+    total = 0.0
+    for n in range(warmup + steps):
+        t = W.seq_lens_at(ws, n).numpy()
+        t0 = time.perf_counter()
+        orc.decode_step(0, n, Q[n], K, V, t, units=units, want_delta=False)
+        dt = time.perf_counter() - t0
+        if n >= warmup:
+            total += dt * scale
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    sample = (f"{len(units)} of {w.batch * w.q_heads} (sequence, head) units per step, {steps} steps, "
+              f"time scaled by {scale:g}")
+    return w.batch * steps / total, 1e3 * total / steps, threads, sample
+
+
+def workload_config(w: W.Workload, extra=None):
+    cfg = {"workload": w.name, "layers": 1, "batch": w.batch, "q_heads": w.q_heads, "kv_heads": w.kv_heads,
+           "head_dim": 128, "context": w.context, "top_k": w.top_k, "window": w.window, "sinks": w.sinks,
+           "refresh_interval": w.refresh, "dilate_r": w.dilate_r, "dilate_m": "k/3",
+           "l2": "flushed between steps (256 MiB write outside the timed events); cache 4.3 GB >> L2"}
+    cfg.update(extra or {})
+    return cfg
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = W.C2_LLAMA2_7B
+    val, ms, threads, sample = oracle_throughput(w, args.steps, args.warmup, heads_per_step=8)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------- the CUDA arm
+def run_cuda(args):
+    from paper_2602_08329_b200 import binding as P
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    Wn, Kn = args.warmup, args.steps
+    total_steps = Wn + Kn
+    w = W.C2_LLAMA2_7B.scaled(steps=total_steps, seed=W.C2_LLAMA2_7B.seed + 97 * rank)
+    k, v = W.make_kv(w, dev)
+    q_all = W.make_queries(w, dev)[0]                     # [steps][B][Hq][128]
+    B, Hq, Hkv = w.batch, w.q_heads, w.kv_heads
+    ctx = P.Context(1, B, Hq, Hkv, w.capacity, w.top_k, w.window, w.sinks, max_dilate_r=w.dilate_r)
+    sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r)
+    t_all = torch.stack([W.seq_lens_at(w, n) for n in range(total_steps)]).to(dev)   # [steps][B]
+    views = [P.make_view(k, v, t_all[n], max_seq_len=w.capacity) for n in range(total_steps)]
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def timed_steps(first, count, fn):
+        """Run `count` steps; per-step CUDA events on the launching stream; L2 flushed between."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(count)]
+        for i in range(count):
+            flush.zero_()
+            evs[i][0].record(stream)
+            fn(first + i)
+            evs[i][1].record(stream)
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def step_device(n):
+        ctx.decode_step(0, n, sched, q_all[n], views[n], B, out)
+
+    # ---- warm-up, then the timed region
+    timed_steps(0, Wn, step_device)
+    sampler = ClockSampler(local, uuid=str(torch.cuda.get_device_properties(dev).uuid))
+    sampler.start()
+    launches0 = ctx.launch_count
+    barrier()
+    ctx.profile_begin(8 * Kn + 16)
+    ms = timed_steps(Wn, Kn, step_device)
+    prof = ctx.profile_end()
+    barrier()
+    launches = ctx.launch_count - launches0
+    clocks = sampler.stop()
+    assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+    total_ms = sum(ms)
+    total_ms_max = reduce_max_ms(total_ms, dist, dev)
+    value = job_throughput(world, B, Kn, total_ms_max)
+
+    refresh_ms = [m for i, m in enumerate(ms) if (Wn + i) % w.refresh == 0]
+    shared_ms = [m for i, m in enumerate(ms) if (Wn + i) % w.refresh != 0]
+
+    # ---- algorithmic bytes: K once on retrieval steps, gathered K/V rows on every step
+    counts = []
+    for n in range(Wn, Wn + Kn):                          # untimed replay to read the set sizes
+        step_device(n)
+        _, cnt = ctx.get_index_set(B)
+        counts.append(int(cnt.sum()))
+    t_cpu = t_all.cpu()
+    score_bytes = [int(t_cpu[n].sum()) * Hkv * 256 for n in range(Wn, Wn + Kn) if n % w.refresh == 0]
+    gather_bytes = [c * 512 for c in counts]
+    hbm_peak, peak_kind = load_peaks()
+    kernels = {}
+    for name, byts in (("score", score_bytes), ("attn_sparse", gather_bytes)):
+        kms, kn = prof.get(name, (0.0, 0))
+        if kn:
+            per_launch = sum(byts) / len(byts)
+            gbs = per_launch / (kms / kn * 1e-3) / 1e9
+            kernels[name] = {"launches": kn, "total_ms": kms, "avg_us": 1e3 * kms / kn,
+                             "algorithmic_bytes_per_launch": per_launch, "achieved_gbs": gbs,
+                             "frac_of_measured_peak": gbs / hbm_peak, "frac_of_8tbs": gbs / 8000.0}
+    for name in ("select", "build_set"):
+        kms, kn = prof.get(name, (0.0, 0))
+        if kn:
+            kernels[name] = {"launches": kn, "total_ms": kms, "avg_us": 1e3 * kms / kn}
+    dom = max((n for n in ("score", "attn_sparse") if n in kernels),
+              key=lambda n: kernels[n]["total_ms"])
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved_gbs"], "peak": hbm_peak,
+                "unit": "GB/s", "frac": kernels[dom]["achieved_gbs"] / hbm_peak,
+                "peak_source": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                "launches": kernels[dom]["launches"], "avg_us": kernels[dom]["avg_us"],
+                "algorithmic_bytes_per_launch": kernels[dom]["algorithmic_bytes_per_launch"]}
+    bytes_touched = sum(score_bytes) + sum(gather_bytes)
+    path_gbs = bytes_touched / (total_ms * 1e-3) / 1e9
+
+    # ---- in-library dense flash-decode baseline, same protocol
+    nd = min(4, Kn)
+    dense_ms = timed_steps(Wn, nd, lambda n: ctx.dense_decode_attn(q_all[n], views[n], B, out))
+    dense_us = 1e3 * statistics.median(dense_ms[1:] or dense_ms)
+    dense_bytes = int(t_cpu[Wn + nd - 1].sum()) * Hkv * 512
+
+    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
+    bi = torch.arange(B)
+    host = []
+    for n in range(Wn, Wn + Kn):
+        pos = (t_cpu[n] - 1).long()
+        host.append((q_all[n].cpu().pin_memory(), k[bi, :, pos].cpu().contiguous().pin_memory(),
+                     v[bi, :, pos].cpu().contiguous().pin_memory(), t_cpu[n].contiguous().pin_memory()))
+    host_out = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
+    t_scratch = torch.zeros(B, dtype=torch.int32, device=dev)
+    view_h = P.make_view(k, v, t_scratch, max_seq_len=w.capacity)
+
+    def step_host(n):
+        hq, hk, hv, ht = host[n - Wn]
+        ctx.decode_step_host(0, n, sched, hq, hk, hv, ht, view_h, B, host_out)
+
+    barrier()
+    e2e_ms = timed_steps(Wn, Kn, step_host)
+    barrier()
+    e2e_max_ms = reduce_max_ms(sum(e2e_ms), dist, dev)
+    e2e_value = job_throughput(world, B, Kn, e2e_max_ms)
+    h2d = B * Hq * 256 + 2 * B * Hkv * 256 + B * 4
+    d2h = B * Hq * 256
+
+    if rank != 0:
+        ctx.close()
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cval, cms, threads, sample = oracle_throughput(W.C2_LLAMA2_7B, steps=4 * w.refresh, warmup=0,
+                                                       heads_per_step=Hq)
+        cpu = {"value": cval, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+               "ms_per_step": cms}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": Kn, "warmup": Wn,
+        "ms_per_step": total_ms_max / Kn, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+        "config": workload_config(w, {"parallelism": f"replicas x{world} (no collective)"}),
+        "us_per_layer_step": 1e3 * total_ms_max / Kn,
+        "refresh_step_us": 1e3 * statistics.median(refresh_ms) if refresh_ms else None,
+        "shared_step_us": 1e3 * statistics.median(shared_ms) if shared_ms else None,
+        "dense_baseline_us_per_layer_step": dense_us,
+        "dense_baseline_gbs": dense_bytes / (dense_us * 1e-6) / 1e9,
+        "speedup_vs_dense_baseline": dense_us / (1e3 * total_ms / Kn),
+        "path_bytes_touched_per_step": bytes_touched / Kn,
+        "path_achieved_gbs": path_gbs, "path_frac_of_measured_peak": path_gbs / hbm_peak,
+        "path_frac_of_8tbs": path_gbs / 8000.0,
+        "mean_set_size": sum(counts) / (len(counts) * B * Hq),
+        "retrieval_ratio": len(score_bytes) / Kn,
+        "roofline": roofline, "kernels": kernels,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_max_ms / Kn},
+        "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        print("warning: fewer than 3 warm-up steps", file=sys.stderr)
+    return run_reference(args) if args.impl == "reference" else run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

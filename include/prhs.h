@@ -1,0 +1,250 @@
+/*
+ * prhs.h -- C ABI of the B200 sparse decode-attention library for Pre-hoc Sparsity
+ * (PrHS) with Clustered Indices Sharing (CIS).
+ *
+ * One decode step of one layer has three parts:
+ *   1. retrieval (first step of a block, first layer of a layer group only): score the
+ *      query against every cached key and select the exact top-k over the middle range;
+ *   2. index-set builder: sinks U (shared, dilated) middle set U recency window;
+ *   3. gathered split-K flash-decoding attention over the selected K/V rows only.
+ * A dropped-mass diagnostic (delta) reports how much softmax mass the selection lost.
+ *
+ * Conventions
+ *   - Positions are 0-based.  t_b = seq_lens[b] is the number of cached positions visible
+ *     to sequence b's current query, the current token (position t_b - 1) included.
+ *     sinks = [0, S0), middle candidates = [S0, t - W), local window = [t - W, t).
+ *   - head_dim is 128.  q, K, V and attention outputs are bf16; logits, log-sum-exps and
+ *     delta are fp32; indices and counts are int32.
+ *   - Query head h uses KV head h / (num_q_heads / num_kv_heads).  Index sets are per
+ *     (sequence, query head).
+ *   - "device" pointers are CUDA device memory owned by the caller unless stated; "host"
+ *     pointers are ordinary (preferably pinned) host memory.  The library never frees or
+ *     keeps caller memory beyond the call (asynchronous work on `stream` excepted).
+ *   - Every call validates its arguments on the host and returns a prhs_status; nothing
+ *     traps, asserts or spins on the device.  Device-side anomalies (an index outside
+ *     [0, t_b), a candidate overflow) are recorded in a flag word read by prhs_check().
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default
+ *     stream) and is asynchronous unless stated.  Workspaces and the shared-set state are
+ *     allocated in prhs_create(); no call below allocates.
+ *   - A context must be used from one host thread at a time and on one stream at a time.
+ */
+#ifndef PRHS_H_
+#define PRHS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct prhs_ctx prhs_ctx;
+
+typedef enum {
+  PRHS_OK = 0,
+  PRHS_ERR_INVALID_ARG = 1, /* NULL pointer, bad shape, value out of the configured range */
+  PRHS_ERR_UNSUPPORTED = 2, /* head_dim != 128, page_size not in {0,16}, group size > 16   */
+  PRHS_ERR_OOM = 3,         /* prhs_create could not allocate its workspaces               */
+  PRHS_ERR_CUDA = 4,        /* a CUDA runtime call failed; see prhs_last_error             */
+  PRHS_ERR_STATE = 5,       /* no shared set for this block/group (leader not called yet)   */
+  PRHS_ERR_CAPACITY = 6,    /* batch, k, window, ... exceed what prhs_create was given      */
+  PRHS_ERR_DEVICE_FLAG = 7  /* prhs_check: a kernel recorded an anomaly                    */
+} prhs_status;
+
+/* Sizes fixed at prhs_create(); workspaces are dimensioned from them. */
+typedef struct {
+  int32_t num_layers;    /* layers whose shared sets are kept (groups = ceil(L / layer_group)) */
+  int32_t max_batch;     /* B */
+  int32_t num_q_heads;   /* Hq */
+  int32_t num_kv_heads;  /* Hkv, divides Hq; Hq / Hkv <= 16 */
+  int32_t head_dim;      /* must be 128 */
+  int32_t max_context;   /* largest t_b ever passed (cache capacity in positions), <= 2^20 */
+  int32_t page_size;     /* 0 = contiguous cache, 16 = paged cache */
+  int32_t max_k;         /* largest middle budget k */
+  int32_t max_window;    /* largest recency window W */
+  int32_t max_sinks;     /* largest sink count S0 */
+  int32_t max_dilate_r;  /* largest dilation radius r */
+  int32_t max_dilate_m;  /* largest number of dilated winners m; -1 = floor(max_k / 3) */
+  int32_t min_layer_group; /* smallest layer_group that will be used (sizes the state); >= 1 */
+} prhs_config;
+
+/* A view of one layer's KV cache (device memory, bf16, caller-owned).
+ *   contiguous (page_table == NULL): row i of (b, kvh) is at
+ *        k + b*stride_outer + kvh*stride_head + i*128            (element offsets)
+ *   paged (page_table != NULL, 16 positions per page): row i of (b, kvh) is at
+ *        k + page_table[b*page_table_stride + i/16]*stride_outer + kvh*stride_head + (i%16)*128
+ * Rows are 128 contiguous bf16 (256 bytes); k, v and every stride must keep rows 16-byte
+ * aligned (strides multiples of 8 elements). */
+typedef struct {
+  const void* k;
+  const void* v;
+  int64_t stride_outer;
+  int64_t stride_head;
+  const int32_t* page_table; /* device [B][page_table_stride] or NULL */
+  int32_t page_table_stride;
+  const int32_t* seq_lens;   /* device [B]: t_b, current token included; 0 <= t_b <= max_seq_len */
+  int32_t max_seq_len;       /* host-side upper bound of every t_b (sizes the launch); 0 = max_context */
+  int32_t num_pages;         /* paged: pages in the pool (bounds check); contiguous: ignored */
+} prhs_kv_view;
+
+/* Schedule flags */
+#define PRHS_DILATE_ANCHOR 1u /* the retrieving (layer, step) also attends over the dilated set */
+#define PRHS_WANT_DELTA    2u /* prhs_decode_step fills out_delta (runs a dense log-sum-exp pass
+                                 on every non-retrieving call: diagnostic, not the timed path)  */
+
+/* The knobs of CIS (Sec. 4.1; defaults Sec. 5.1) plus the cross-layer group size. */
+typedef struct {
+  int32_t refresh_interval;     /* s: block size in decode steps; step % s == 0 retrieves; >= 1 */
+  int32_t layer_group;          /* G_L: layers [g*G_L, (g+1)*G_L) reuse layer g*G_L's set; 1 = off */
+  int32_t top_k;                /* k: middle budget; ignored where top_k_per_seq != NULL        */
+  const int32_t* top_k_per_seq; /* device [B] or NULL; every entry <= max_k                     */
+  int32_t window;               /* W = C_local */
+  int32_t sinks;                /* S0 = C_sink */
+  int32_t dilate_r;             /* r of Eq. 10 */
+  int32_t dilate_m;             /* m of Eq. 10; -1 = floor(k / 3) per sequence                  */
+  uint32_t flags;
+} prhs_schedule;
+
+/* Create / destroy a context on the current CUDA device.  prhs_create allocates every
+ * workspace (scores, split-K partials, index lists) and the shared-set state; it returns
+ * PRHS_ERR_OOM and leaves *out NULL if the device cannot hold them.  Synchronous. */
+prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out);
+prhs_status prhs_destroy(prhs_ctx* ctx);
+
+/* Retrieval pass (Sec. 2.3 "Top-k Oracle"; Sec. 4.1 "Selection Criteria"; Eq. 10).
+ * For every (b, h): logits a_i = q_h . k_i / sqrt(128) over i < t_b (Eq. 2); S* = the
+ * min(k_b, t_b - W - S0) middle candidates of largest logit, ordered by descending logit,
+ * equal logits by ascending position; S^ = S* U { p + j : p among the first m of S*,
+ * |j| <= r } clipped to [0, t_b).  S* and S^ are stored in the context as the shared set
+ * of `layer`'s group, anchored at `step`.
+ *   q            device bf16 [batch][Hq][128]
+ *   out_idx      device int32 [batch][Hq][max_k] or NULL: S* in descending-logit order,
+ *                entries past the count are -1
+ *   out_count    device int32 [batch][Hq] or NULL: |S*|
+ *   out_lse_full device fp32 [batch][Hq] or NULL: log sum_{i<t_b} exp(a_i)
+ * `layer` must be the first layer of its group. */
+prhs_status prhs_score_topk(prhs_ctx* ctx, int32_t layer, int32_t step, const void* q,
+                            const prhs_kv_view* kv, const prhs_schedule* sched, int32_t batch,
+                            int32_t* out_idx, int32_t* out_count, float* out_lse_full,
+                            void* stream);
+
+/* Index-set builder (Sec. 4.1: C_t = sinks U middle U local; Def. 3.2 key-value sharing).
+ * C = [0, min(S0,t)) U M U [max(0,t-W), t) at the CURRENT t_b, ascending and unique, where
+ * M = S* if (layer, step) is the retrieving call itself and PRHS_DILATE_ANCHOR is off,
+ * else M = S^ of the group's anchor.  PRHS_ERR_STATE if the group has no set anchored at
+ * step - step % s.
+ *   out_idx   device int32 [batch][Hq][idx_stride], idx_stride >= prhs_index_capacity()
+ *   out_count device int32 [batch][Hq] */
+prhs_status prhs_build_index_set(prhs_ctx* ctx, int32_t layer, int32_t step,
+                                 const prhs_schedule* sched, const prhs_kv_view* kv, int32_t batch,
+                                 int32_t* out_idx, int32_t idx_stride, int32_t* out_count,
+                                 void* stream);
+
+/* Token-sparse attention (Def. 3.1): for every (b, h), softmax attention of q_h restricted
+ * to the rows idx[b][h][0..count) of the cache and renormalised over them, computed as
+ * split-K online softmax followed by a merge.
+ *   idx      device int32 [batch][Hq][idx_stride], each entry in [0, t_b); order is free,
+ *            ascending order gathers fastest; duplicates are attended twice
+ *   count    device int32 [batch][Hq]; 0 gives a zero output row and lse = -inf
+ *   out      device bf16 [batch][Hq][128]
+ *   out_lse  device fp32 [batch][Hq] or NULL: log sum_{i in C} exp(a_i)
+ * An index outside [0, t_b) is skipped and recorded in the device flag word. */
+prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,
+                                    const int32_t* idx, const int32_t* count, int32_t idx_stride,
+                                    int32_t batch, void* out, float* out_lse, void* stream);
+
+/* Dense flash-decoding baseline (Eq. 2): attention over all i < t_b. Same outputs. */
+prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,
+                                   int32_t batch, void* out, float* out_lse, void* stream);
+
+/* One (layer, step) of the schedule (Sec. 4.4 "Parallel Acceleration": retrieval for heads
+ * that need it, cached sets for the rest, attention over valid indices only).
+ * Retrieves iff layer % G_L == 0 and step % s == 0; then builds the set and attends.
+ * Within a step a group's first layer must be called before its other layers.
+ *   out        device bf16 [batch][Hq][128]
+ *   out_delta  device fp32 [batch][Hq] or NULL (used only with PRHS_WANT_DELTA) */
+prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                             const void* q, const prhs_kv_view* kv, int32_t batch, void* out,
+                             float* out_delta, void* stream);
+
+/* The same step for a caller whose per-step tensors live in HOST memory (contiguous cache
+ * only).  Copies q, the new token's key and value rows and seq_lens host->device, writes
+ * the rows into the cache at position t_b - 1, runs prhs_decode_step, copies the output
+ * device->host and synchronises the stream before returning.
+ *   host_q [batch][Hq][128], host_new_k / host_new_v [batch][Hkv][128], host_out
+ *   [batch][Hq][128]: bf16 host memory;  host_seq_lens [batch] int32 host memory.
+ *   kv->k / kv->v are written (the view's const is cast away); kv->seq_lens must point to
+ *   a device int32 [batch] buffer that this call overwrites. */
+prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step,
+                                  const prhs_schedule* sched, const void* host_q,
+                                  const void* host_new_k, const void* host_new_v,
+                                  const int32_t* host_seq_lens, const prhs_kv_view* kv,
+                                  int32_t batch, void* host_out, void* stream);
+
+/* Dropped mass (Sec. 2.3): delta = 1 - sum_{i in C} A_i with A the full softmax over
+ * i < t_b.  Runs a dense log-sum-exp pass and a sparse pass.  out_delta device fp32
+ * [batch][Hq]. */
+prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, const int32_t* idx,
+                       const int32_t* count, int32_t idx_stride, int32_t batch, float* out_delta,
+                       void* stream);
+
+/* Largest index-list length any call can produce: S0 + k + 2*r*m + W from prhs_config. */
+int32_t prhs_index_capacity(const prhs_ctx* ctx);
+
+/* Copy the set the last prhs_decode_step / prhs_build_index_set(ctx-internal) produced to
+ * the host: host_idx int32 [batch][Hq][prhs_index_capacity()], host_count int32
+ * [batch][Hq].  Synchronous; for tests and diagnostics. */
+prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx,
+                               int32_t* host_count, void* stream);
+
+/* Copy the stored shared sets of `layer`'s group to the host: host_s_star (descending
+ * logit) [batch][Hq][max_k], host_s_hat (ascending) [batch][Hq][max_k + 2*r*m], their
+ * counts [batch][Hq] each.  Any pointer may be NULL.  Synchronous. */
+prhs_status prhs_get_shared_set(prhs_ctx* ctx, int32_t layer, int32_t batch, int32_t* host_s_star,
+                                int32_t* host_n_star, int32_t* host_s_hat, int32_t* host_n_hat,
+                                void* stream);
+
+/* Copy the logits of the last retrieval pass to the host: fp32 [batch][Hq][ld] with
+ * ld = prhs_scores_ld().  Synchronous; for tests. */
+prhs_status prhs_get_scores(prhs_ctx* ctx, int32_t batch, float* host_scores, void* stream);
+int32_t prhs_scores_ld(const prhs_ctx* ctx);
+
+/* Synchronise `stream` and report: PRHS_ERR_CUDA on an asynchronous CUDA error,
+ * PRHS_ERR_DEVICE_FLAG if a kernel recorded an anomaly (the flag word is then cleared;
+ * *out_flags, if not NULL, receives it), else PRHS_OK. */
+#define PRHS_FLAG_BAD_INDEX       1u /* an index outside [0, t_b) was skipped                */
+#define PRHS_FLAG_BAD_PAGE        2u /* a page id outside [0, num_pages) was skipped          */
+#define PRHS_FLAG_SELECT_FALLBACK 4u /* informational: selection took the multi-pass path     */
+prhs_status prhs_check(prhs_ctx* ctx, void* stream, uint32_t* out_flags);
+
+/* Per-kernel device timing for benchmarks (no counterpart in the paper: measurement support).
+ * Between prhs_profile_begin and prhs_profile_end every kernel launch of the context is
+ * bracketed by a pair of CUDA events on its stream (at most max_launches launches; later
+ * ones are not recorded).  prhs_profile_end synchronises `stream` and sums the elapsed
+ * milliseconds and the launch counts per kernel kind into host arrays of
+ * PRHS_KERNEL_KINDS entries.  Events are created in prhs_profile_begin, not per launch. */
+#define PRHS_KERNEL_KINDS 6
+#define PRHS_KIND_SCORE 0        /* dense scoring (retrieval, or the delta diagnostic)  */
+#define PRHS_KIND_SELECT 1       /* top-k selection + dilation                         */
+#define PRHS_KIND_BUILD 2        /* index-set builder                                  */
+#define PRHS_KIND_ATTN_SPARSE 3  /* gathered attention + merge                         */
+#define PRHS_KIND_ATTN_DENSE 4   /* dense flash-decoding baseline                      */
+#define PRHS_KIND_MISC 5         /* row append, log-sum-exp reduction                  */
+prhs_status prhs_profile_begin(prhs_ctx* ctx, int32_t max_launches);
+prhs_status prhs_profile_end(prhs_ctx* ctx, void* stream, float* host_ms_per_kind,
+                             int64_t* host_launches_per_kind);
+const char* prhs_kernel_kind_name(int32_t kind);
+
+/* Number of kernels this context has launched since creation (host-side counter). */
+int64_t prhs_launch_count(const prhs_ctx* ctx);
+
+/* Message of the last error on this context (or of the last failed prhs_create when ctx is
+ * NULL).  The pointer stays valid until the next call on the context. */
+const char* prhs_last_error(const prhs_ctx* ctx);
+
+/* Library version string. */
+const char* prhs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRHS_H_ */

@@ -1,0 +1,96 @@
+// Shared device helpers for the PrHS sparse decode-attention kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace prhs {
+
+constexpr int kHeadDim = 128;              // elements per K/V row
+constexpr int kRowBytes = kHeadDim * 2;    // 256 B per bf16 row
+constexpr int kPageShift = 4;              // 16 positions per page
+constexpr float kScale = 0.08838834764831845f;        // 1 / sqrt(128)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+constexpr uint32_t kFlagBadIndex = 1u;
+constexpr uint32_t kFlagBadPage = 2u;
+constexpr uint32_t kFlagSelectFallback = 4u;
+
+// Device-side copy of a KV view (see prhs_kv_view): element strides, optional page table.
+struct KvDev {
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  long long stride_outer;
+  long long stride_head;
+  const int* page_table;
+  int page_table_stride;
+  const int* seq_lens;
+  int num_pages;
+};
+
+// Element offset of row `i` of (b, kvh); -1 (and a flag) for a page id out of range.
+__device__ __forceinline__ long long row_offset(const KvDev& kv, int b, int kvh, int i,
+                                                uint32_t* flags) {
+  if (kv.page_table != nullptr) {
+    int page = __ldg(kv.page_table + (long long)b * kv.page_table_stride + (i >> kPageShift));
+    if ((unsigned)page >= (unsigned)kv.num_pages) {
+      atomicOr(flags, kFlagBadPage);
+      return -1;
+    }
+    return (long long)page * kv.stride_outer + (long long)kvh * kv.stride_head +
+           (long long)(i & ((1 << kPageShift) - 1)) * kHeadDim;
+  }
+  return (long long)b * kv.stride_outer + (long long)kvh * kv.stride_head + (long long)i * kHeadDim;
+}
+
+// bf16 pair (packed in 32 bits) -> two floats; exact.
+__device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+// 16-byte read-only load that does not allocate in L1 (streamed once).
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+// Dot product of 8 bf16 (one uint4) with 8 floats.
+__device__ __forceinline__ float dot8(const uint4& kx, const float* q) {
+  float s = bf_lo(kx.x) * q[0];
+  s = fmaf(bf_hi(kx.x), q[1], s);
+  s = fmaf(bf_lo(kx.y), q[2], s);
+  s = fmaf(bf_hi(kx.y), q[3], s);
+  s = fmaf(bf_lo(kx.z), q[4], s);
+  s = fmaf(bf_hi(kx.z), q[5], s);
+  s = fmaf(bf_lo(kx.w), q[6], s);
+  s = fmaf(bf_hi(kx.w), q[7], s);
+  return s;
+}
+
+// Sum over the 16 lanes of a half-warp (all 16 lanes receive the total).
+__device__ __forceinline__ float half_warp_sum(float s) {
+  s += __shfl_xor_sync(0xffffffffu, s, 8);
+  s += __shfl_xor_sync(0xffffffffu, s, 4);
+  s += __shfl_xor_sync(0xffffffffu, s, 2);
+  s += __shfl_xor_sync(0xffffffffu, s, 1);
+  return s;
+}
+
+// Order-preserving map fp32 -> uint32: larger float <=> larger key (-0 < +0, NaNs at the ends).
+__device__ __forceinline__ uint32_t float_to_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Combine two online-softmax states kept in the log2 domain: (m, l) <- (m, l) (+) (m2, l2).
+__device__ __forceinline__ void ml_combine(float& m, float& l, float m2, float l2) {
+  float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) return;
+  l = l * exp2f(m - mn) + l2 * exp2f(m2 - mn);
+  m = mn;
+}
+
+}  // namespace prhs

@@ -1,0 +1,674 @@
+// Host side of the PrHS sparse decode-attention library: context, argument validation,
+// launch configuration and the C ABI declared in include/prhs.h.
+#include "../../include/prhs.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "attn.cuh"
+#include "common.cuh"
+#include "score.cuh"
+#include "select.cuh"
+
+using namespace prhs;
+
+namespace {
+
+constexpr int kChunkRows = 2048;        // keys scored per CTA (multiple of kScoreRowsPerIter)
+constexpr int kMaxSplits = 64;          // split-K partial slots per (b, h)
+constexpr int kMaxSmemBytes = 227 * 1024;
+constexpr int kMaxContext = 1 << 20;
+
+std::string g_create_error;
+
+}  // namespace
+
+struct prhs_ctx {
+  prhs_config cfg{};
+  int device = 0, sm_count = 148;
+  int gq = 1, num_groups = 1, max_m = 0, shat_cap = 0, idx_cap = 0, ld = 0, sort_cap = 2;
+  int max_chunks = 1, resident_cap = 0;
+  size_t sel_smem = 0;
+  // workspaces (device)
+  float* scores = nullptr;
+  float2* part_ml = nullptr;
+  float* lse_full = nullptr;
+  float* lse_c = nullptr;
+  float* partials = nullptr;
+  unsigned int* tickets = nullptr;
+  int* idx = nullptr;
+  int* count = nullptr;
+  uint32_t* flags = nullptr;
+  __nv_bfloat16* scratch_out = nullptr;
+  // shared-set state (device), per layer group
+  int *sstar_desc = nullptr, *sstar_asc = nullptr, *shat_asc = nullptr;
+  int *n_star = nullptr, *n_hat = nullptr, *anchor_t = nullptr;
+  std::vector<int> anchor_step;     // host: step at which each group last retrieved, -1 = never
+  // staging for the host-buffer entry point (device)
+  __nv_bfloat16 *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_out = nullptr;
+  int last_batch = 0, last_layer_group = 1;
+  long long launches = 0;
+  // optional per-launch event timing
+  struct ProfRec { cudaEvent_t a, b; int kind; };
+  std::vector<ProfRec> prof;
+  int prof_used = 0;
+  bool prof_on = false;
+  std::string err;
+};
+
+namespace {
+
+prhs_status fail(prhs_ctx* ctx, prhs_status st, const std::string& msg) {
+  if (ctx) ctx->err = msg; else g_create_error = msg;
+  return st;
+}
+
+#define PRHS_CUDA(ctx, expr)                                                              \
+  do {                                                                                    \
+    cudaError_t e_ = (expr);                                                              \
+    if (e_ != cudaSuccess)                                                                \
+      return fail(ctx, PRHS_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t n) {
+  return cudaMalloc(reinterpret_cast<void**>(p), std::max<size_t>(n, 1) * sizeof(T));
+}
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+size_t units_max(const prhs_ctx* c) { return (size_t)c->cfg.max_batch * c->cfg.num_q_heads; }
+
+prhs_status check_view(prhs_ctx* ctx, const prhs_kv_view* kv, int batch, KvDev* out, int* max_t) {
+  if (!kv || !kv->k || !kv->v || !kv->seq_lens) return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: NULL pointer");
+  if (batch < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "batch must be >= 1");
+  if (batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch exceeds max_batch");
+  if ((kv->stride_outer % 8) || (kv->stride_head % 8) || ((uintptr_t)kv->k % 16) || ((uintptr_t)kv->v % 16))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: rows must be 16-byte aligned");
+  if (kv->stride_outer <= 0 || kv->stride_head <= 0)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: strides must be positive");
+  const bool paged = kv->page_table != nullptr;
+  if (paged != (ctx->cfg.page_size == 16))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: page table does not match the configured page_size");
+  if (paged && (kv->page_table_stride < 1 || kv->num_pages < 1))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: bad page table stride or pool size");
+  int mt = kv->max_seq_len > 0 ? kv->max_seq_len : ctx->cfg.max_context;
+  if (mt > ctx->cfg.max_context) return fail(ctx, PRHS_ERR_CAPACITY, "max_seq_len exceeds max_context");
+  out->k = static_cast<const __nv_bfloat16*>(kv->k);
+  out->v = static_cast<const __nv_bfloat16*>(kv->v);
+  out->stride_outer = kv->stride_outer;
+  out->stride_head = kv->stride_head;
+  out->page_table = kv->page_table;
+  out->page_table_stride = kv->page_table_stride;
+  out->seq_lens = kv->seq_lens;
+  out->num_pages = kv->num_pages;
+  *max_t = mt;
+  return PRHS_OK;
+}
+
+prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
+  if (!s) return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: NULL");
+  if (s->refresh_interval < 1 || s->layer_group < 1)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: refresh_interval and layer_group must be >= 1");
+  if (s->layer_group < ctx->cfg.min_layer_group)
+    return fail(ctx, PRHS_ERR_CAPACITY, "schedule: layer_group below min_layer_group");
+  if (s->top_k < 0 || s->window < 0 || s->sinks < 0 || s->dilate_r < 0 || s->dilate_m < -1)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: negative budget");
+  if (s->top_k > ctx->cfg.max_k || s->window > ctx->cfg.max_window || s->sinks > ctx->cfg.max_sinks ||
+      s->dilate_r > ctx->cfg.max_dilate_r || (s->dilate_m >= 0 && s->dilate_m > ctx->max_m))
+    return fail(ctx, PRHS_ERR_CAPACITY, "schedule: budget exceeds the configured maximum");
+  return PRHS_OK;
+}
+
+// Brackets one kernel launch: counts it and, in profiling mode, records an event pair.
+struct LaunchScope {
+  prhs_ctx* c;
+  cudaStream_t st;
+  int slot = -1;
+  LaunchScope(prhs_ctx* ctx, int kind, cudaStream_t stream) : c(ctx), st(stream) {
+    c->launches++;
+    if (c->prof_on && c->prof_used < (int)c->prof.size()) {
+      slot = c->prof_used++;
+      c->prof[slot].kind = kind;
+      cudaEventRecord(c->prof[slot].a, st);
+    }
+  }
+  ~LaunchScope() {
+    if (slot >= 0) cudaEventRecord(c->prof[slot].b, st);
+  }
+};
+
+// ---- launchers -----------------------------------------------------------------------
+template <int GQ>
+void launch_score_t(prhs_ctx* c, const __nv_bfloat16* q, const KvDev& kv, int batch, int nchunks,
+                    int write_scores, cudaStream_t st) {
+  dim3 grid(nchunks, c->cfg.num_q_heads / GQ, batch);
+  score_kernel<GQ><<<grid, kScoreThreads, 0, st>>>(q, kv, c->scores, c->ld, c->part_ml, nchunks,
+                                                   kChunkRows, c->cfg.num_q_heads, c->gq,
+                                                   write_scores, c->flags);
+}
+
+prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
+                         int write_scores, cudaStream_t st, int* nchunks_out) {
+  const int nchunks = std::max(1, (max_t + kChunkRows - 1) / kChunkRows);
+  const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
+  {
+    LaunchScope ls(c, PRHS_KIND_SCORE, st);
+    if (c->gq % 8 == 0) launch_score_t<8>(c, qq, kv, batch, nchunks, write_scores, st);
+    else if (c->gq % 4 == 0) launch_score_t<4>(c, qq, kv, batch, nchunks, write_scores, st);
+    else if (c->gq % 2 == 0) launch_score_t<2>(c, qq, kv, batch, nchunks, write_scores, st);
+    else launch_score_t<1>(c, qq, kv, batch, nchunks, write_scores, st);
+  }
+  *nchunks_out = nchunks;
+  PRHS_CUDA(c, cudaGetLastError());
+  return PRHS_OK;
+}
+
+int pick_splits(const prhs_ctx* c, int units, int max_count) {
+  const int target = c->sm_count * 8;
+  int s = (target + units - 1) / units;
+  s = std::min(s, std::max(1, (max_count + 63) / 64));
+  return std::max(1, std::min(s, kMaxSplits));
+}
+
+prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
+                        int idx_stride, int max_count, int batch, void* out, float* out_lse,
+                        const float* lse_full, float* out_delta, cudaStream_t st) {
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.kv = kv;
+  p.idx = idx;
+  p.count = count;
+  p.idx_stride = idx ? idx_stride : 0x7fffffff;
+  p.num_q_heads = c->cfg.num_q_heads;
+  p.group_size = c->gq;
+  p.splits = pick_splits(c, batch * c->cfg.num_q_heads, max_count);
+  p.partials = c->partials;
+  p.tickets = c->tickets;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.out_lse = out_lse;
+  p.lse_full = lse_full;
+  p.out_delta = lse_full ? out_delta : nullptr;
+  p.flags = c->flags;
+  dim3 grid(p.splits, c->cfg.num_q_heads, batch);
+  {
+    LaunchScope ls(c, idx ? PRHS_KIND_ATTN_SPARSE : PRHS_KIND_ATTN_DENSE, st);
+    gather_attn_kernel<<<grid, kAttnThreads, 0, st>>>(p);
+  }
+  PRHS_CUDA(c, cudaGetLastError());
+  return PRHS_OK;
+}
+
+int group_of(const prhs_schedule* s, int layer) { return layer / s->layer_group; }
+
+size_t state_off(const prhs_ctx* c, int group, size_t per_unit) {
+  return (size_t)group * units_max(c) * per_unit;
+}
+
+prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const KvDev& kv, int max_t,
+                         const prhs_schedule* s, int batch, int32_t* out_idx, int32_t* out_count,
+                         float* out_lse_full, cudaStream_t st) {
+  const int g = group_of(s, layer);
+  int nchunks = 1;
+  prhs_status rc = launch_score(c, q, kv, batch, max_t, 1, st, &nchunks);
+  if (rc != PRHS_OK) return rc;
+  SelectParams p;
+  p.scores = c->scores;
+  p.ld = c->ld;
+  p.part_ml = c->part_ml;
+  p.nchunks = nchunks;
+  p.seq_lens = kv.seq_lens;
+  p.k_per_seq = s->top_k_per_seq;
+  p.k = s->top_k;
+  p.sinks = s->sinks;
+  p.window = s->window;
+  p.r = s->dilate_r;
+  p.m = s->dilate_m;
+  p.max_k = c->cfg.max_k;
+  p.shat_cap = c->shat_cap;
+  p.num_q_heads = c->cfg.num_q_heads;
+  p.sstar_desc = c->sstar_desc + state_off(c, g, c->cfg.max_k);
+  p.sstar_asc = c->sstar_asc + state_off(c, g, c->cfg.max_k);
+  p.shat_asc = c->shat_asc + state_off(c, g, c->shat_cap);
+  p.n_star = c->n_star + state_off(c, g, 1);
+  p.n_hat = c->n_hat + state_off(c, g, 1);
+  p.anchor_t = c->anchor_t + (size_t)g * c->cfg.max_batch;
+  p.out_idx = out_idx;
+  p.out_count = out_count;
+  p.lse_full = c->lse_full;
+  p.out_lse_full = out_lse_full;
+  p.flags = c->flags;
+  p.sort_cap = c->sort_cap;
+  p.resident_cap = c->resident_cap;
+  {
+    LaunchScope ls(c, PRHS_KIND_SELECT, st);
+    select_kernel<<<batch * c->cfg.num_q_heads, kSelThreads, c->sel_smem, st>>>(p);
+  }
+  PRHS_CUDA(c, cudaGetLastError());
+  c->anchor_step[g] = step;
+  c->last_layer_group = s->layer_group;
+  return PRHS_OK;
+}
+
+prhs_status do_build(prhs_ctx* c, int layer, int step, const prhs_schedule* s, const KvDev& kv,
+                     int batch, int32_t* out_idx, int idx_stride, int32_t* out_count,
+                     cudaStream_t st) {
+  const int g = group_of(s, layer);
+  const int anchor = step - step % s->refresh_interval;
+  if (c->anchor_step[g] != anchor)
+    return fail(c, PRHS_ERR_STATE, "no shared set for this block: the group's first layer has not retrieved");
+  const bool own = (layer % s->layer_group == 0) && (step == anchor) && !(s->flags & PRHS_DILATE_ANCHOR);
+  const int* mid = own ? c->sstar_asc + state_off(c, g, c->cfg.max_k)
+                       : c->shat_asc + state_off(c, g, c->shat_cap);
+  const int* nmid = (own ? c->n_star : c->n_hat) + state_off(c, g, 1);
+  {
+    LaunchScope ls(c, PRHS_KIND_BUILD, st);
+    build_set_kernel<<<batch * c->cfg.num_q_heads, 128, 0, st>>>(
+        mid, nmid, own ? c->cfg.max_k : c->shat_cap, kv.seq_lens, s->sinks, s->window,
+        c->cfg.num_q_heads, out_idx, idx_stride, out_count);
+  }
+  PRHS_CUDA(c, cudaGetLastError());
+  return PRHS_OK;
+}
+
+prhs_status check_layer(prhs_ctx* c, int layer, int step, const prhs_schedule* s) {
+  if (layer < 0 || layer >= c->cfg.num_layers) return fail(c, PRHS_ERR_INVALID_ARG, "layer out of range");
+  if (step < 0) return fail(c, PRHS_ERR_INVALID_ARG, "step must be >= 0");
+  if (group_of(s, layer) >= c->num_groups) return fail(c, PRHS_ERR_CAPACITY, "layer group out of range");
+  return PRHS_OK;
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+const char* prhs_version(void) { return "prhs-b200 0.1"; }
+
+const char* prhs_last_error(const prhs_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+int64_t prhs_launch_count(const prhs_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t prhs_index_capacity(const prhs_ctx* ctx) { return ctx ? ctx->idx_cap : 0; }
+
+int32_t prhs_scores_ld(const prhs_ctx* ctx) { return ctx ? ctx->ld : 0; }
+
+prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !out) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: NULL argument");
+  if (cfg->head_dim != kHeadDim) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "head_dim must be 128");
+  if (cfg->page_size != 0 && cfg->page_size != 16)
+    return fail(nullptr, PRHS_ERR_UNSUPPORTED, "page_size must be 0 or 16");
+  if (cfg->num_layers < 1 || cfg->max_batch < 1 || cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 ||
+      cfg->max_context < 1 || cfg->max_k < 0 || cfg->max_window < 0 || cfg->max_sinks < 0 ||
+      cfg->max_dilate_r < 0 || cfg->max_dilate_m < -1 || cfg->min_layer_group < 1)
+    return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: non-positive size");
+  if (cfg->num_q_heads % cfg->num_kv_heads) return fail(nullptr, PRHS_ERR_INVALID_ARG, "Hkv must divide Hq");
+  if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
+  if (cfg->max_context > kMaxContext) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context above 2^20");
+  if (cfg->max_k > 65536) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_k above 65536");
+
+  prhs_ctx* c = new (std::nothrow) prhs_ctx();
+  if (!c) return fail(nullptr, PRHS_ERR_OOM, "host allocation failed");
+  c->cfg = *cfg;
+  c->gq = cfg->num_q_heads / cfg->num_kv_heads;
+  c->num_groups = (cfg->num_layers + cfg->min_layer_group - 1) / cfg->min_layer_group;
+  c->max_m = cfg->max_dilate_m < 0 ? cfg->max_k / 3 : cfg->max_dilate_m;
+  c->shat_cap = cfg->max_k + 2 * cfg->max_dilate_r * c->max_m;
+  c->idx_cap = cfg->max_sinks + c->shat_cap + cfg->max_window;
+  c->ld = (cfg->max_context + 63) & ~63;
+  c->max_chunks = (cfg->max_context + kChunkRows - 1) / kChunkRows;
+  while (c->sort_cap < cfg->max_k) c->sort_cap <<= 1;
+  c->anchor_step.assign(c->num_groups, -1);
+
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+  if (e != cudaSuccess) {
+    std::string msg = std::string("no usable CUDA device: ") + cudaGetErrorString(e);
+    delete c;
+    return fail(nullptr, PRHS_ERR_CUDA, msg);
+  }
+  // selection kernel shared memory: header + sort buffer + max(resident keys, position bitmap)
+  const int fixed = kSelHeaderWords * 4 + c->sort_cap * 8;
+  const int bitmap_words = (cfg->max_context + 31) / 32;
+  const int avail_words = (kMaxSmemBytes - fixed) / 4;
+  if (avail_words < bitmap_words) {
+    delete c;
+    return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context / max_k too large for the selection kernel");
+  }
+  c->resident_cap = std::min(cfg->max_context, avail_words);
+  c->sel_smem = (size_t)fixed + 4 * (size_t)std::max(bitmap_words, c->resident_cap);
+  e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
+
+  const size_t U = units_max(c), G = c->num_groups;
+  if (e == cudaSuccess) e = dev_alloc(&c->scores, U * c->ld);
+  if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * c->max_chunks);
+  if (e == cudaSuccess) e = dev_alloc(&c->lse_full, U);
+  if (e == cudaSuccess) e = dev_alloc(&c->lse_c, U);
+  if (e == cudaSuccess) e = dev_alloc(&c->partials, U * kMaxSplits * kPartStride);
+  if (e == cudaSuccess) e = dev_alloc(&c->tickets, U);
+  if (e == cudaSuccess) e = dev_alloc(&c->idx, U * c->idx_cap);
+  if (e == cudaSuccess) e = dev_alloc(&c->count, U);
+  if (e == cudaSuccess) e = dev_alloc(&c->flags, 1);
+  if (e == cudaSuccess) e = dev_alloc(&c->scratch_out, U * kHeadDim);
+  if (e == cudaSuccess) e = dev_alloc(&c->sstar_desc, G * U * cfg->max_k);
+  if (e == cudaSuccess) e = dev_alloc(&c->sstar_asc, G * U * cfg->max_k);
+  if (e == cudaSuccess) e = dev_alloc(&c->shat_asc, G * U * c->shat_cap);
+  if (e == cudaSuccess) e = dev_alloc(&c->n_star, G * U);
+  if (e == cudaSuccess) e = dev_alloc(&c->n_hat, G * U);
+  if (e == cudaSuccess) e = dev_alloc(&c->anchor_t, G * cfg->max_batch);
+  if (e == cudaSuccess) e = dev_alloc(&c->st_q, U * kHeadDim);
+  if (e == cudaSuccess) e = dev_alloc(&c->st_out, U * kHeadDim);
+  if (e == cudaSuccess) e = dev_alloc(&c->st_k, (size_t)cfg->max_batch * cfg->num_kv_heads * kHeadDim);
+  if (e == cudaSuccess) e = dev_alloc(&c->st_v, (size_t)cfg->max_batch * cfg->num_kv_heads * kHeadDim);
+  if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, U * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(c->flags, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(c->n_star, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->n_hat, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->count, 0, U * sizeof(int));
+  if (e != cudaSuccess) {
+    std::string msg = std::string("prhs_create: ") + cudaGetErrorString(e);
+    const bool oom = (e == cudaErrorMemoryAllocation);
+    cudaGetLastError();
+    prhs_destroy(c);
+    return fail(nullptr, oom ? PRHS_ERR_OOM : PRHS_ERR_CUDA, msg);
+  }
+  *out = c;
+  return PRHS_OK;
+}
+
+prhs_status prhs_destroy(prhs_ctx* c) {
+  if (!c) return PRHS_OK;
+  void* ptrs[] = {c->scores, c->part_ml, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
+                  c->count, c->flags, c->scratch_out, c->sstar_desc, c->sstar_asc, c->shat_asc,
+                  c->n_star, c->n_hat, c->anchor_t, c->st_q, c->st_out, c->st_k, c->st_v};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  for (auto& r : c->prof) {
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  delete c;
+  return PRHS_OK;
+}
+
+prhs_status prhs_score_topk(prhs_ctx* ctx, int32_t layer, int32_t step, const void* q,
+                            const prhs_kv_view* kv, const prhs_schedule* sched, int32_t batch,
+                            int32_t* out_idx, int32_t* out_count, float* out_lse_full, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!q) return fail(ctx, PRHS_ERR_INVALID_ARG, "q is NULL");
+  prhs_status rc = check_sched(ctx, sched);
+  if (rc != PRHS_OK) return rc;
+  rc = check_layer(ctx, layer, step, sched);
+  if (rc != PRHS_OK) return rc;
+  if (layer % sched->layer_group) return fail(ctx, PRHS_ERR_INVALID_ARG, "retrieval runs on the first layer of a group");
+  KvDev dv;
+  int max_t;
+  rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  return do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, out_idx, out_count, out_lse_full,
+                      as_stream(stream));
+}
+
+prhs_status prhs_build_index_set(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                                 const prhs_kv_view* kv, int32_t batch, int32_t* out_idx,
+                                 int32_t idx_stride, int32_t* out_count, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!out_idx || !out_count) return fail(ctx, PRHS_ERR_INVALID_ARG, "output pointer is NULL");
+  prhs_status rc = check_sched(ctx, sched);
+  if (rc != PRHS_OK) return rc;
+  rc = check_layer(ctx, layer, step, sched);
+  if (rc != PRHS_OK) return rc;
+  if (idx_stride < ctx->idx_cap) return fail(ctx, PRHS_ERR_CAPACITY, "idx_stride below prhs_index_capacity()");
+  KvDev dv;
+  int max_t;
+  rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  return do_build(ctx, layer, step, sched, dv, batch, out_idx, idx_stride, out_count, as_stream(stream));
+}
+
+prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,
+                                    const int32_t* idx, const int32_t* count, int32_t idx_stride,
+                                    int32_t batch, void* out, float* out_lse, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!q || !idx || !count || !out) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (idx_stride < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "idx_stride must be >= 1");
+  KvDev dv;
+  int max_t;
+  prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, idx_stride, batch, out, out_lse, nullptr,
+                     nullptr, as_stream(stream));
+}
+
+prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, int32_t batch,
+                                   void* out, float* out_lse, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!q || !out) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  KvDev dv;
+  int max_t;
+  prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, max_t, batch, out, out_lse, nullptr, nullptr,
+                     as_stream(stream));
+}
+
+prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                             const void* q, const prhs_kv_view* kv, int32_t batch, void* out,
+                             float* out_delta, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!q || !out) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  prhs_status rc = check_sched(ctx, sched);
+  if (rc != PRHS_OK) return rc;
+  rc = check_layer(ctx, layer, step, sched);
+  if (rc != PRHS_OK) return rc;
+  KvDev dv;
+  int max_t;
+  rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  cudaStream_t st = as_stream(stream);
+  const bool want_delta = (sched->flags & PRHS_WANT_DELTA) && out_delta;
+  const bool retrieve = (layer % sched->layer_group == 0) && (step % sched->refresh_interval == 0);
+  if (retrieve) {
+    rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, st);
+    if (rc != PRHS_OK) return rc;
+  } else if (want_delta) {
+    int nchunks = 1;
+    rc = launch_score(ctx, q, dv, batch, max_t, 0, st, &nchunks);
+    if (rc != PRHS_OK) return rc;
+    const int n = batch * ctx->cfg.num_q_heads;
+    {
+      LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+      lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, ctx->lse_full, n);
+    }
+    PRHS_CUDA(ctx, cudaGetLastError());
+  }
+  rc = do_build(ctx, layer, step, sched, dv, batch, ctx->idx, ctx->idx_cap, ctx->count, st);
+  if (rc != PRHS_OK) return rc;
+  ctx->last_batch = batch;
+  return launch_attn(ctx, q, dv, ctx->idx, ctx->count, ctx->idx_cap, ctx->idx_cap, batch, out,
+                     ctx->lse_c, want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr,
+                     st);
+}
+
+prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                                  const void* host_q, const void* host_new_k, const void* host_new_v,
+                                  const int32_t* host_seq_lens, const prhs_kv_view* kv, int32_t batch,
+                                  void* host_out, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!host_q || !host_new_k || !host_new_v || !host_seq_lens || !host_out || !kv)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (kv->page_table) return fail(ctx, PRHS_ERR_UNSUPPORTED, "host entry point needs a contiguous cache");
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  for (int b = 0; b < batch; ++b)
+    if (host_seq_lens[b] < 1 || host_seq_lens[b] > ctx->cfg.max_context)
+      return fail(ctx, PRHS_ERR_INVALID_ARG, "seq_lens entry out of range");
+  cudaStream_t st = as_stream(stream);
+  const size_t qb = (size_t)batch * ctx->cfg.num_q_heads * kRowBytes;
+  const size_t kb = (size_t)batch * ctx->cfg.num_kv_heads * kRowBytes;
+  PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_q, host_q, qb, cudaMemcpyHostToDevice, st));
+  PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_k, host_new_k, kb, cudaMemcpyHostToDevice, st));
+  PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_v, host_new_v, kb, cudaMemcpyHostToDevice, st));
+  PRHS_CUDA(ctx, cudaMemcpyAsync(const_cast<int32_t*>(kv->seq_lens), host_seq_lens, batch * sizeof(int32_t),
+                                 cudaMemcpyHostToDevice, st));
+  {
+    LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+    append_rows_kernel<<<dim3(ctx->cfg.num_kv_heads, batch), 32, 0, st>>>(
+        ctx->st_k, ctx->st_v, static_cast<__nv_bfloat16*>(const_cast<void*>(kv->k)),
+        static_cast<__nv_bfloat16*>(const_cast<void*>(kv->v)), kv->stride_outer, kv->stride_head,
+        kv->seq_lens, ctx->cfg.num_kv_heads);
+  }
+  PRHS_CUDA(ctx, cudaGetLastError());
+  prhs_status rc = prhs_decode_step(ctx, layer, step, sched, ctx->st_q, kv, batch, ctx->st_out, nullptr, stream);
+  if (rc != PRHS_OK) return rc;
+  PRHS_CUDA(ctx, cudaMemcpyAsync(host_out, ctx->st_out, qb, cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, const int32_t* idx,
+                       const int32_t* count, int32_t idx_stride, int32_t batch, float* out_delta,
+                       void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!q || !idx || !count || !out_delta) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (idx_stride < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "idx_stride must be >= 1");
+  KvDev dv;
+  int max_t;
+  prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  cudaStream_t st = as_stream(stream);
+  int nchunks = 1;
+  rc = launch_score(ctx, q, dv, batch, max_t, 0, st, &nchunks);
+  if (rc != PRHS_OK) return rc;
+  const int n = batch * ctx->cfg.num_q_heads;
+  {
+    LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+    lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, ctx->lse_full, n);
+  }
+  PRHS_CUDA(ctx, cudaGetLastError());
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, idx_stride, batch, ctx->scratch_out,
+                     ctx->lse_c, ctx->lse_full, out_delta, st);
+}
+
+prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx, int32_t* host_count,
+                               void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  cudaStream_t st = as_stream(stream);
+  const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
+  if (host_idx)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_idx, ctx->idx, n * ctx->idx_cap * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (host_count)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_count, ctx->count, n * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+prhs_status prhs_get_shared_set(prhs_ctx* ctx, int32_t layer, int32_t batch, int32_t* host_s_star,
+                                int32_t* host_n_star, int32_t* host_s_hat, int32_t* host_n_hat,
+                                void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  // groups are indexed with the layer_group of the schedule that last retrieved
+  const int g = layer / ctx->last_layer_group;
+  if (layer < 0 || g >= ctx->num_groups) return fail(ctx, PRHS_ERR_INVALID_ARG, "layer out of range");
+  cudaStream_t st = as_stream(stream);
+  const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
+  if (host_s_star)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_star, ctx->sstar_desc + state_off(ctx, g, ctx->cfg.max_k),
+                                   n * ctx->cfg.max_k * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (host_n_star)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_star, ctx->n_star + state_off(ctx, g, 1), n * sizeof(int),
+                                   cudaMemcpyDeviceToHost, st));
+  if (host_s_hat)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_hat, ctx->shat_asc + state_off(ctx, g, ctx->shat_cap),
+                                   n * ctx->shat_cap * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (host_n_hat)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_hat, ctx->n_hat + state_off(ctx, g, 1), n * sizeof(int),
+                                   cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+prhs_status prhs_get_scores(prhs_ctx* ctx, int32_t batch, float* host_scores, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!host_scores) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  cudaStream_t st = as_stream(stream);
+  PRHS_CUDA(ctx, cudaMemcpyAsync(host_scores, ctx->scores,
+                                 (size_t)batch * ctx->cfg.num_q_heads * ctx->ld * sizeof(float),
+                                 cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+const char* prhs_kernel_kind_name(int32_t kind) {
+  static const char* names[PRHS_KERNEL_KINDS] = {"score", "select", "build_set", "attn_sparse",
+                                                 "attn_dense", "misc"};
+  return (kind >= 0 && kind < PRHS_KERNEL_KINDS) ? names[kind] : "?";
+}
+
+prhs_status prhs_profile_begin(prhs_ctx* ctx, int32_t max_launches) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (max_launches < 1 || max_launches > (1 << 20))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "max_launches out of range");
+  while ((int)ctx->prof.size() < max_launches) {
+    prhs_ctx::ProfRec r;
+    r.kind = 0;
+    PRHS_CUDA(ctx, cudaEventCreate(&r.a));
+    cudaError_t e = cudaEventCreate(&r.b);
+    if (e != cudaSuccess) {
+      cudaEventDestroy(r.a);
+      return fail(ctx, PRHS_ERR_CUDA, cudaGetErrorString(e));
+    }
+    ctx->prof.push_back(r);
+  }
+  ctx->prof_used = 0;
+  ctx->prof_on = true;
+  return PRHS_OK;
+}
+
+prhs_status prhs_profile_end(prhs_ctx* ctx, void* stream, float* host_ms_per_kind,
+                             int64_t* host_launches_per_kind) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  ctx->prof_on = false;
+  PRHS_CUDA(ctx, cudaStreamSynchronize(as_stream(stream)));
+  for (int k = 0; k < PRHS_KERNEL_KINDS; ++k) {
+    if (host_ms_per_kind) host_ms_per_kind[k] = 0.f;
+    if (host_launches_per_kind) host_launches_per_kind[k] = 0;
+  }
+  for (int i = 0; i < ctx->prof_used; ++i) {
+    float ms = 0.f;
+    PRHS_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->prof[i].a, ctx->prof[i].b));
+    if (host_ms_per_kind) host_ms_per_kind[ctx->prof[i].kind] += ms;
+    if (host_launches_per_kind) host_launches_per_kind[ctx->prof[i].kind] += 1;
+  }
+  ctx->prof_used = 0;
+  return PRHS_OK;
+}
+
+prhs_status prhs_check(prhs_ctx* ctx, void* stream, uint32_t* out_flags) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  uint32_t f = 0;
+  PRHS_CUDA(ctx, cudaMemcpyAsync(&f, ctx->flags, sizeof(f), cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  PRHS_CUDA(ctx, cudaGetLastError());
+  if (out_flags) *out_flags = f;
+  if (f) {
+    PRHS_CUDA(ctx, cudaMemsetAsync(ctx->flags, 0, sizeof(uint32_t), st));
+    PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  }
+  if (f & (PRHS_FLAG_BAD_INDEX | PRHS_FLAG_BAD_PAGE)) {
+    char buf[96];
+    snprintf(buf, sizeof buf, "device flag word 0x%x", f);
+    return fail(ctx, PRHS_ERR_DEVICE_FLAG, buf);
+  }
+  return PRHS_OK;
+}
+
+}  // extern "C"

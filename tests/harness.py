@@ -1,0 +1,188 @@
+"""Shared helpers for the GPU parity tests: run the CUDA path through the C ABI and the CPU
+oracle on the same seeded tensors, and compare with the tolerances the benchmark fixes.
+
+Tolerances (bf16 inputs, fp32 accumulation on the GPU, float64 in the oracle):
+  index sets      bit-exact, except positions whose oracle logit lies within 1e-3 relative
+                  of the k-th (or, for dilation extras, the m-th) largest logit
+  attention y     max-abs 2e-2 against the oracle evaluated on the GPU's own index set
+  delta           1e-4 absolute
+  logits          1e-4 absolute + 1e-5 relative (fp32 accumulation order)
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import prhs_oracle as O
+from paper_2602_08329_b200 import binding as P
+from paper_2602_08329_b200 import workloads as W
+
+Y_TOL = 2e-2
+DELTA_TOL = 1e-4
+TIE_REL = 1e-3
+
+
+def np32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy()
+
+
+def tie_band(a_ref: float) -> float:
+    return TIE_REL * max(abs(a_ref), 1e-3)
+
+
+def check_topk_legal(a32: np.ndarray, got_desc: np.ndarray, want_desc: np.ndarray, where=""):
+    """`got_desc` must equal the oracle's S* except for near-ties with the k-th logit."""
+    assert len(got_desc) == len(want_desc), f"{where}: |S*| {len(got_desc)} != {len(want_desc)}"
+    if len(want_desc) == 0:
+        return
+    assert len(set(got_desc.tolist())) == len(got_desc), f"{where}: duplicate winners"
+    a_k = float(a32[want_desc[-1]])
+    diff = np.setxor1d(got_desc, want_desc)
+    for i in diff:
+        assert abs(float(a32[i]) - a_k) <= tie_band(a_k), \
+            f"{where}: position {i} logit {a32[i]} differs from the oracle set beyond the tie band of {a_k}"
+    # descending order (ties by lower position) up to the same band
+    ag = a32[got_desc].astype(np.float64)
+    assert np.all(np.diff(ag) <= tie_band(a_k)), f"{where}: S* not in descending-logit order"
+    if len(diff) == 0:
+        same = got_desc == want_desc
+        for j in np.nonzero(~same)[0]:
+            assert abs(float(a32[got_desc[j]]) - float(a32[want_desc[j]])) <= tie_band(a32[want_desc[j]]), \
+                f"{where}: order differs at rank {j} beyond a near-tie"
+
+
+def make_ctx(w: W.Workload, **over):
+    kw = dict(num_layers=w.layers, max_batch=w.batch, num_q_heads=w.q_heads, num_kv_heads=w.kv_heads,
+              max_context=w.capacity, max_k=max(w.top_k, int(w.k_frac * w.context)),
+              max_window=w.window, max_sinks=w.sinks, max_dilate_r=max(w.dilate_r, 1), max_dilate_m=-1,
+              page_size=w.page_size, min_layer_group=w.layer_group)
+    kw.update(over)
+    return P.Context(**kw)
+
+
+def make_sched(w: W.Workload, device, flags=0, **over):
+    kps = W.top_k_per_seq(w)
+    kps_dev = kps.to(device) if kps is not None else None
+    kw = dict(top_k=w.top_k, window=w.window, sinks=w.sinks, refresh_interval=w.refresh,
+              layer_group=w.layer_group, dilate_r=w.dilate_r, dilate_m=-1, top_k_per_seq=kps_dev,
+              flags=flags)
+    kw.update(over)
+    return P.make_schedule(**kw)
+
+
+def oracle_sched(w: W.Workload, **over) -> O.Schedule:
+    kps = W.top_k_per_seq(w)
+    kw = dict(top_k=w.top_k, window=w.window, sinks=w.sinks, refresh_interval=w.refresh,
+              layer_group=w.layer_group, dilate_r=w.dilate_r, dilate_m=-1,
+              top_k_per_seq=None if kps is None else kps.numpy())
+    kw.update(over)
+    return O.Schedule(**kw)
+
+
+class HostKV:
+    """Lazy host copies of single (layer, b, kvh) cache slices as float32 numpy arrays."""
+
+    def __init__(self):
+        self.cache = {}
+
+    def get(self, tag, tensor, b, kvh):
+        key = (tag, b, kvh)
+        if key not in self.cache:
+            self.cache[key] = np32(tensor[b, kvh])
+        return self.cache[key]
+
+
+def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, want_delta=True,
+                        paged=False, check_scores=True):
+    """Drive prhs_decode_step over the workload's schedule and compare sampled (b, h) units.
+
+    The oracle follows the same schedule.  After each retrieval the GPU's S* is checked for
+    legality against the oracle's and then adopted by the oracle, so that every later
+    comparison in the block (dilation, shared sets, attention, delta) is exact.
+    Returns a dict of summary statistics.
+    """
+    layers = list(range(w.layers)) if layers is None else layers
+    steps = w.steps if steps is None else steps
+    ctx = make_ctx(w)
+    flags = P.PRHS_WANT_DELTA if want_delta else 0
+    sched = make_sched(w, device, flags=flags)
+    osched = oracle_sched(w)
+    orc = O.PrhsOracle(osched, w.q_heads, w.kv_heads)
+    q_all = W.make_queries(w, device)
+    kv = {l: (k, v) for l, k, v in W.make_layer_kv(w, device, layers=layers)}
+    table = pool = None
+    paged_kv = {}
+    if paged:
+        table, pool = W.make_page_table(w)
+        for l in layers:
+            paged_kv[l] = (W.to_paged(w, kv[l][0], table, pool), W.to_paged(w, kv[l][1], table, pool))
+        table_dev = table.to(device)
+    host = HostKV()
+    B, Hq = w.batch, w.q_heads
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=device)
+    dlt = torch.empty(B, Hq, dtype=torch.float32, device=device)
+    stats = dict(max_y_err=0.0, max_delta_err=0.0, near_tie_sets=0, checked=0, deltas=[], set_sizes=[])
+    gq = w.q_heads // w.kv_heads
+    for n in range(steps):
+        t_host = W.seq_lens_at(w, n)
+        t_dev = t_host.to(device)
+        for l in layers:
+            k_l, v_l = kv[l]
+            if paged:
+                view = P.make_view(paged_kv[l][0], paged_kv[l][1], t_dev, page_table=table_dev,
+                                   max_seq_len=w.capacity)
+            else:
+                view = P.make_view(k_l, v_l, t_dev, max_seq_len=w.capacity)
+            q = q_all[l, n].contiguous()
+            ctx.decode_step(l, n, sched, q, view, B, out, dlt if want_delta else None)
+            idx, cnt = ctx.get_index_set(B)
+            assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+            y_gpu, d_gpu = np32(out), np32(dlt)
+            retrieve = orc.is_retrieval(l, n)
+            if retrieve:
+                s_star, n_star, s_hat, n_hat = ctx.get_shared_set(l, B)
+                scores = ctx.get_scores(B) if check_scores else None
+            qh = np32(q)
+            for (b, h) in units:
+                kvh = h // gq
+                Kh, Vh = host.get(("k", l), k_l, b, kvh), host.get(("v", l), v_l, b, kvh)
+                t = int(t_host[b])
+                where = f"layer {l} step {n} unit ({b},{h})"
+                if retrieve:
+                    a = O.dense_scores(qh[b, h], Kh, t)
+                    a32 = O.rank_logits(a)
+                    want = O.topk_middle(a, t, w.sinks, w.window, osched.k_for(b))
+                    got = s_star[b, h, : int(n_star[b, h])].numpy().astype(np.int64)
+                    before = len(np.setxor1d(got, want))
+                    check_topk_legal(a32, got, want, where)
+                    stats["near_tie_sets"] += int(before > 0)
+                    if check_scores:
+                        sg = scores[b, h, :t].numpy()
+                        assert np.allclose(sg, a32, atol=1e-4, rtol=1e-5), f"{where}: logits differ"
+                    # adopt the GPU's (legal) S*; dilation must then match exactly
+                    g = l // w.layer_group
+                    sh = orc.groups.setdefault(g, O._Shared())
+                    if sh.step != n:
+                        sh.step, sh.s_star, sh.s_hat = n, {}, {}
+                    sh.s_star[(b, h)] = got
+                    sh.s_hat[(b, h)] = O.dilate(got, osched.m_for(b), osched.dilate_r, t)
+                    got_hat = s_hat[b, h, : int(n_hat[b, h])].numpy().astype(np.int64)
+                    assert np.array_equal(got_hat, sh.s_hat[(b, h)]), f"{where}: dilated set differs"
+                C_want = orc.index_set(l, n, b, h, t)
+                C_got = idx[b, h, : int(cnt[b, h])].numpy().astype(np.int64)
+                assert np.array_equal(C_got, C_want), f"{where}: index set differs"
+                y_ref, lse_c = O.attn_over_set(qh[b, h], Kh, Vh, C_want)
+                err = float(np.max(np.abs(y_gpu[b, h] - O.bf16_round(y_ref))))
+                assert err <= Y_TOL, f"{where}: attention max-abs error {err}"
+                stats["max_y_err"] = max(stats["max_y_err"], err)
+                stats["set_sizes"].append(len(C_want))
+                if want_delta:
+                    a = O.dense_scores(qh[b, h], Kh, t)
+                    d_ref = O.delta_from_lse(lse_c, O.logsumexp(a))
+                    derr = abs(float(d_gpu[b, h]) - d_ref)
+                    assert derr <= DELTA_TOL, f"{where}: delta {d_gpu[b, h]} vs {d_ref}"
+                    stats["max_delta_err"] = max(stats["max_delta_err"], derr)
+                    stats["deltas"].append(d_ref)
+                stats["checked"] += 1
+    ctx.close()
+    return stats

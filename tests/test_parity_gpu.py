@@ -1,0 +1,399 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle.
+
+Small cases compare every element; the benchmark's full-size configurations compare sampled
+(sequence, head) units that the oracle computes one by one, in the launch configuration the
+benchmark times.  Tolerances are stated in tests/harness.py.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import prhs_oracle as O
+from paper_2602_08329_b200 import binding as P
+from paper_2602_08329_b200 import workloads as W
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def all_units(w):
+    return [(b, h) for b in range(w.batch) for h in range(w.q_heads)]
+
+
+def small(name="small", **kw):
+    base = dict(layers=1, batch=2, q_heads=4, kv_heads=2, context=1500, steps=4, top_k=48, window=16,
+                sinks=4, refresh=2, heavy_hitters=8, decay_span=64, seed=11)
+    base.update(kw)
+    return W.Workload(name, **base)
+
+
+# ------------------------------------------------------------------ stage by stage
+@pytest.mark.parametrize("gq", [1, 2, 4, 8])
+def test_sparse_attention_over_given_sets(cuda_device, gq):
+    w = small(q_heads=8, kv_heads=8 // gq, context=3000, seed=20 + gq)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = torch.tensor([2999, 1234], dtype=torch.int32)
+    g = np.random.default_rng(gq)
+    cap = 700
+    idx = torch.full((w.batch, w.q_heads, cap), -7, dtype=torch.int32)
+    cnt = torch.zeros(w.batch, w.q_heads, dtype=torch.int32)
+    sets = {}
+    sizes = [0, 1, 15, 16, 17, 255, 256, 257, 511, 640, 700, 33, 300, 64, 129, 5]
+    for b in range(w.batch):
+        for h in range(w.q_heads):
+            n = min(sizes[(b * w.q_heads + h) % len(sizes)], int(t_host[b]))
+            C = np.sort(g.permutation(int(t_host[b]))[:n])
+            sets[(b, h)] = C
+            idx[b, h, :n] = torch.from_numpy(C.astype(np.int32))
+            cnt[b, h] = n
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    dlt = torch.empty_like(lse)
+    ctx.sparse_decode_attn(q, view, idx.to(cuda_device), cnt.to(cuda_device), w.batch, out, lse)
+    ctx.delta(q, view, idx.to(cuda_device), cnt.to(cuda_device), w.batch, dlt)
+    assert ctx.check() == 0
+    y, ls, dl, qh = H.np32(out), H.np32(lse), H.np32(dlt), H.np32(q)
+    for (b, h), C in sets.items():
+        kvh = h // gq
+        Kh, Vh = H.np32(k[b, kvh]), H.np32(v[b, kvh])
+        y_ref, lse_ref = O.attn_over_set(qh[b, h], Kh, Vh, C)
+        assert np.max(np.abs(y[b, h] - O.bf16_round(y_ref))) <= H.Y_TOL
+        if len(C) == 0:
+            assert ls[b, h] == -math.inf and np.all(y[b, h] == 0) and dl[b, h] == 1.0
+            continue
+        assert abs(ls[b, h] - lse_ref) <= 1e-4
+        a = O.dense_scores(qh[b, h], Kh, int(t_host[b]))
+        assert abs(dl[b, h] - O.delta_from_lse(lse_ref, O.logsumexp(a))) <= H.DELTA_TOL
+    ctx.close()
+
+
+@pytest.mark.parametrize("gq", [1, 4])
+def test_dense_baseline_matches_oracle(cuda_device, gq):
+    w = small(q_heads=4, kv_heads=4 // gq, context=5000, seed=30 + gq)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 1].contiguous()
+    t_host = torch.tensor([5003, 777], dtype=torch.int32)
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    ctx.dense_decode_attn(q, view, w.batch, out, lse)
+    assert ctx.check() == 0
+    y, ls, qh = H.np32(out), H.np32(lse), H.np32(q)
+    for b, h in all_units(w):
+        y_ref, lse_ref = O.dense_attention(qh[b, h], H.np32(k[b, h // gq]), H.np32(v[b, h // gq]), int(t_host[b]))
+        assert np.max(np.abs(y[b, h] - O.bf16_round(y_ref))) <= H.Y_TOL
+        assert abs(ls[b, h] - lse_ref) <= 1e-4
+    ctx.close()
+
+
+@pytest.mark.parametrize("gq,context", [(1, 1500), (2, 2500), (4, 4100), (8, 700)])
+def test_score_topk_and_dilation(cuda_device, gq, context):
+    w = small(q_heads=8, kv_heads=8 // gq, context=context, top_k=96, seed=40 + gq)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = torch.tensor([context + 1, context // 2 + 3], dtype=torch.int32)
+    ctx = H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    oi = torch.empty(w.batch, w.q_heads, w.top_k, dtype=torch.int32, device=cuda_device)
+    oc = torch.empty(w.batch, w.q_heads, dtype=torch.int32, device=cuda_device)
+    ol = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    ctx.score_topk(0, 0, q, view, sched, w.batch, oi, oc, ol)
+    assert ctx.check() == 0
+    scores = ctx.get_scores(w.batch)
+    s_star, n_star, s_hat, n_hat = ctx.get_shared_set(0, w.batch)
+    assert torch.equal(s_star[:, :, : w.top_k], oi.cpu()) and torch.equal(n_star, oc.cpu())
+    qh, lf = H.np32(q), H.np32(ol)
+    for b, h in all_units(w):
+        t = int(t_host[b])
+        Kh = H.np32(k[b, h // gq])
+        a = O.dense_scores(qh[b, h], Kh, t)
+        a32 = O.rank_logits(a)
+        assert np.allclose(scores[b, h, :t].numpy(), a32, atol=1e-4, rtol=1e-5)
+        assert abs(lf[b, h] - O.logsumexp(a)) <= 1e-4
+        want = O.topk_middle(a, t, w.sinks, w.window, w.top_k)
+        got = s_star[b, h, : int(n_star[b, h])].numpy().astype(np.int64)
+        H.check_topk_legal(a32, got, want, f"unit ({b},{h})")
+        assert np.all(s_star[b, h, int(n_star[b, h]):].numpy() == -1)
+        hat = s_hat[b, h, : int(n_hat[b, h])].numpy().astype(np.int64)
+        assert np.array_equal(hat, O.dilate(got, w.top_k // 3, 1, t))
+    ctx.close()
+
+
+def test_identical_keys_take_the_tie_path(cuda_device):
+    # all logits equal: S* must be the k lowest middle positions, in position order
+    w = small(batch=1, q_heads=2, kv_heads=1, context=3000, top_k=100)
+    k, v = W.make_kv(w, cuda_device)
+    k[:] = k[:, :, :1, :]
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = torch.tensor([2900], dtype=torch.int32)
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), 1)
+    s_star, n_star, s_hat, n_hat = ctx.get_shared_set(0, 1)
+    for h in range(2):
+        assert int(n_star[0, h]) == 100
+        assert np.array_equal(s_star[0, h, :100].numpy(), np.arange(4, 104))
+        assert np.array_equal(s_hat[0, h, : int(n_hat[0, h])].numpy(), np.arange(3, 104))
+    ctx.close()
+
+
+def test_partial_ties_at_the_threshold(cuda_device):
+    # duplicated key rows straddle the k-th place: the lower positions must win
+    w = small(batch=1, q_heads=1, kv_heads=1, context=2000, top_k=10, heavy_hitters=0)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t = 2001
+    a = O.dense_scores(H.np32(q)[0, 0], H.np32(k[0, 0]), t)
+    order = O.topk_middle(a, t, 4, 16, 12)
+    src = int(order[9])                                    # the 10th best key ...
+    dup = [p for p in (100, 900, 1500) if p not in set(order.tolist())]
+    for p in dup:
+        k[0, 0, p] = k[0, 0, src]                          # ... now appears several times
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, torch.tensor([t], dtype=torch.int32, device=cuda_device), max_seq_len=w.capacity)
+    ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), 1)
+    s_star, n_star, _, _ = ctx.get_shared_set(0, 1)
+    a = O.dense_scores(H.np32(q)[0, 0], H.np32(k[0, 0]), t)
+    want = O.topk_middle(a, t, 4, 16, 10)
+    assert np.array_equal(s_star[0, 0, :10].numpy(), want)
+    assert int(want[-1]) == min(dup + [src])
+    ctx.close()
+
+
+def test_degenerate_lengths(cuda_device):
+    # t <= S0 + W (empty middle), t == 1, k larger than the middle range
+    w = small(batch=4, q_heads=2, kv_heads=2, context=300, top_k=64, window=16, sinks=4, steps=1)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = torch.tensor([1, 20, 50, 301], dtype=torch.int32)
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    out = torch.empty(4, 2, 128, dtype=torch.bfloat16, device=cuda_device)
+    dlt = torch.empty(4, 2, dtype=torch.float32, device=cuda_device)
+    sched = H.make_sched(w, cuda_device, flags=P.PRHS_WANT_DELTA, refresh_interval=1)
+    ctx.decode_step(0, 0, sched, q, view, 4, out, dlt)
+    assert ctx.check() == 0
+    idx, cnt = ctx.get_index_set(4)
+    qh, y, d = H.np32(q), H.np32(out), H.np32(dlt)
+    for b, h in all_units(w):
+        t = int(t_host[b])
+        Kh, Vh = H.np32(k[b, h]), H.np32(v[b, h])
+        a = O.dense_scores(qh[b, h], Kh, t)
+        C = O.build_set(t, 4, 16, O.topk_middle(a, t, 4, 16, 64))
+        assert np.array_equal(idx[b, h, : int(cnt[b, h])].numpy(), C)
+        if t <= 4 + 16 + 64:
+            assert len(C) == t and abs(d[b, h]) <= H.DELTA_TOL      # nothing dropped
+        y_ref, _ = O.attn_over_set(qh[b, h], Kh, Vh, C)
+        assert np.max(np.abs(y[b, h] - O.bf16_round(y_ref))) <= H.Y_TOL
+    ctx.close()
+
+
+def test_full_budget_equals_dense(cuda_device):
+    w = small(batch=1, q_heads=4, kv_heads=2, context=900, top_k=1024, steps=1)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = torch.tensor([901], dtype=torch.int32, device=cuda_device)
+    ctx = H.make_ctx(w)
+    view = P.make_view(k, v, t_dev, max_seq_len=w.capacity)
+    out = torch.empty(1, 4, 128, dtype=torch.bfloat16, device=cuda_device)
+    dense = torch.empty_like(out)
+    dlt = torch.empty(1, 4, dtype=torch.float32, device=cuda_device)
+    ctx.decode_step(0, 0, H.make_sched(w, cuda_device, flags=P.PRHS_WANT_DELTA), q, view, 1, out, dlt)
+    ctx.dense_decode_attn(q, view, 1, dense)
+    _, cnt = ctx.get_index_set(1)
+    assert torch.all(cnt == 901)
+    assert torch.max(torch.abs(out.float() - dense.float())) <= 1e-2
+    assert torch.max(torch.abs(dlt)) <= H.DELTA_TOL
+    ctx.close()
+
+
+def test_bad_index_is_flagged_not_faulted(cuda_device):
+    w = small(batch=1, q_heads=1, kv_heads=1, context=500)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = torch.tensor([400], dtype=torch.int32, device=cuda_device)
+    idx = torch.tensor([[[0, 5, 400, -3, 399, 10 ** 6]]], dtype=torch.int32, device=cuda_device)
+    cnt = torch.tensor([[6]], dtype=torch.int32, device=cuda_device)
+    ctx = H.make_ctx(w)
+    out = torch.empty(1, 1, 128, dtype=torch.bfloat16, device=cuda_device)
+    ctx.sparse_decode_attn(q, P.make_view(k, v, t_dev), idx, cnt, 1, out)
+    with pytest.raises(P.PrhsError) as e:
+        ctx.check()
+    assert e.value.status == 7
+    assert ctx.check() == 0                                  # the flag word was cleared
+    y_ref, _ = O.attn_over_set(H.np32(q)[0, 0], H.np32(k[0, 0]), H.np32(v[0, 0]), np.array([0, 5, 399]))
+    assert np.max(np.abs(H.np32(out)[0, 0] - O.bf16_round(y_ref))) <= H.Y_TOL
+    ctx.close()
+
+
+def test_results_are_deterministic(cuda_device):
+    w = small(context=2500)
+    outs = []
+    for _ in range(2):
+        torch.cuda.empty_cache()
+        k, v = W.make_kv(w, cuda_device)
+        q = W.make_queries(w, cuda_device)
+        ctx = H.make_ctx(w)
+        sched = H.make_sched(w, cuda_device)
+        out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+        res = []
+        for n in range(w.steps):
+            view = P.make_view(k, v, W.seq_lens_at(w, n).to(cuda_device), max_seq_len=w.capacity)
+            ctx.decode_step(0, n, sched, q[0, n].contiguous(), view, w.batch, out)
+            idx, cnt = ctx.get_index_set(w.batch)
+            res.append((out.clone().cpu(), idx.clone(), cnt.clone()))
+        outs.append(res)
+        ctx.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a[2], b[2])
+        for bb in range(w.batch):
+            for h in range(w.q_heads):
+                c = int(a[2][bb, h])
+                assert torch.equal(a[1][bb, h, :c], b[1][bb, h, :c])
+        assert torch.equal(a[0], b[0])
+
+
+# ------------------------------------------------------------- schedules end to end
+def test_schedule_small_every_unit(cuda_device):
+    w = small(steps=6, refresh=3, context=2200)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w))
+    assert st["checked"] == 6 * w.batch * w.q_heads
+
+
+def test_schedule_cross_layer_groups(cuda_device):
+    w = small(layers=4, layer_group=2, steps=4, refresh=2, q_heads=4, kv_heads=1, context=1800, seed=12)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w))
+    assert st["checked"] == 4 * 4 * w.batch * w.q_heads
+
+
+def test_schedule_paged_and_ragged(cuda_device):
+    w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=5, q_heads=8, kv_heads=2,
+              context=3000, min_context=300, page_size=16, top_k=0, k_frac=0.03, seed=13)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=True)
+    assert st["checked"] == 2 * 4 * w.batch * w.q_heads
+
+
+def test_paged_identity_equals_contiguous(cuda_device):
+    w = small(batch=2, q_heads=4, kv_heads=2, context=1000, page_size=16, steps=2)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = W.seq_lens_at(w, 0).to(cuda_device)
+    table, pool = W.make_page_table(w)
+    kp, vp = W.to_paged(w, k, table, pool), W.to_paged(w, v, table, pool)
+    outs = []
+    for paged in (False, True):
+        ctx = H.make_ctx(w, page_size=16 if paged else 0)
+        view = (P.make_view(kp, vp, t_dev, page_table=table.to(cuda_device), max_seq_len=w.capacity)
+                if paged else P.make_view(k, v, t_dev, max_seq_len=w.capacity))
+        out = torch.empty(2, 4, 128, dtype=torch.bfloat16, device=cuda_device)
+        ctx.decode_step(0, 0, H.make_sched(w, cuda_device), q, view, 2, out)
+        idx, cnt = ctx.get_index_set(2)
+        outs.append((out.cpu(), idx, cnt))
+        assert ctx.check() == 0
+        ctx.close()
+    assert torch.equal(outs[0][2], outs[1][2]) and torch.equal(outs[0][0], outs[1][0])
+
+
+def test_c1_tiny_exactly_as_specified(cuda_device):
+    st = H.run_schedule_parity(W.C1_TINY, cuda_device, all_units(W.C1_TINY))
+    assert st["checked"] == 4 * 8
+    assert max(st["set_sizes"]) <= 4 + 256 + 2 * 85 + 64
+
+
+# --------------------------------------------------- full-size configurations, sampled units
+def test_c2_full_size_sampled(cuda_device):
+    w = W.C2_LLAMA2_7B.scaled(steps=8)
+    units = [(0, 0), (3, 17), (7, 31), (5, 8)]
+    st = H.run_schedule_parity(w, cuda_device, units)
+    assert st["checked"] == 8 * len(units)
+
+
+def test_c4_long_context_sampled(cuda_device):
+    # 128K context: the selection works from global memory (candidates exceed shared memory)
+    w = W.C4_LLAMA3_128K.scaled(steps=5)
+    units = [(0, 0), (1, 13), (3, 31)]
+    st = H.run_schedule_parity(w, cuda_device, units, check_scores=True)
+    assert st["checked"] == 5 * len(units)
+
+
+def test_c3_stack_slice_sampled(cuda_device):
+    # the Mistral-shaped stack at full per-layer size, first two layer groups
+    w = W.C3_MISTRAL.scaled(layers=8, steps=5, batch=4)
+    units = [(0, 0), (2, 21), (3, 31)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3, 4, 7])
+    assert st["checked"] == 5 * 5 * len(units)
+
+
+def test_c5_serving_mix_sampled(cuda_device):
+    # ragged paged serving mix at reduced batch and layers (full per-sequence sizes)
+    w = W.C5_SERVING.scaled(layers=4, steps=5, batch=6)
+    units = [(0, 0), (2, 9), (5, 31), (3, 16)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3], paged=True)
+    assert st["checked"] == 5 * 3 * len(units)
+
+
+# ------------------------------------------------------------------- host-buffer entry point
+def test_decode_step_host_buffers(cuda_device):
+    w = small(steps=3, refresh=2, context=1200)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)
+    k2, v2 = k.clone(), v.clone()
+    ctx_a, ctx_b = H.make_ctx(w), H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device)
+    out_a = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    t_dev = torch.zeros(w.batch, dtype=torch.int32, device=cuda_device)
+    for n in range(w.steps):
+        t_host = W.seq_lens_at(w, n)
+        ctx_a.decode_step(0, n, sched, q[0, n].contiguous(), P.make_view(k, v, t_host.to(cuda_device)),
+                          w.batch, out_a)
+        # the host entry point appends the new token's rows itself: blank them first
+        pos = (t_host - 1).long()
+        bi = torch.arange(w.batch)
+        new_k, new_v = k[bi, :, pos].cpu().contiguous(), v[bi, :, pos].cpu().contiguous()
+        k2[bi, :, pos] = 0
+        v2[bi, :, pos] = 0
+        host_out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16).pin_memory()
+        ctx_b.decode_step_host(0, n, sched, q[0, n].cpu().contiguous().pin_memory(), new_k.pin_memory(),
+                               new_v.pin_memory(), t_host, P.make_view(k2, v2, t_dev), w.batch, host_out)
+        assert torch.equal(host_out, out_a.cpu())
+    assert torch.equal(k2, k) and torch.equal(v2, v)
+    ctx_a.close(); ctx_b.close()
+
+
+# ------------------------------------------------------------------------- host validation
+def test_host_side_errors(cuda_device):
+    w = small()
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = W.seq_lens_at(w, 0).to(cuda_device)
+    view = P.make_view(k, v, t_dev)
+    ctx = H.make_ctx(w)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+
+    def status(fn):
+        with pytest.raises(P.PrhsError) as e:
+            fn()
+        return e.value.status
+
+    good = H.make_sched(w, cuda_device)
+    assert status(lambda: ctx.decode_step(0, 1, good, q, view, w.batch, out)) == 5       # no anchor yet
+    assert status(lambda: ctx.decode_step(0, 0, good, q, view, w.batch + 1, out)) == 6   # batch
+    assert status(lambda: ctx.decode_step(0, 0, H.make_sched(w, cuda_device, top_k=w.top_k + 1), q, view,
+                                          w.batch, out)) == 6
+    assert status(lambda: ctx.decode_step(0, 0, H.make_sched(w, cuda_device, refresh_interval=0), q, view,
+                                          w.batch, out)) == 1
+    assert status(lambda: ctx.decode_step(5, 0, good, q, view, w.batch, out)) == 1       # layer range
+    assert status(lambda: ctx.decode_step(0, 0, good, None, view, w.batch, out)) == 1    # NULL q
+    with pytest.raises(P.PrhsError) as e:
+        P.Context(1, 1, 4, 2, 1000, 16, 16, 4, head_dim=64)
+    assert e.value.status == 2
+    ctx.decode_step(0, 0, good, q, view, w.batch, out)                                   # still usable
+    assert ctx.check() == 0
+    ctx.close()
