@@ -196,6 +196,8 @@ def run_cuda(args):
     Wn, Kn = args.warmup, args.steps
     total_steps = Wn + Kn
     w = W.C2_LLAMA2_7B.scaled(steps=total_steps, seed=W.C2_LLAMA2_7B.seed + 97 * rank)
+    if args.batch:
+        w = w.scaled(batch=args.batch)      # smaller case for profiler captures only
     k, v = W.make_kv(w, dev)
     q_all = W.make_queries(w, dev)[0]                     # [steps][B][Hq][128]
     B, Hq, Hkv = w.batch, w.q_heads, w.kv_heads
@@ -275,6 +277,13 @@ def run_cuda(args):
     bytes_touched = sum(score_bytes) + sum(gather_bytes)
     path_gbs = bytes_touched / (total_ms * 1e-3) / 1e9
 
+    if args.path_only:                      # profiler captures: the hot path alone
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "kernels": kernels,
+                              "config": workload_config(w), "note": "path only (profiling run)"}))
+        ctx.close()
+        return 0
+
     # ---- in-library dense flash-decode baseline, same protocol
     nd = min(4, Kn)
     dense_ms = timed_steps(Wn, nd, lambda n: ctx.dense_decode_attn(q_all[n], views[n], B, out))
@@ -352,6 +361,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling captures)")
+    ap.add_argument("--path-only", action="store_true", help="skip the dense, e2e and CPU legs")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         print("warning: fewer than 3 warm-up steps", file=sys.stderr)
