@@ -236,7 +236,8 @@ def run_cuda(args):
     barrier()
     launches = ctx.launch_count - launches0
     clocks = sampler.stop()
-    assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+    dev_flags = ctx.check()
+    assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
     total_ms = sum(ms)
     total_ms_max = reduce_max_ms(total_ms, dist, dev)
     value = job_throughput(world, B, Kn, total_ms_max)
@@ -280,6 +281,7 @@ def run_cuda(args):
     if args.path_only:                      # profiler captures: the hot path alone
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "kernels": kernels,
+                              "select_fallback": bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK),
                               "config": workload_config(w), "note": "path only (profiling run)"}))
         ctx.close()
         return 0
@@ -342,6 +344,7 @@ def run_cuda(args):
         "path_frac_of_8tbs": path_gbs / 8000.0,
         "mean_set_size": sum(counts) / (len(counts) * B * Hq),
         "retrieval_ratio": len(score_bytes) / Kn,
+        "select_fallback": bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK),
         "roofline": roofline, "kernels": kernels,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_max_ms / Kn},

@@ -72,8 +72,9 @@ typedef struct {
  *        k + b*stride_outer + kvh*stride_head + i*128            (element offsets)
  *   paged (page_table != NULL, 16 positions per page): row i of (b, kvh) is at
  *        k + page_table[b*page_table_stride + i/16]*stride_outer + kvh*stride_head + (i%16)*128
- * Rows are 128 contiguous bf16 (256 bytes); k, v and every stride must keep rows 16-byte
- * aligned (strides multiples of 8 elements). */
+ * Rows are 128 contiguous bf16 (256 bytes); k and v must be 16-byte aligned and both strides
+ * multiples of 128 elements (whole rows), with fewer than 2^32 rows between the base and the
+ * last row addressed. */
 typedef struct {
   const void* k;
   const void* v;
@@ -190,9 +191,11 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
 /* Largest index-list length any call can produce: S0 + k + 2*r*m + W from prhs_config. */
 int32_t prhs_index_capacity(const prhs_ctx* ctx);
 
-/* Copy the set the last prhs_decode_step / prhs_build_index_set(ctx-internal) produced to
- * the host: host_idx int32 [batch][Hq][prhs_index_capacity()], host_count int32
- * [batch][Hq].  Synchronous; for tests and diagnostics. */
+/* The index set the last prhs_decode_step attended over (the step builds it inside the
+ * attention kernel; this call materialises it with the stand-alone builder and copies it to
+ * the host): host_idx int32 [batch][Hq][prhs_index_capacity()], host_count int32
+ * [batch][Hq].  The seq_lens buffer of that step must still hold the step's lengths.
+ * Synchronous; for tests and diagnostics. */
 prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx,
                                int32_t* host_count, void* stream);
 

@@ -20,16 +20,23 @@ build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int
   const int nm = __ldg(n_mid + unit);
   const int s0 = min(sinks, t);
   const int wlo = max(max(t - window, 0), s0);
+  // M is ascending: the number of entries below a bound is the position of the bound.  Count
+  // in parallel (one coalesced pass) instead of a binary search of dependent cold loads.
   __shared__ int sh_lo, sh_hi;
-  if (threadIdx.x < 2) {
-    const int bound = threadIdx.x == 0 ? s0 : wlo;   // first entry >= bound
-    int a = 0, c = nm;
-    while (a < c) {
-      const int mid_i = (a + c) >> 1;
-      if (__ldg(M + mid_i) < bound) a = mid_i + 1; else c = mid_i;
-    }
-    if (threadIdx.x == 0) sh_lo = a; else sh_hi = a;
+  if (threadIdx.x == 0) { sh_lo = 0; sh_hi = 0; }
+  __syncthreads();
+  int c0 = 0, c1 = 0;
+  for (int i = threadIdx.x; i < nm; i += blockDim.x) {
+    const int x = __ldg(M + i);
+    c0 += x < s0;
+    c1 += x < wlo;
   }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    c0 += __shfl_xor_sync(0xffffffffu, c0, off);
+    c1 += __shfl_xor_sync(0xffffffffu, c1, off);
+  }
+  if ((threadIdx.x & 31) == 0) { atomicAdd(&sh_lo, c0); atomicAdd(&sh_hi, c1); }
   __syncthreads();
   const int lo = sh_lo, hi = max(sh_hi, sh_lo);
   const int nmid = hi - lo;
@@ -46,16 +53,20 @@ build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int
 }
 
 // ------------------------------------------------------------ gathered / dense attention
-constexpr int kAttnThreads = 256;                 // 16 half-warps
-constexpr int kAttnHalfWarps = kAttnThreads / 16;
 constexpr int kPartStride = kHeadDim + 2;         // o[128] (unnormalised), m, l per split
 
 struct AttnParams {
   const __nv_bfloat16* q;   // [B][Hq][128]
   KvDev kv;
-  const int* idx;           // [B][Hq][idx_stride] or nullptr = all positions [0, t)
-  const int* count;         // [B][Hq] (ignored when idx == nullptr)
+  const int* idx;           // [B][Hq][idx_stride] or nullptr
+  const int* count;         // [B][Hq] (with idx)
   int idx_stride;
+  // fused index-set builder (used when idx == nullptr and mid != nullptr): the list is
+  // [0, s0) ++ M clipped to [s0, wlo) ++ [wlo, t) with M = mid[unit][0..n_mid[unit]) ascending
+  const int* mid;
+  const int* n_mid;
+  int mid_stride, sinks, window;
+  // idx == nullptr and mid == nullptr: all positions [0, t) (dense baseline)
   int num_q_heads, group_size;
   int splits;
   float* partials;          // [B][Hq][splits][kPartStride]
@@ -67,161 +78,329 @@ struct AttnParams {
   uint32_t* flags;
 };
 
-// grid (splits, Hq, B).  Each half-warp owns blocks of 16 consecutive list entries; a lane
-// holds 8 of the 128 elements of a row, so one 16-byte load per lane fetches a whole row
-// per half-warp.  Four K rows and four V rows are in flight per half-warp.  Every
-// half-warp keeps its own online-softmax state (log2 domain); states are combined in shared
-// memory, written as a split partial, and the last CTA to arrive for a (b, h) merges the
-// splits (ticket counter, no waiting).
-__global__ void __launch_bounds__(kAttnThreads) gather_attn_kernel(AttnParams p) {
+// ---------------------------------------------------------------- cp.async helpers
+constexpr uint32_t kBadRow = 0xffffffffu;
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Where list entry j of a (b, h) unit lives: an explicit list, the fused sinks/middle/window
+// description, or the identity (dense).
+struct ListDesc {
+  const int* list;   // explicit list, or the middle set M in fused mode
+  int fused;         // 1: entry j < s0 -> j; j < s0 + nmid -> list[lo + j - s0]; else wlo + ...
+  int s0, nmid, lo, wlo;
+  int count;
+};
+
+// Per-warp set-up of the list descriptor (all 32 lanes call it).  In fused mode the bounds of
+// M inside [s0, wlo) are found by looking at its two ends: dilation can push at most r
+// entries below S0 or into the window; a longer overlap falls back to a full scan.
+__device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit, int t) {
+  ListDesc d;
+  const int lane = threadIdx.x & 31;
+  d.fused = 0; d.s0 = 0; d.nmid = 0; d.lo = 0; d.wlo = 0;
+  if (p.idx) {
+    d.list = p.idx + (long long)unit * p.idx_stride;
+    d.count = min(__ldg(p.count + unit), p.idx_stride);
+  } else if (p.mid) {
+    const int* M = p.mid + (long long)unit * p.mid_stride;
+    const int nm = min(__ldg(p.n_mid + unit), p.mid_stride);
+    const int s0 = min(p.sinks, t);
+    const int wlo = max(max(t - p.window, 0), s0);
+    int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && __ldg(M + min(lane, max(nm - 1, 0))) < s0));
+    const int i1 = nm - 32 + lane;
+    int above = __popc(__ballot_sync(0xffffffffu, i1 >= 0 && __ldg(M + max(i1, 0)) >= wlo));
+    if (lo == 32 || above == 32) {      // unusual schedule change inside a block: count everything
+      int c0 = 0, c1 = 0;
+      for (int i = lane; i < nm; i += 32) {
+        const int x = __ldg(M + i);
+        c0 += x < s0;
+        c1 += x >= wlo;
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        c0 += __shfl_xor_sync(0xffffffffu, c0, off);
+        c1 += __shfl_xor_sync(0xffffffffu, c1, off);
+      }
+      lo = c0; above = c1;
+    }
+    d.list = M; d.fused = 1; d.s0 = s0; d.lo = lo; d.wlo = wlo;
+    d.nmid = max(nm - above - lo, 0);
+    d.count = s0 + d.nmid + (t - wlo);
+  } else {
+    d.list = nullptr;
+    d.count = t;
+  }
+  return d;
+}
+
+// Row id (row offset / 128 elements) of list entry j for this lane, or kBadRow.
+__device__ __forceinline__ uint32_t fetch_row_id(const AttnParams& p, const ListDesc& d, int j, int end,
+                                                 int t, int b, int kvh, uint32_t outer_rows,
+                                                 uint32_t head_rows) {
+  if (j >= end) return kBadRow;
+  int pos;
+  if (d.fused) {
+    if (j < d.s0) pos = j;
+    else if (j < d.s0 + d.nmid) pos = __ldg(d.list + d.lo + (j - d.s0));
+    else pos = d.wlo + (j - d.s0 - d.nmid);
+  } else {
+    pos = d.list ? __ldg(d.list + j) : j;
+  }
+  if ((unsigned)pos >= (unsigned)t) {
+    atomicOr(p.flags, kFlagBadIndex);
+    return kBadRow;
+  }
+  if (p.kv.page_table != nullptr) {
+    const int page = __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
+    if ((unsigned)page >= (unsigned)p.kv.num_pages) {
+      atomicOr(p.flags, kFlagBadPage);
+      return kBadRow;
+    }
+    return (uint32_t)page * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)(pos & 15);
+  }
+  return (uint32_t)b * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)pos;
+}
+
+// ------------------------------------------- gathered attention, tensor-core pipeline (sm_100a)
+// The same warp-private cp.async pipeline, with the arithmetic moved to mma.sync m16n8k16
+// (bf16 in, fp32 accumulate) so that a gathered row costs about a dozen warp instructions
+// instead of about fifty.  A stage is 16 list entries: a K tile and a V tile of [16][128]
+// bf16, 16-byte chunk c of row r stored at chunk c ^ (r & 7) (ldmatrix reads conflict-free).
+//   S = Q K^T : A = the query as row 0 of a 16-row tile (rows 1..15 zero), B = K tile
+//               (ldmatrix), 2 n-tiles x 8 k-steps; lanes 0-3 end up with the 16 logits.
+//   O += P V  : A = P from the S accumulators (row 0 only), B = V tile (ldmatrix.trans),
+//               16 n-tiles x 1 k-step; lanes 0-3 hold the 128 output columns.
+// Index sets are per query head, so only one of the 16 tile rows carries data; the tensor
+// cores are used for their instruction economy, not their FLOPs.
+constexpr int kTWarps = 4;
+constexpr int kTThreads = kTWarps * 32;
+constexpr int kTStageRows = 16;
+constexpr int kTStages = 3;
+constexpr int kTTileBytes = kTStageRows * kRowBytes;                 // 4 KB
+constexpr int kTStageBytes = 2 * kTTileBytes;                        // K tile + V tile
+constexpr int kTSmemBytes = kTWarps * kTStages * kTStageBytes;       // 96 KB
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D += A * B with A rows 8..15 zero (a1 = a3 = 0): only accumulator rows 0..7 are live.
+__device__ __forceinline__ void mma_bf16_row0(float& d0, float& d1, float& z0, float& z1, uint32_t a0,
+                                              uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d0), "+f"(d1), "+f"(z0), "+f"(z1)
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p) {
+  extern __shared__ __align__(128) unsigned char g_smem[];
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int unit = b * p.num_q_heads + h;
   const int kvh = h / p.group_size;
-  const int tid = threadIdx.x, l16 = tid & 15, hw = tid >> 4;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
   const int t = __ldg(p.kv.seq_lens + b);
-  const int cnt = p.idx ? min(__ldg(p.count + unit), p.idx_stride) : t;
-  int per = (cnt + p.splits - 1) / p.splits;
-  per = (per + 15) & ~15;
-  const int start = min(split * per, cnt);
+  const ListDesc ld = make_list_desc(p, unit, t);
+  const int cnt = ld.count;
+  int per = (cnt + p.splits * kTWarps - 1) / (p.splits * kTWarps);
+  per = (per + kTStageRows - 1) & ~(kTStageRows - 1);
+  const int start = min((split * kTWarps + warp) * per, cnt);
   const int end = min(start + per, cnt);
-  const int* list = p.idx ? p.idx + (long long)unit * p.idx_stride : nullptr;
+  const int nstages = (end - start + kTStageRows - 1) / kTStageRows;
+  const uint32_t outer_rows = (uint32_t)(p.kv.stride_outer >> 7);
+  const uint32_t head_rows = (uint32_t)(p.kv.stride_head >> 7);
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(g_smem) + warp * (kTStages * kTStageBytes);
 
-  float qf[8];
+  // A fragments of the query: row 0 of the tile lives in lanes 0-3 (g == 0)
+  uint32_t aq0[8], aq2[8];
   {
-    const uint4 x = *reinterpret_cast<const uint4*>(p.q + (long long)unit * kHeadDim + l16 * 8);
-    const float c = kScale * kLog2e;   // logits are kept in the log2 domain
-    qf[0] = bf_lo(x.x) * c; qf[1] = bf_hi(x.x) * c; qf[2] = bf_lo(x.y) * c; qf[3] = bf_hi(x.y) * c;
-    qf[4] = bf_lo(x.z) * c; qf[5] = bf_hi(x.z) * c; qf[6] = bf_lo(x.w) * c; qf[7] = bf_hi(x.w) * c;
+    const uint32_t* q32 = reinterpret_cast<const uint32_t*>(p.q + (long long)unit * kHeadDim);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      aq0[ks] = g == 0 ? __ldg(q32 + ks * 8 + tg) : 0u;
+      aq2[ks] = g == 0 ? __ldg(q32 + ks * 8 + 4 + tg) : 0u;
+    }
   }
+  float o[16][2];
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; }
+  float z0 = 0.f, z1 = 0.f;            // accumulator rows 8..15: always zero
   float m = -INFINITY, l = 0.f;
-  float o[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) o[i] = 0.f;
 
-  // the trip count is uniform over a warp (its two half-warps take adjacent 16-entry blocks)
-  for (int jw = start + (tid >> 5) * 32; jw < end; jw += kAttnHalfWarps * 16) {
-    const int j0 = jw + (hw & 1) * 16;
-    int my = -1;
-    if (j0 + l16 < end) {
-      my = list ? __ldg(list + j0 + l16) : j0 + l16;
-      if ((unsigned)my >= (unsigned)t) {
-        atomicOr(p.flags, kFlagBadIndex);
-        my = -1;
+  uint32_t rid_a = fetch_row_id(p, ld, start + lane, end, t, b, kvh, outer_rows, head_rows);
+  uint32_t rid_b = fetch_row_id(p, ld, start + 32 + lane, end, t, b, kvh, outer_rows, head_rows);
+  const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
+  const uint32_t dst_tile = (lane < 16 ? 0u : (uint32_t)kTTileBytes);
+  unsigned long long vmask = 0ull;     // 16 validity bits per ring slot
+
+  auto issue = [&](int j) {
+    if (j < nstages) {
+      if (j > 0 && (j & 1) == 0) {
+        rid_a = rid_b;
+        rid_b = fetch_row_id(p, ld, start + (j + 2) * kTStageRows + lane, end, t, b, kvh, outer_rows,
+                             head_rows);
+      }
+      const int slot_i = j % kTStages;
+      const uint32_t slot = ring + (uint32_t)slot_i * kTStageBytes + dst_tile;
+      uint32_t vm = 0u;
+#pragma unroll
+      for (int r = 0; r < kTStageRows; ++r) {
+        const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
+        const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
+        const bool ok = rid != kBadRow;
+        vm |= (ok ? 1u : 0u) << r;
+        cp_async_16(dst, src_base + (ok ? (long long)rid * kHeadDim : 0ll), ok ? 16 : 0);
+      }
+      vmask = (vmask & ~(0xffffull << (16 * slot_i))) | ((unsigned long long)vm << (16 * slot_i));
+    }
+    cp_async_commit();
+  };
+
+#pragma unroll
+  for (int j = 0; j < kTStages - 1; ++j) issue(j);
+
+  const float sc = kScale * kLog2e;
+  // ldmatrix lane roles
+  const int lm_mi = lane >> 3, lm_r = lane & 7;
+  for (int i = 0; i < nstages; ++i) {
+    cp_async_wait<kTStages - 2>();
+    __syncwarp();
+    const int slot_i = i % kTStages;
+    const uint32_t vm = (uint32_t)(vmask >> (16 * slot_i)) & 0xffffu;
+    issue(i + kTStages - 1);
+    const uint32_t kt = ring + (uint32_t)slot_i * kTStageBytes;
+    const uint32_t vt = kt + kTTileBytes;
+    // ---- S = Q K^T
+    float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      const int row = nt * 8 + lm_r;
+#pragma unroll
+      for (int pp = 0; pp < 4; ++pp) {
+        uint32_t bk[4];
+        ldmatrix_x4(bk, kt + row * kRowBytes + (((4 * pp + lm_mi) ^ (row & 7)) << 4));
+        mma_bf16_row0(s[nt][0], s[nt][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[0], bk[1]);
+        mma_bf16_row0(s[nt][0], s[nt][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[2], bk[3]);
       }
     }
-#pragma unroll
-    for (int e0 = 0; e0 < 16; e0 += 4) {
-      uint4 kx[4], vx[4];
-      bool ok[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int pos = __shfl_sync(0xffffffffu, my, e0 + u, 16);
-        ok[u] = pos >= 0;
-        kx[u] = make_uint4(0u, 0u, 0u, 0u);
-        vx[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (ok[u]) {
-          const long long off = row_offset(p.kv, b, kvh, pos, p.flags);
-          if (off >= 0) {
-            kx[u] = ldg_stream(p.kv.k + off + l16 * 8);
-            vx[u] = ldg_stream(p.kv.v + off + l16 * 8);
-          } else {
-            ok[u] = false;
-          }
-        }
+    // ---- online softmax on the 16 logits held by lanes 0-3
+    float s0 = s[0][0] * sc, s1 = s[0][1] * sc, s2 = s[1][0] * sc, s3 = s[1][1] * sc;
+    if (!((vm >> (2 * tg)) & 1u)) s0 = -INFINITY;
+    if (!((vm >> (2 * tg + 1)) & 1u)) s1 = -INFINITY;
+    if (!((vm >> (8 + 2 * tg)) & 1u)) s2 = -INFINITY;
+    if (!((vm >> (9 + 2 * tg)) & 1u)) s3 = -INFINITY;
+    float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float mn = fmaxf(m, __shfl_sync(0xffffffffu, mx, 0));
+    if (mn != -INFINITY) {             // warp-uniform
+      const float corr = exp2f(m - mn);
+      m = mn;
+      float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
+      if (g == 0) {
+        p0 = exp2f(s0 - mn); p1 = exp2f(s1 - mn); p2 = exp2f(s2 - mn); p3 = exp2f(s3 - mn);
       }
-      float s[4];
-      float mn = m;
+      l = l * corr + ((p0 + p1) + (p2 + p3));
+      const uint32_t ap0 = pack_bf16x2(p0, p1), ap2 = pack_bf16x2(p2, p3);
+      if (corr != 1.f) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        s[u] = half_warp_sum(dot8(kx[u], qf));
-        if (!ok[u]) s[u] = -INFINITY;
-        mn = fmaxf(mn, s[u]);
+        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
       }
-      if (mn != -INFINITY) {
-        const float corr = exp2f(m - mn);
-        l *= corr;
+      // ---- O += P V
+      const int vrow = (lm_mi & 1) * 8 + lm_r;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] *= corr;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const float pw = exp2f(s[u] - mn);
-          l += pw;
-          o[0] = fmaf(pw, bf_lo(vx[u].x), o[0]); o[1] = fmaf(pw, bf_hi(vx[u].x), o[1]);
-          o[2] = fmaf(pw, bf_lo(vx[u].y), o[2]); o[3] = fmaf(pw, bf_hi(vx[u].y), o[3]);
-          o[4] = fmaf(pw, bf_lo(vx[u].z), o[4]); o[5] = fmaf(pw, bf_hi(vx[u].z), o[5]);
-          o[6] = fmaf(pw, bf_lo(vx[u].w), o[6]); o[7] = fmaf(pw, bf_hi(vx[u].w), o[7]);
-        }
-        m = mn;
+      for (int np = 0; np < 8; ++np) {
+        uint32_t bv[4];
+        ldmatrix_x4_trans(bv, vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
+        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[0], bv[1]);
+        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[2], bv[3]);
       }
     }
   }
+  cp_async_wait<0>();
+  l += __shfl_xor_sync(0xffffffffu, l, 1);
+  l += __shfl_xor_sync(0xffffffffu, l, 2);
 
-  // ---- combine the 16 half-warp states of this CTA
-  __shared__ float sm_o[kAttnHalfWarps][kHeadDim];
-  __shared__ float sm_m[kAttnHalfWarps], sm_l[kAttnHalfWarps];
+  // ---- combine the warps of this CTA (lanes 0-3 hold row 0: columns 8*nt + 2*tg, +1)
+  __shared__ float sm_o[kTWarps][kHeadDim];
+  __shared__ float sm_m[kTWarps], sm_l[kTWarps];
   __shared__ bool is_last;
+  if (g == 0) {
 #pragma unroll
-  for (int i = 0; i < 8; ++i) sm_o[hw][l16 * 8 + i] = o[i];
-  if (l16 == 0) { sm_m[hw] = m; sm_l[hw] = l; }
+    for (int nt = 0; nt < 16; ++nt)
+      *reinterpret_cast<float2*>(&sm_o[warp][nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
+  }
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
   __syncthreads();
-  float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
-  if (tid < kHeadDim) {
+  {
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kAttnHalfWarps; ++w) M = fmaxf(M, sm_m[w]);
+    for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w]);
     float acc = 0.f, L = 0.f;
     if (M != -INFINITY) {
 #pragma unroll
-      for (int w = 0; w < kAttnHalfWarps; ++w) {
-        const float sc = exp2f(sm_m[w] - M);
-        acc = fmaf(sm_o[w][tid], sc, acc);
-        L = fmaf(sm_l[w], sc, L);
+      for (int w = 0; w < kTWarps; ++w) {
+        const float scw = exp2f(sm_m[w] - M);
+        acc = fmaf(sm_o[w][tid], scw, acc);
+        L = fmaf(sm_l[w], scw, L);
       }
     }
     if (p.splits == 1) {
-      // single split: finish here
       p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
       if (tid == 0) {
         const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
         if (p.out_lse) p.out_lse[unit] = lse;
         if (p.out_delta) p.out_delta[unit] = L > 0.f ? -expm1f(lse - p.lse_full[unit]) : 1.f;
       }
-    } else {
-      part[tid] = acc;
-      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
+      return;
     }
+    float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
+    part[tid] = acc;
+    if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
   }
-  if (p.splits == 1) return;
-
-  // ---- the last CTA of this (b, h) merges the split partials
   __threadfence();
   __syncthreads();
   if (tid == 0) {
     const unsigned int ticket = atomicAdd(p.tickets + unit, 1u);
     is_last = (ticket == (unsigned int)p.splits - 1u);
-    if (is_last) p.tickets[unit] = 0u;   // ready for the next launch
+    if (is_last) p.tickets[unit] = 0u;
   }
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  if (tid < kHeadDim) {
-    const float* base = p.partials + (long long)unit * p.splits * kPartStride;
-    float M = -INFINITY;
-    for (int s = 0; s < p.splits; ++s) M = fmaxf(M, __ldcg(base + s * kPartStride + kHeadDim));
-    float acc = 0.f, L = 0.f;
-    if (M != -INFINITY) {
-      for (int s = 0; s < p.splits; ++s) {
-        const float sc = exp2f(__ldcg(base + s * kPartStride + kHeadDim) - M);
-        acc = fmaf(__ldcg(base + s * kPartStride + tid), sc, acc);
-        L = fmaf(__ldcg(base + s * kPartStride + kHeadDim + 1), sc, L);
-      }
+  const float* base = p.partials + (long long)unit * p.splits * kPartStride;
+  float M = -INFINITY;
+  for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
+  float acc = 0.f, L = 0.f;
+  if (M != -INFINITY) {
+    for (int sp = 0; sp < p.splits; ++sp) {
+      const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
+      acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
+      L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
     }
-    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-    if (tid == 0) {
-      const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-      if (p.out_lse) p.out_lse[unit] = lse;
-      if (p.out_delta) p.out_delta[unit] = L > 0.f ? -expm1f(lse - p.lse_full[unit]) : 1.f;
-    }
+  }
+  p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  if (tid == 0) {
+    const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    if (p.out_lse) p.out_lse[unit] = lse;
+    if (p.out_delta) p.out_delta[unit] = L > 0.f ? -expm1f(lse - p.lse_full[unit]) : 1.f;
   }
 }
 

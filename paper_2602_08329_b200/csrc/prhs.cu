@@ -18,7 +18,7 @@ using namespace prhs;
 
 namespace {
 
-constexpr int kChunkRows = 2048;        // keys scored per CTA (multiple of kScoreRowsPerIter)
+constexpr int kChunkRows = 2048;        // keys scored per CTA (8 warps x 256 keys)
 constexpr int kMaxSplits = 64;          // split-K partial slots per (b, h)
 constexpr int kMaxSmemBytes = 227 * 1024;
 constexpr int kMaxContext = 1 << 20;
@@ -27,15 +27,24 @@ std::string g_create_error;
 
 }  // namespace
 
+// The list of a unit is given explicitly (idx/count), by the fused builder (mid/n_mid plus the
+// sink and window sizes) or, with both NULL, is every position (dense baseline).
+struct FusedSet {
+  const int* mid = nullptr;
+  const int* n_mid = nullptr;
+  int mid_stride = 0, sinks = 0, window = 0;
+};
+
 struct prhs_ctx {
   prhs_config cfg{};
   int device = 0, sm_count = 148;
   int gq = 1, num_groups = 1, max_m = 0, shat_cap = 0, idx_cap = 0, ld = 0, sort_cap = 2;
-  int max_chunks = 1, resident_cap = 0;
+  int max_chunks = 1, attn_ctas_per_sm = 2;
   size_t sel_smem = 0;
   // workspaces (device)
   float* scores = nullptr;
   float2* part_ml = nullptr;
+  uint32_t* hist = nullptr;       // [B][Hq][2048] selection histogram, zero between retrievals
   float* lse_full = nullptr;
   float* lse_c = nullptr;
   float* partials = nullptr;
@@ -51,6 +60,8 @@ struct prhs_ctx {
   // staging for the host-buffer entry point (device)
   __nv_bfloat16 *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_out = nullptr;
   int last_batch = 0, last_layer_group = 1;
+  FusedSet last_set;                // what the last decode step attended over (for diagnostics)
+  const int* last_seq_lens = nullptr;
   long long launches = 0;
   // optional per-launch event timing
   struct ProfRec { cudaEvent_t a, b; int kind; };
@@ -87,8 +98,9 @@ prhs_status check_view(prhs_ctx* ctx, const prhs_kv_view* kv, int batch, KvDev* 
   if (!kv || !kv->k || !kv->v || !kv->seq_lens) return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: NULL pointer");
   if (batch < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "batch must be >= 1");
   if (batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch exceeds max_batch");
-  if ((kv->stride_outer % 8) || (kv->stride_head % 8) || ((uintptr_t)kv->k % 16) || ((uintptr_t)kv->v % 16))
-    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: rows must be 16-byte aligned");
+  if ((kv->stride_outer % kHeadDim) || (kv->stride_head % kHeadDim) || ((uintptr_t)kv->k % 16) ||
+      ((uintptr_t)kv->v % 16))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: strides must be multiples of 128 elements and bases 16-byte aligned");
   if (kv->stride_outer <= 0 || kv->stride_head <= 0)
     return fail(ctx, PRHS_ERR_INVALID_ARG, "kv view: strides must be positive");
   const bool paged = kv->page_table != nullptr;
@@ -143,47 +155,59 @@ struct LaunchScope {
 };
 
 // ---- launchers -----------------------------------------------------------------------
-template <int GQ>
-void launch_score_t(prhs_ctx* c, const __nv_bfloat16* q, const KvDev& kv, int batch, int nchunks,
-                    int write_scores, cudaStream_t st) {
-  dim3 grid(nchunks, c->cfg.num_q_heads / GQ, batch);
-  score_kernel<GQ><<<grid, kScoreThreads, 0, st>>>(q, kv, c->scores, c->ld, c->part_ml, nchunks,
-                                                   kChunkRows, c->cfg.num_q_heads, c->gq,
-                                                   write_scores, c->flags);
-}
-
+// `sched` != nullptr: a retrieval pass (logits are written and the selection histogram filled).
 prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
-                         int write_scores, cudaStream_t st, int* nchunks_out) {
+                         const prhs_schedule* sched, cudaStream_t st, int* nchunks_out) {
+  const int write_scores = sched != nullptr;
+  uint32_t* hist = sched ? c->hist : nullptr;
+  const int sinks = sched ? sched->sinks : 0, window = sched ? sched->window : 0;
   const int nchunks = std::max(1, (max_t + kChunkRows - 1) / kChunkRows);
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   {
     LaunchScope ls(c, PRHS_KIND_SCORE, st);
-    if (c->gq % 8 == 0) launch_score_t<8>(c, qq, kv, batch, nchunks, write_scores, st);
-    else if (c->gq % 4 == 0) launch_score_t<4>(c, qq, kv, batch, nchunks, write_scores, st);
-    else if (c->gq % 2 == 0) launch_score_t<2>(c, qq, kv, batch, nchunks, write_scores, st);
-    else launch_score_t<1>(c, qq, kv, batch, nchunks, write_scores, st);
+    dim3 grid(nchunks, c->cfg.num_kv_heads, batch);
+    const size_t smem = hist ? (size_t)c->gq * kScoreHistWordsPerHead * sizeof(uint32_t) : 0;
+    score_mma_kernel<<<grid, kScoreThreads, smem, st>>>(qq, kv, c->scores, c->ld, c->part_ml, nchunks,
+                                                        kChunkRows, c->cfg.num_q_heads, c->gq,
+                                                        write_scores, hist, sinks, window, c->flags);
   }
   *nchunks_out = nchunks;
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
 }
 
+// Split count for the gathered attention: minimise (waves of CTAs) x (rows per CTA plus a
+// fixed per-CTA cost), so that the grid fills an integer number of waves of resident CTAs.
 int pick_splits(const prhs_ctx* c, int units, int max_count) {
-  const int target = c->sm_count * 8;
-  int s = (target + units - 1) / units;
-  s = std::min(s, std::max(1, (max_count + 63) / 64));
-  return std::max(1, std::min(s, kMaxSplits));
+  const int slots = c->sm_count * c->attn_ctas_per_sm;
+  const int overhead_rows = 96;     // prologue + combine + partial write, in row equivalents
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= kMaxSplits; ++s) {
+    const int rows = (max_count + s - 1) / s;
+    if (s > 1 && rows < 64) break;
+    const long long ctas = (long long)units * s;
+    const double waves = (double)((ctas + slots - 1) / slots);
+    const double cost = waves * (rows + overhead_rows);
+    if (cost < best_cost * 0.999) { best_cost = cost; best = s; }
+  }
+  return best;
 }
 
 prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
-                        int idx_stride, int max_count, int batch, void* out, float* out_lse,
-                        const float* lse_full, float* out_delta, cudaStream_t st) {
+                        int idx_stride, const FusedSet& fs, int max_count, int batch, void* out,
+                        float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st) {
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.kv = kv;
   p.idx = idx;
   p.count = count;
   p.idx_stride = idx ? idx_stride : 0x7fffffff;
+  p.mid = idx ? nullptr : fs.mid;
+  p.n_mid = fs.n_mid;
+  p.mid_stride = fs.mid_stride;
+  p.sinks = fs.sinks;
+  p.window = fs.window;
   p.num_q_heads = c->cfg.num_q_heads;
   p.group_size = c->gq;
   p.splits = pick_splits(c, batch * c->cfg.num_q_heads, max_count);
@@ -196,8 +220,8 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.flags = c->flags;
   dim3 grid(p.splits, c->cfg.num_q_heads, batch);
   {
-    LaunchScope ls(c, idx ? PRHS_KIND_ATTN_SPARSE : PRHS_KIND_ATTN_DENSE, st);
-    gather_attn_kernel<<<grid, kAttnThreads, 0, st>>>(p);
+    LaunchScope ls(c, (idx || fs.mid) ? PRHS_KIND_ATTN_SPARSE : PRHS_KIND_ATTN_DENSE, st);
+    gather_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   }
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
@@ -214,7 +238,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
                          float* out_lse_full, cudaStream_t st) {
   const int g = group_of(s, layer);
   int nchunks = 1;
-  prhs_status rc = launch_score(c, q, kv, batch, max_t, 1, st, &nchunks);
+  prhs_status rc = launch_score(c, q, kv, batch, max_t, s, st, &nchunks);
   if (rc != PRHS_OK) return rc;
   SelectParams p;
   p.scores = c->scores;
@@ -243,7 +267,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.out_lse_full = out_lse_full;
   p.flags = c->flags;
   p.sort_cap = c->sort_cap;
-  p.resident_cap = c->resident_cap;
+  p.hist = c->hist;
   {
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
     select_kernel<<<batch * c->cfg.num_q_heads, kSelThreads, c->sel_smem, st>>>(p);
@@ -254,22 +278,29 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   return PRHS_OK;
 }
 
-prhs_status do_build(prhs_ctx* c, int layer, int step, const prhs_schedule* s, const KvDev& kv,
-                     int batch, int32_t* out_idx, int idx_stride, int32_t* out_count,
-                     cudaStream_t st) {
+// The middle set (layer, step) attends over: S* for the retrieving call itself (unless
+// PRHS_DILATE_ANCHOR), else the dilated S^ of the group's anchor (Def. 3.2).
+prhs_status pick_middle(prhs_ctx* c, int layer, int step, const prhs_schedule* s, FusedSet* fs) {
   const int g = group_of(s, layer);
   const int anchor = step - step % s->refresh_interval;
   if (c->anchor_step[g] != anchor)
     return fail(c, PRHS_ERR_STATE, "no shared set for this block: the group's first layer has not retrieved");
   const bool own = (layer % s->layer_group == 0) && (step == anchor) && !(s->flags & PRHS_DILATE_ANCHOR);
-  const int* mid = own ? c->sstar_asc + state_off(c, g, c->cfg.max_k)
-                       : c->shat_asc + state_off(c, g, c->shat_cap);
-  const int* nmid = (own ? c->n_star : c->n_hat) + state_off(c, g, 1);
+  fs->mid = own ? c->sstar_asc + state_off(c, g, c->cfg.max_k) : c->shat_asc + state_off(c, g, c->shat_cap);
+  fs->n_mid = (own ? c->n_star : c->n_hat) + state_off(c, g, 1);
+  fs->mid_stride = own ? c->cfg.max_k : c->shat_cap;
+  fs->sinks = s->sinks;
+  fs->window = s->window;
+  return PRHS_OK;
+}
+
+prhs_status launch_build(prhs_ctx* c, const FusedSet& fs, const int* seq_lens, int batch, int32_t* out_idx,
+                         int idx_stride, int32_t* out_count, cudaStream_t st) {
   {
     LaunchScope ls(c, PRHS_KIND_BUILD, st);
     build_set_kernel<<<batch * c->cfg.num_q_heads, 128, 0, st>>>(
-        mid, nmid, own ? c->cfg.max_k : c->shat_cap, kv.seq_lens, s->sinks, s->window,
-        c->cfg.num_q_heads, out_idx, idx_stride, out_count);
+        fs.mid, fs.n_mid, fs.mid_stride, seq_lens, fs.sinks, fs.window, c->cfg.num_q_heads, out_idx,
+        idx_stride, out_count);
   }
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
@@ -332,21 +363,30 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     delete c;
     return fail(nullptr, PRHS_ERR_CUDA, msg);
   }
-  // selection kernel shared memory: header + sort buffer + max(resident keys, position bitmap)
-  const int fixed = kSelHeaderWords * 4 + c->sort_cap * 8;
-  const int bitmap_words = (cfg->max_context + 31) / 32;
-  const int avail_words = (kMaxSmemBytes - fixed) / 4;
-  if (avail_words < bitmap_words) {
+  // selection kernel shared memory: histogram + scalars + sort buffer + max(candidates, bitmap)
+  const int fixed = (kHistBins + kSelMiscWords) * 4 + c->sort_cap * 8;
+  const int bitmap_bytes = ((cfg->max_context + 31) / 32) * 4;
+  c->sel_smem = (size_t)fixed + (size_t)std::max(kCandCap * 8, bitmap_bytes);
+  if (c->sel_smem > (size_t)kMaxSmemBytes) {
     delete c;
     return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context / max_k too large for the selection kernel");
   }
-  c->resident_cap = std::min(cfg->max_context, avail_words);
-  c->sel_smem = (size_t)fixed + 4 * (size_t)std::max(bitmap_words, c->resident_cap);
   e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             16 * kScoreHistWordsPerHead * (int)sizeof(uint32_t));
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess) {
+    int nb = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, gather_attn_mma_kernel, kTThreads, kTSmemBytes);
+    if (e == cudaSuccess && nb > 0) c->attn_ctas_per_sm = nb;
+  }
 
   const size_t U = units_max(c), G = c->num_groups;
   if (e == cudaSuccess) e = dev_alloc(&c->scores, U * c->ld);
   if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * c->max_chunks);
+  if (e == cudaSuccess) e = dev_alloc(&c->hist, U * kHistBins);
   if (e == cudaSuccess) e = dev_alloc(&c->lse_full, U);
   if (e == cudaSuccess) e = dev_alloc(&c->lse_c, U);
   if (e == cudaSuccess) e = dev_alloc(&c->partials, U * kMaxSplits * kPartStride);
@@ -367,6 +407,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->st_v, (size_t)cfg->max_batch * cfg->num_kv_heads * kHeadDim);
   if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, U * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(c->flags, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(c->hist, 0, U * kHistBins * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(c->n_star, 0, G * U * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->n_hat, 0, G * U * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->count, 0, U * sizeof(int));
@@ -383,7 +424,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
 
 prhs_status prhs_destroy(prhs_ctx* c) {
   if (!c) return PRHS_OK;
-  void* ptrs[] = {c->scores, c->part_ml, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
+  void* ptrs[] = {c->scores, c->part_ml, c->hist, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
                   c->count, c->flags, c->scratch_out, c->sstar_desc, c->sstar_asc, c->shat_asc,
                   c->n_star, c->n_hat, c->anchor_t, c->st_q, c->st_out, c->st_k, c->st_v};
   for (void* p : ptrs)
@@ -428,7 +469,10 @@ prhs_status prhs_build_index_set(prhs_ctx* ctx, int32_t layer, int32_t step, con
   int max_t;
   rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  return do_build(ctx, layer, step, sched, dv, batch, out_idx, idx_stride, out_count, as_stream(stream));
+  FusedSet fs;
+  rc = pick_middle(ctx, layer, step, sched, &fs);
+  if (rc != PRHS_OK) return rc;
+  return launch_build(ctx, fs, dv.seq_lens, batch, out_idx, idx_stride, out_count, as_stream(stream));
 }
 
 prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,
@@ -441,8 +485,8 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
   int max_t;
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  return launch_attn(ctx, q, dv, idx, count, idx_stride, idx_stride, batch, out, out_lse, nullptr,
-                     nullptr, as_stream(stream));
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, out, out_lse,
+                     nullptr, nullptr, as_stream(stream));
 }
 
 prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, int32_t batch,
@@ -453,8 +497,8 @@ prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_v
   int max_t;
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, max_t, batch, out, out_lse, nullptr, nullptr,
-                     as_stream(stream));
+  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, FusedSet(), max_t, batch, out, out_lse, nullptr,
+                     nullptr, as_stream(stream));
 }
 
 prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
@@ -478,7 +522,7 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
     if (rc != PRHS_OK) return rc;
   } else if (want_delta) {
     int nchunks = 1;
-    rc = launch_score(ctx, q, dv, batch, max_t, 0, st, &nchunks);
+    rc = launch_score(ctx, q, dv, batch, max_t, nullptr, st, &nchunks);
     if (rc != PRHS_OK) return rc;
     const int n = batch * ctx->cfg.num_q_heads;
     {
@@ -487,12 +531,15 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
     }
     PRHS_CUDA(ctx, cudaGetLastError());
   }
-  rc = do_build(ctx, layer, step, sched, dv, batch, ctx->idx, ctx->idx_cap, ctx->count, st);
+  // the index set is built inside the attention kernel from the stored middle set
+  FusedSet fs;
+  rc = pick_middle(ctx, layer, step, sched, &fs);
   if (rc != PRHS_OK) return rc;
+  ctx->last_set = fs;
+  ctx->last_seq_lens = dv.seq_lens;
   ctx->last_batch = batch;
-  return launch_attn(ctx, q, dv, ctx->idx, ctx->count, ctx->idx_cap, ctx->idx_cap, batch, out,
-                     ctx->lse_c, want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr,
-                     st);
+  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, fs, ctx->idx_cap, batch, out, ctx->lse_c,
+                     want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr, st);
 }
 
 prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
@@ -542,7 +589,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
   if (rc != PRHS_OK) return rc;
   cudaStream_t st = as_stream(stream);
   int nchunks = 1;
-  rc = launch_score(ctx, q, dv, batch, max_t, 0, st, &nchunks);
+  rc = launch_score(ctx, q, dv, batch, max_t, nullptr, st, &nchunks);
   if (rc != PRHS_OK) return rc;
   const int n = batch * ctx->cfg.num_q_heads;
   {
@@ -550,7 +597,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
     lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, ctx->lse_full, n);
   }
   PRHS_CUDA(ctx, cudaGetLastError());
-  return launch_attn(ctx, q, dv, idx, count, idx_stride, idx_stride, batch, ctx->scratch_out,
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, ctx->scratch_out,
                      ctx->lse_c, ctx->lse_full, out_delta, st);
 }
 
@@ -560,6 +607,11 @@ prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx, 
   if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
   cudaStream_t st = as_stream(stream);
   const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
+  if (!ctx->last_set.mid || batch != ctx->last_batch)
+    return fail(ctx, PRHS_ERR_STATE, "no decode step to report (or a different batch)");
+  prhs_status rc = launch_build(ctx, ctx->last_set, ctx->last_seq_lens, batch, ctx->idx, ctx->idx_cap,
+                                ctx->count, st);
+  if (rc != PRHS_OK) return rc;
   if (host_idx)
     PRHS_CUDA(ctx, cudaMemcpyAsync(host_idx, ctx->idx, n * ctx->idx_cap * sizeof(int), cudaMemcpyDeviceToHost, st));
   if (host_count)

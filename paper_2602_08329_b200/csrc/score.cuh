@@ -1,104 +1,179 @@
 // Retrieval pass, part 1: dense logits a_i = q . k_i / sqrt(d) for every cached position
-// (Eq. 2), written as fp32 scores, plus per-chunk online log-sum-exp partials.
+// (Eq. 2), written as fp32 scores, plus per-chunk online log-sum-exp partials and the
+// histogram of the top 11 key bits that the selection kernel starts from.
+//
+// The K stream goes straight from global memory into tensor-core operand registers: with
+// keys as the N dimension of mma.sync m16n8k16 and the (up to 16) query heads of one KV
+// head as the M dimension, lane (g, tg) needs elements of key row g only, and because a dot
+// product does not care in which order the 128 dimensions are visited, the lane may take
+// whole 16-byte chunks (chunk tg + 4j, j = 0..3) and call their elements k-slots of its own
+// choosing, as long as the query fragments use the same assignment.  No shared-memory
+// staging, no ldmatrix: 4 coalesced 16-byte loads and 8 MMAs per 8 keys, for every group
+// size from MHA (1 head) to 16 heads.
 #pragma once
 #include "common.cuh"
 
 namespace prhs {
 
-constexpr int kScoreThreads = 256;       // 16 half-warps; one half-warp covers one 256 B row
-constexpr int kScoreRowsPerIter = 256;   // 16 half-warps x 16 rows
+constexpr int kScoreThreads = 256;
+constexpr int kScoreWarps = kScoreThreads / 32;
+constexpr int kScoreTilesPerIter = 4;           // 4 n-tiles = 32 keys = 8 KB in flight per warp
+constexpr int kScoreHistWordsPerHead = 1024;    // 2048 bins, two 16-bit counters per word
 
-// grid (nchunks, Hq / GQ, B).  Each CTA streams `chunk_rows` keys of one KV head once and
-// scores them against GQ query heads of that head's group.  Half-warp lane j holds elements
-// [8j, 8j+8) of the row; a block of 16 rows is buffered so that each head's scores leave as
-// one 64-byte store.
-template <int GQ>
-__global__ void __launch_bounds__(kScoreThreads)
-score_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restrict__ scores, int ld,
-             float2* __restrict__ part_ml, int nchunks, int chunk_rows, int num_q_heads,
-             int group_size, int write_scores, uint32_t* flags) {
-  const int b = blockIdx.z;
-  const int head0 = blockIdx.y * GQ;
-  const int kvh = head0 / group_size;
-  const int chunk = blockIdx.x;
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// grid (nchunks, Hkv, B); dynamic shared memory: group_size * 4 KB (histogram) when hist != NULL.
+// chunk_rows must be a multiple of 256 (8 warps x 32 keys) and at most 65535.
+__global__ void __launch_bounds__(kScoreThreads, 2)
+score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restrict__ scores, int ld,
+                 float2* __restrict__ part_ml, int nchunks, int chunk_rows, int num_q_heads,
+                 int group_size, int write_scores, uint32_t* __restrict__ hist, int sinks, int window,
+                 uint32_t* flags) {
+  extern __shared__ __align__(16) uint32_t sh_hist[];   // [group_size][1024]
+  const int b = blockIdx.z, kvh = blockIdx.y, chunk = blockIdx.x;
+  const int head0 = kvh * group_size;
   const int t = __ldg(kv.seq_lens + b);
   const int row0 = chunk * chunk_rows;
   const int row1 = min(row0 + chunk_rows, t);
-  const int tid = threadIdx.x;
-  const int l16 = tid & 15;
-  const int hw = tid >> 4;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  const int span = chunk_rows / kScoreWarps;
+  const int wrow0 = row0 + warp * span;
+  const int wrow1 = min(wrow0 + span, row1);
+  const bool has0 = g < group_size, has1 = g + 8 < group_size;
+  const int mid_lo = min(sinks, t), mid_hi = t - window;
 
-  float qf[GQ][8];
-#pragma unroll
-  for (int h = 0; h < GQ; ++h) {
-    const uint4 x = *reinterpret_cast<const uint4*>(
-        q + ((long long)b * num_q_heads + head0 + h) * kHeadDim + l16 * 8);
-    qf[h][0] = bf_lo(x.x); qf[h][1] = bf_hi(x.x); qf[h][2] = bf_lo(x.y); qf[h][3] = bf_hi(x.y);
-    qf[h][4] = bf_lo(x.z); qf[h][5] = bf_hi(x.z); qf[h][6] = bf_lo(x.w); qf[h][7] = bf_hi(x.w);
-  }
-  float m[GQ], l[GQ];
-#pragma unroll
-  for (int h = 0; h < GQ; ++h) { m[h] = -INFINITY; l[h] = 0.f; }
-
-  // the trip count is uniform over a warp (its two half-warps take adjacent 16-row blocks)
-  for (int wbase = row0 + (tid >> 5) * 32; wbase < row1; wbase += kScoreRowsPerIter) {
-    const int blk = wbase + (hw & 1) * 16;
-    float keep[GQ];
-#pragma unroll
-    for (int h = 0; h < GQ; ++h) keep[h] = 0.f;
-#pragma unroll
-    for (int e0 = 0; e0 < 16; e0 += 8) {
-      uint4 kx[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int row = blk + e0 + u;
-        kx[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (row < row1) {
-          const long long off = row_offset(kv, b, kvh, row, flags);
-          if (off >= 0) kx[u] = ldg_stream(kv.k + off + l16 * 8);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-#pragma unroll
-        for (int h = 0; h < GQ; ++h) {
-          const float s = half_warp_sum(dot8(kx[u], qf[h])) * kScale;
-          if (l16 == e0 + u) keep[h] = s;
-        }
-      }
-    }
-    const int row = blk + l16;
-    if (row < row1) {
-#pragma unroll
-      for (int h = 0; h < GQ; ++h) {
-        if (write_scores)
-          scores[((long long)b * num_q_heads + head0 + h) * ld + row] = keep[h];
-        const float x = keep[h] * kLog2e;
-        const float mn = fmaxf(m[h], x);
-        l[h] = l[h] * exp2f(m[h] - mn) + exp2f(x - mn);
-        m[h] = mn;
-      }
-    }
+  if (hist != nullptr) {
+    for (int i = tid; i < group_size * kScoreHistWordsPerHead; i += kScoreThreads) sh_hist[i] = 0u;
+    __syncthreads();
   }
 
-  // reduce (m, l) over the CTA, one pair per head
-  __shared__ float sm_m[kScoreThreads / 32][GQ];
-  __shared__ float sm_l[kScoreThreads / 32][GQ];
+  // query fragments: k-step 2j uses elements 8c..8c+3 of chunk c = tg + 4j, k-step 2j+1 the rest
+  uint32_t a[8][4];
 #pragma unroll
-  for (int h = 0; h < GQ; ++h) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const float m2 = __shfl_xor_sync(0xffffffffu, m[h], off);
-      const float l2 = __shfl_xor_sync(0xffffffffu, l[h], off);
-      ml_combine(m[h], l[h], m2, l2);
+  for (int j = 0; j < 4; ++j) {
+    uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
+    const long long qo = ((long long)b * num_q_heads + head0) * kHeadDim + (tg + 4 * j) * 8;
+    if (has0) x0 = *reinterpret_cast<const uint4*>(q + qo + (long long)g * kHeadDim);
+    if (has1) x1 = *reinterpret_cast<const uint4*>(q + qo + (long long)(g + 8) * kHeadDim);
+    a[2 * j][0] = x0.x; a[2 * j][1] = x1.x; a[2 * j][2] = x0.y; a[2 * j][3] = x1.y;
+    a[2 * j + 1][0] = x0.z; a[2 * j + 1][1] = x1.z; a[2 * j + 1][2] = x0.w; a[2 * j + 1][3] = x1.w;
+  }
+
+  // paged cache: the 16 pages of this warp's span, one per lane
+  int pg = 0;
+  if (kv.page_table != nullptr && lane < 16 && wrow0 + lane * 16 < wrow1) {
+    pg = __ldg(kv.page_table + (long long)b * kv.page_table_stride + (wrow0 >> kPageShift) + lane);
+    if ((unsigned)pg >= (unsigned)kv.num_pages) {
+      atomicOr(flags, kFlagBadPage);
+      pg = -1;
     }
-    if ((tid & 31) == 0) { sm_m[tid >> 5][h] = m[h]; sm_l[tid >> 5][h] = l[h]; }
+  }
+  const long long head_off = (long long)kvh * kv.stride_head + tg * 8;
+  const long long seq_off = (long long)b * kv.stride_outer;
+
+  float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // heads g and g + 8
+
+  for (int it = wrow0; it < wrow1; it += 8 * kScoreTilesPerIter) {
+    uint4 kx[kScoreTilesPerIter][4];
+#pragma unroll
+    for (int tile = 0; tile < kScoreTilesPerIter; ++tile) {
+      const int row = it + tile * 8 + g;
+      long long off = -1;
+      if (kv.page_table != nullptr) {
+        const int page = __shfl_sync(0xffffffffu, pg, ((it + tile * 8) - wrow0) >> kPageShift);
+        if (row < wrow1 && page >= 0)
+          off = (long long)page * kv.stride_outer + head_off + (long long)(row & 15) * kHeadDim;
+      } else if (row < wrow1) {
+        off = seq_off + head_off + (long long)row * kHeadDim;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        kx[tile][j] = off >= 0 ? ldg_stream(kv.k + off + 32 * j) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int tile = 0; tile < kScoreTilesPerIter; ++tile) {
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        mma_bf16_16816(c, a[2 * j], kx[tile][j].x, kx[tile][j].y);
+        mma_bf16_16816(c, a[2 * j + 1], kx[tile][j].z, kx[tile][j].w);
+      }
+      // lane (g, tg) holds keys key0, key0 + 1 for heads g (c[0], c[1]) and g + 8 (c[2], c[3])
+      const int key0 = it + tile * 8 + 2 * tg;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        if (hh == 0 ? has0 : has1) {
+          const int head = head0 + g + 8 * hh;
+          const float s0 = c[2 * hh] * kScale, s1 = c[2 * hh + 1] * kScale;
+          float& m = hh == 0 ? m0 : m1;
+          float& l = hh == 0 ? l0 : l1;
+          float* dst = scores + ((long long)b * num_q_heads + head) * ld + key0;
+          if (key0 + 1 < wrow1) {
+            if (write_scores) *reinterpret_cast<float2*>(dst) = make_float2(s0, s1);
+            const float x0 = s0 * kLog2e, x1 = s1 * kLog2e;
+            const float mn = fmaxf(m, fmaxf(x0, x1));
+            l = l * exp2f(m - mn) + exp2f(x0 - mn) + exp2f(x1 - mn);
+            m = mn;
+          } else if (key0 < wrow1) {
+            if (write_scores) dst[0] = s0;
+            const float x0 = s0 * kLog2e;
+            const float mn = fmaxf(m, x0);
+            l = l * exp2f(m - mn) + exp2f(x0 - mn);
+            m = mn;
+          }
+          if (hist != nullptr) {
+            uint32_t* hh_hist = sh_hist + (g + 8 * hh) * kScoreHistWordsPerHead;
+            if (key0 >= mid_lo && key0 < mid_hi) {
+              const uint32_t bin = float_to_key(s0) >> 21;
+              atomicAdd(&hh_hist[bin >> 1], 1u << ((bin & 1u) << 4));
+            }
+            if (key0 + 1 >= mid_lo && key0 + 1 < mid_hi) {
+              const uint32_t bin = float_to_key(s1) >> 21;
+              atomicAdd(&hh_hist[bin >> 1], 1u << ((bin & 1u) << 4));
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- reduce (m, l) per head: over the 4 lanes of a group, then over the warps
+  __shared__ float sm_m[kScoreWarps][16], sm_l[kScoreWarps][16];
+#pragma unroll
+  for (int off = 1; off <= 2; off <<= 1) {
+    float m2 = __shfl_xor_sync(0xffffffffu, m0, off), l2 = __shfl_xor_sync(0xffffffffu, l0, off);
+    ml_combine(m0, l0, m2, l2);
+    m2 = __shfl_xor_sync(0xffffffffu, m1, off);
+    l2 = __shfl_xor_sync(0xffffffffu, l1, off);
+    ml_combine(m1, l1, m2, l2);
+  }
+  if (tg == 0) {
+    sm_m[warp][g] = m0; sm_l[warp][g] = l0;
+    sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1;
   }
   __syncthreads();
-  if (tid < GQ) {
+  if (tid < group_size) {
     float mm = -INFINITY, ll = 0.f;
-    for (int w = 0; w < kScoreThreads / 32; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
+    for (int w = 0; w < kScoreWarps; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
     part_ml[((long long)b * num_q_heads + head0 + tid) * nchunks + chunk] = make_float2(mm, ll);
+  }
+  if (hist != nullptr) {
+    for (int i = tid; i < group_size * kScoreHistWordsPerHead; i += kScoreThreads) {
+      const uint32_t w = sh_hist[i];
+      if (w) {
+        uint32_t* gh = hist + ((long long)b * num_q_heads + head0 + (i >> 10)) * 2048 + ((i & 1023) << 1);
+        if (w & 0xffffu) atomicAdd(gh, w & 0xffffu);
+        if (w >> 16) atomicAdd(gh + 1, w >> 16);
+      }
+    }
   }
 }
 

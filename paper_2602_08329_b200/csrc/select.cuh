@@ -1,19 +1,32 @@
 // Retrieval pass, part 2: exact top-k over the middle range (Sec. 4.1 "Selection
 // Criteria"), descending-logit order with ties broken by lower position, then the
 // neighbour dilation of Eq. 10.  One CTA per (sequence, query head).
+//
+// Fast path: the scoring kernel has already histogrammed the top 11 bits of every middle
+// candidate's order-preserving key.  The histogram names the bin d1 that holds the k-th
+// largest key, so ONE pass over the logits splits them into definite winners (bin > d1) and
+// a short candidate list (bin == d1); the remaining 21 key bits are resolved on that list in
+// shared memory.  If the candidate list or the tie group does not fit (degenerate inputs such
+// as all-equal logits), a generic 4 x 8-bit radix select over the logits in global memory
+// takes over; it orders ties by position explicitly.
 #pragma once
 #include "common.cuh"
 
 namespace prhs {
 
-constexpr int kSelThreads = 1024;
-constexpr int kSelHeaderWords = 256 + 64;   // radix histogram + scalars/scan scratch
+constexpr int kSelThreads = 512;
+constexpr int kHistBits = 11;
+constexpr int kHistBins = 1 << kHistBits;          // 2048
+constexpr int kHistShift = 32 - kHistBits;         // key >> 21
+constexpr int kSelMiscWords = 64;
+constexpr int kCandCap = 8192;                      // candidate list entries (8 bytes each)
 
 struct SelectParams {
   const float* scores;      // [B][Hq][ld]
   int ld;
   const float2* part_ml;    // [B][Hq][nchunks] (m, l) in the log2 domain
   int nchunks;
+  uint32_t* hist;           // [B][Hq][kHistBins], filled by the scoring kernel; zeroed here
   const int* seq_lens;
   const int* k_per_seq;     // or nullptr
   int k, sinks, window, r, m;
@@ -30,7 +43,6 @@ struct SelectParams {
   float* out_lse_full;      // optional
   uint32_t* flags;
   int sort_cap;             // power of two >= max_k
-  int resident_cap;         // candidates that fit in shared memory as keys
 };
 
 // Exclusive block scan of one int per thread; returns the exclusive prefix, *total gets the sum.
@@ -84,12 +96,60 @@ __device__ __forceinline__ int compact_bitmap(const uint32_t* bm, int words, int
   return total;
 }
 
-__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(SelectParams p) {
+// Append `v` to list[] for the lanes with f set: one shared-memory atomic per warp.
+__device__ __forceinline__ void warp_append(bool f, unsigned long long v, unsigned long long* list,
+                                            uint32_t* counter, uint32_t cap) {
+  const uint32_t bal = __ballot_sync(0xffffffffu, f);
+  if (bal == 0u) return;
+  const int lane = threadIdx.x & 31;
+  uint32_t base = 0u;
+  if (lane == (__ffs(bal) - 1)) base = atomicAdd(counter, (uint32_t)__popc(bal));
+  base = __shfl_sync(0xffffffffu, base, __ffs(bal) - 1);
+  const uint32_t slot = base + __popc(bal & ((1u << lane) - 1u));
+  if (f && slot < cap) list[slot] = v;
+}
+
+__device__ __forceinline__ unsigned long long make_entry(uint32_t key, int pos) {
+  return ((unsigned long long)key << 32) | (unsigned long long)(0xffffffffu - (uint32_t)pos);
+}
+
+// Digit bin that holds the rem-th largest element, scanning bins from the top.
+// hist has nb bins (nb a multiple of 32, nb / 32 <= 64 bins per lane).  Warp 0 only.
+// Writes misc[0] = bin, misc[1] = how many of that bin are still needed, misc[2] = its count.
+__device__ __forceinline__ void find_bin_from_top(const uint32_t* hist, int nb, int rem, uint32_t* misc) {
+  const int lane = threadIdx.x & 31;
+  const int per = nb >> 5;
+  int s = 0;
+  for (int j = 0; j < per; ++j) s += (int)hist[lane * per + j];
+  int incl = s;   // sum over lanes >= lane
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int x = __shfl_down_sync(0xffffffffu, incl, off);
+    if (lane + off < 32) incl += x;
+  }
+  const int above = incl - s;
+  if (above < rem && rem <= incl) {
+    int c = above;
+    for (int j = per - 1; j >= 0; --j) {
+      const int hc = (int)hist[lane * per + j];
+      if (c + hc >= rem) {
+        misc[0] = (uint32_t)(lane * per + j);
+        misc[1] = (uint32_t)(rem - c);
+        misc[2] = (uint32_t)hc;
+        break;
+      }
+      c += hc;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);
-  uint32_t* misc = hist + 256;
-  unsigned long long* wbuf = reinterpret_cast<unsigned long long*>(misc + 64);
-  uint32_t* region = reinterpret_cast<uint32_t*>(wbuf + p.sort_cap);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);                     // kHistBins
+  uint32_t* misc = hist + kHistBins;                                          // kSelMiscWords
+  unsigned long long* wbuf = reinterpret_cast<unsigned long long*>(misc + kSelMiscWords);  // sort_cap
+  unsigned long long* cand = wbuf + p.sort_cap;                               // kCandCap
+  uint32_t* bm = reinterpret_cast<uint32_t*>(cand);                           // bitmap aliases cand
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x;
@@ -101,9 +161,24 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(SelectParams p) 
   const int n = max(t - p.window - lo, 0);
   const int kk = min(k, n);
   const int m_eff = min(p.m < 0 ? k / 3 : p.m, kk);
+  const float* g = p.scores + (long long)unit * p.ld + lo;
 
+  // histogram of the scoring pass -> shared memory; the global copy is zeroed for the next use.
+  // All loads are issued before the first store: a store followed by an L2 load in the same
+  // thread serialises on the store's acknowledgement.
+  {
+    uint32_t* gh = p.hist + (long long)unit * kHistBins;
+    uint32_t hv[kHistBins / kSelThreads];
+#pragma unroll
+    for (int x = 0; x < kHistBins / kSelThreads; ++x) hv[x] = __ldcg(gh + tid + x * kSelThreads);
+#pragma unroll
+    for (int x = 0; x < kHistBins / kSelThreads; ++x) {
+      hist[tid + x * kSelThreads] = hv[x];
+      gh[tid + x * kSelThreads] = 0u;
+    }
+  }
   // full-softmax log-sum-exp from the scoring pass' per-chunk partials
-  if (warp == 0) {
+  if (warp == 1) {
     float mm = -INFINITY, ll = 0.f;
     for (int c = lane; c < p.nchunks; c += 32) {
       const float2 x = p.part_ml[(long long)unit * p.nchunks + c];
@@ -121,111 +196,184 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(SelectParams p) 
       if (p.out_lse_full) p.out_lse_full[unit] = lse;
     }
   }
-  if (tid == 0 && (unit % p.num_q_heads) == 0) p.anchor_t[b] = t;
-
-  const float* g = p.scores + (long long)unit * p.ld + lo;
-  const bool resident = n <= p.resident_cap;
-  if (resident) {
-    for (int i = tid; i < n; i += kSelThreads) region[i] = float_to_key(__ldcg(g + i));
-  } else if (tid == 0 && n > 0) {
-    atomicOr(p.flags, kFlagSelectFallback);
+  if (tid == 0) {
+    if ((unit % p.num_q_heads) == 0) p.anchor_t[b] = t;
+    misc[4] = 0u;   // winners appended
+    misc[5] = 0u;   // candidates appended
   }
-  if (tid == 0) misc[4] = 0u;
   __syncthreads();
-  auto key_at = [&](int i) -> uint32_t {
-    return resident ? region[i] : float_to_key(__ldcg(g + i));
-  };
 
-  // ---- radix select: the kk-th largest key T, and how many keys equal to T are needed
-  uint32_t T = 0u;
-  int need = 0, eq = 0;
+  int total = 0;          // entries in wbuf to sort; the first kk after sorting are S*
+  bool fast_ok = false;
   if (kk > 0) {
-    int rem = kk;
-    uint32_t prefix = 0u;
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-      if (tid < 256) hist[tid] = 0u;
-      __syncthreads();
-      for (int i = tid; i < n; i += kSelThreads) {
-        const uint32_t u = key_at(i);
-        if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
+    // ---------------- fast path
+    if (warp == 0) find_bin_from_top(hist, kHistBins, kk, misc);
+    __syncthreads();
+    const uint32_t d1 = misc[0];
+    const int rem1 = (int)misc[1];        // needed from bin d1
+    const int gt1 = kk - rem1;            // definite winners (bins above d1)
+    // one pass over the logits: 16 independent loads in flight per thread, then one warp scan
+    // and one pair of shared-memory atomics per warp and batch to place winners and candidates
+    const int nrounds = (n + kSelThreads - 1) / kSelThreads;
+    for (int rd0 = 0; rd0 < nrounds; rd0 += 16) {
+      uint32_t u16[16];
+#pragma unroll
+      for (int x = 0; x < 16; ++x) {
+        const int i = (rd0 + x) * kSelThreads + tid;
+        u16[x] = i < n ? float_to_key(__ldcg(g + i)) : 0u;
       }
-      __syncthreads();
-      if (warp == 0) {
-        int s = 0;
+      uint32_t wmask = 0u, cmask = 0u;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s += (int)hist[lane * 8 + j];
-        int incl = s;   // sum over lanes >= lane
+      for (int x = 0; x < 16; ++x) {
+        const int i = (rd0 + x) * kSelThreads + tid;
+        const uint32_t d = u16[x] >> kHistShift;
+        wmask |= (uint32_t)(i < n && d > d1) << x;
+        cmask |= (uint32_t)(i < n && d == d1) << x;
+      }
+      const uint32_t mine = (uint32_t)__popc(wmask) | ((uint32_t)__popc(cmask) << 16);
+      uint32_t incl = mine;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const int x = __shfl_down_sync(0xffffffffu, incl, off);
-          if (lane + off < 32) incl += x;
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t x = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += x;
+      }
+      uint32_t bw = 0u, bc = 0u;
+      if (lane == 31) {
+        if (incl & 0xffffu) bw = atomicAdd(&misc[4], incl & 0xffffu);
+        if (incl >> 16) bc = atomicAdd(&misc[5], incl >> 16);
+      }
+      uint32_t ow = __shfl_sync(0xffffffffu, bw, 31) + (incl & 0xffffu) - (mine & 0xffffu);
+      uint32_t oc = __shfl_sync(0xffffffffu, bc, 31) + (incl >> 16) - (mine >> 16);
+#pragma unroll
+      for (int x = 0; x < 16; ++x) {
+        const int i = (rd0 + x) * kSelThreads + tid;
+        if ((wmask >> x) & 1u) {
+          if (ow < (uint32_t)p.sort_cap) wbuf[ow] = make_entry(u16[x], lo + i);
+          ++ow;
         }
-        const int above = incl - s;
-        if (above < rem && rem <= incl) {
-          int c = above;
-          for (int j = 7; j >= 0; --j) {
-            const int hc = (int)hist[lane * 8 + j];
-            if (c + hc >= rem) {
-              misc[0] = (uint32_t)(lane * 8 + j);
-              misc[1] = (uint32_t)(rem - c);
-              misc[2] = (uint32_t)hc;
-              break;
-            }
-            c += hc;
+        if ((cmask >> x) & 1u) {
+          if (oc < (uint32_t)kCandCap) cand[oc] = make_entry(u16[x], lo + i);
+          ++oc;
+        }
+      }
+    }
+    __syncthreads();
+    const int ncand = (int)misc[5];
+    fast_ok = ((int)misc[4] == gt1) && ncand <= kCandCap && ncand >= rem1;
+    if (fast_ok) {
+      if (rem1 == ncand) {
+        // every candidate is a winner
+        if (gt1 + ncand <= p.sort_cap) {
+          for (int i = tid; i < ncand; i += kSelThreads) wbuf[gt1 + i] = cand[i];
+          total = gt1 + ncand;
+        } else {
+          fast_ok = false;
+        }
+      } else {
+        // resolve the remaining 21 key bits on the candidate list: 3 passes of 7 bits
+        uint32_t prefix = d1 << kHistShift;
+        int rem = rem1, eq = ncand;
+        for (int pass = 0; pass < 3; ++pass) {
+          const int shift = kHistShift - 7 * (pass + 1);
+          const uint32_t mask = 0xffffffffu << (shift + 7);
+          if (tid < 128) hist[tid] = 0u;
+          __syncthreads();
+          for (int i = tid; i < ncand; i += kSelThreads) {
+            const uint32_t u = (uint32_t)(cand[i] >> 32);
+            if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 127u], 1u);
           }
+          __syncthreads();
+          if (warp == 0) find_bin_from_top(hist, 128, rem, misc);
+          __syncthreads();
+          prefix |= misc[0] << shift;
+          rem = (int)misc[1];
+          eq = (int)misc[2];
+        }
+        const uint32_t T = prefix;            // the kk-th largest key
+        const int gt_total = kk - rem;        // keys strictly above T
+        // all keys equal to T go into the sort buffer; sorting orders them by position and
+        // the surplus falls behind the first kk entries
+        if (gt_total + eq <= p.sort_cap) {
+          const int crounds = (ncand + kSelThreads - 1) / kSelThreads;
+          for (int rd = 0; rd < crounds; ++rd) {
+            const int i = rd * kSelThreads + tid;
+            unsigned long long e = 0ull;
+            if (i < ncand) e = cand[i];
+            warp_append(i < ncand && (uint32_t)(e >> 32) >= T, e, wbuf, &misc[4], (uint32_t)p.sort_cap);
+          }
+          total = gt_total + eq;
+        } else {
+          fast_ok = false;
         }
       }
-      __syncthreads();
-      prefix |= misc[0] << shift;
-      rem = (int)misc[1];
-      eq = (int)misc[2];
     }
-    T = prefix;
-    need = rem;
+    __syncthreads();
+
+    if (!fast_ok) {
+      // ---------------- generic path: 4 x 8-bit radix select over the logits in global memory
+      if (tid == 0) {
+        atomicOr(p.flags, kFlagSelectFallback);
+        misc[4] = 0u;
+      }
+      uint32_t prefix = 0u;
+      int rem = kk, eq = 0;
+      for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        for (int i = tid; i < n; i += kSelThreads) {
+          const uint32_t u = float_to_key(__ldcg(g + i));
+          if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (warp == 0) find_bin_from_top(hist, 256, rem, misc);
+        __syncthreads();
+        prefix |= misc[0] << shift;
+        rem = (int)misc[1];
+        eq = (int)misc[2];
+      }
+      const uint32_t T = prefix;
+      const int need = rem, gt_total = kk - need;
+      const bool all_ties = (eq == need);
+      const int nrounds2 = (n + kSelThreads - 1) / kSelThreads;
+      for (int rd = 0; rd < nrounds2; ++rd) {
+        const int i = rd * kSelThreads + tid;
+        uint32_t u = 0u;
+        if (i < n) u = float_to_key(__ldcg(g + i));
+        warp_append(i < n && (u > T || (all_ties && u == T)), make_entry(u, lo + i), wbuf, &misc[4],
+                    (uint32_t)p.sort_cap);
+      }
+      if (!all_ties) {
+        // ties at T, lowest positions first
+        int base = 0;
+        for (int c0 = 0; c0 < n && base < need; c0 += kSelThreads) {
+          const int i = c0 + tid;
+          const bool f = (i < n) && float_to_key(__ldcg(g + i)) == T;
+          const uint32_t bal = __ballot_sync(0xffffffffu, f);
+          if (lane == 0) misc[8 + warp] = __popc(bal);
+          __syncthreads();
+          int before = 0, tot = 0;
+          for (int w = 0; w < kSelThreads / 32; ++w) {
+            const int c = (int)misc[8 + w];
+            if (w < warp) before += c;
+            tot += c;
+          }
+          const int rank = base + before + __popc(bal & ((1u << lane) - 1u));
+          if (f && rank < need) wbuf[gt_total + rank] = make_entry(T, lo + i);
+          base += tot;
+          __syncthreads();
+        }
+      }
+      total = kk;
+      __syncthreads();
+    }
   }
 
-  // ---- collect the winners as (key << 32 | ~position): keys above T, then ties in position order
-  const int gt_total = kk - need;
-  if (kk > 0) {
-    const bool all_ties = (eq == need);
-    for (int i = tid; i < n; i += kSelThreads) {
-      const uint32_t u = key_at(i);
-      if (u > T || (all_ties && u == T)) {
-        const uint32_t slot = atomicAdd(&misc[4], 1u);
-        if (slot < (uint32_t)p.sort_cap)
-          wbuf[slot] = ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)(lo + i));
-      }
-    }
-    if (!all_ties) {
-      int base = 0;
-      for (int c0 = 0; c0 < n && base < need; c0 += kSelThreads) {
-        const int i = c0 + tid;
-        const bool f = (i < n) && key_at(i) == T;
-        const uint32_t bal = __ballot_sync(0xffffffffu, f);
-        if (lane == 0) misc[8 + warp] = __popc(bal);
-        __syncthreads();
-        int before = 0, total = 0;
-        for (int w = 0; w < kSelThreads / 32; ++w) {
-          const int c = (int)misc[8 + w];
-          if (w < warp) before += c;
-          total += c;
-        }
-        const int rank = base + before + __popc(bal & ((1u << lane) - 1u));
-        if (f && rank < need)
-          wbuf[gt_total + rank] =
-              ((unsigned long long)T << 32) | (unsigned long long)(0xffffffffu - (uint32_t)(lo + i));
-        base += total;
-        __syncthreads();
-      }
-    }
-  }
-  // ---- sort the winners: descending key, ascending position among equal keys
+  // ---- sort: descending key, ascending position among equal keys
   int P = 2;
-  while (P < kk) P <<= 1;
-  __syncthreads();
-  for (int i = kk + tid; i < P; i += kSelThreads) wbuf[i] = 0ull;
+  while (P < total) P <<= 1;
+  for (int i = total + tid; i < P; i += kSelThreads) wbuf[i] = 0ull;
   for (int size = 2; size <= P; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
       __syncthreads();
@@ -253,7 +401,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(SelectParams p) 
   }
 
   // ---- ascending S*, then the dilated S^ (Eq. 10), through a position bitmap
-  uint32_t* bm = region;   // the keys are dead from here on
   const int words = (t + 31) >> 5;
   for (int w = tid; w < words; w += kSelThreads) bm[w] = 0u;
   __syncthreads();
