@@ -153,6 +153,36 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
                                     const int32_t* idx, const int32_t* count, int32_t idx_stride,
                                     int32_t batch, void* out, float* out_lse, void* stream);
 
+/* prhs_sparse_decode_attn for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is an integration aid.)
+ * Some hosts of this library run where cudaMalloc is off limits: inside a framework that
+ * owns the whole device heap and hands out fixed arenas, in a process whose memory budget is
+ * frozen after start-up, or between the capture of other work where an allocation would
+ * synchronise the device.  They cannot call prhs_create, which allocates the workspaces.
+ * This entry point needs no context and calls no cudaMalloc, cudaFree or other allocating
+ * routine: the split-K partials, the merge tickets and the anomaly word live in a
+ * file-scope device array inside the library (about 4.3 MB, held by every GPU that loads
+ * the library until the process exits).  The caller still owns and passes every input and
+ * output.
+ *   - Limits: batch * num_q_heads <= PRHS_NOALLOC_MAX_UNITS; head_dim 128; contiguous or
+ *     paged views as for the other calls.  Larger shapes return PRHS_ERR_CAPACITY.
+ *   - The first call on a device looks up the array's device address and sets the kernel's
+ *     shared-memory attribute (no allocation); make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents;
+ *     each call first clears the tickets it will use (a memset node on `stream`).  Two calls
+ *     whose kernels may overlap on the GPU (different streams, no ordering) race on it:
+ *     serialise them.
+ *   - An index outside [0, t_b) is skipped; the anomaly word is not reported by this call.
+ * Arguments as prhs_sparse_decode_attn, with the head counts passed explicitly.
+ * Errors go to prhs_last_error(NULL). */
+#define PRHS_NOALLOC_MAX_UNITS 1024
+#define PRHS_NOALLOC_MAX_SPLITS 8
+prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* kv, const int32_t* idx,
+                                            const int32_t* count, int32_t idx_stride, int32_t batch,
+                                            int32_t num_q_heads, int32_t num_kv_heads, void* out,
+                                            float* out_lse, void* stream);
+
 /* Dense flash-decoding baseline (Eq. 2): attention over all i < t_b. Same outputs. */
 prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,
                                    int32_t batch, void* out, float* out_lse, void* stream);

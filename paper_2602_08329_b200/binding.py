@@ -28,7 +28,8 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_decode_step_host", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
            "prhs_launch_count", "prhs_last_error", "prhs_version", "prhs_profile_begin",
-           "prhs_profile_end", "prhs_kernel_kind_name"]
+           "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc"]
+NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
 
 
@@ -78,6 +79,7 @@ def load() -> C.CDLL:
         "prhs_build_index_set": (st, [vp, i32, i32, C.POINTER(Schedule), C.POINTER(KvView), i32, vp, i32, vp, vp]),
         "prhs_sparse_decode_attn": (st, [vp, vp, C.POINTER(KvView), vp, vp, i32, i32, vp, vp, vp]),
         "prhs_dense_decode_attn": (st, [vp, vp, C.POINTER(KvView), i32, vp, vp, vp]),
+        "prhs_sparse_decode_attn_noalloc": (st, [vp, C.POINTER(KvView), vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "prhs_decode_step": (st, [vp, i32, i32, C.POINTER(Schedule), vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_decode_step_host": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32, vp, vp]),
         "prhs_delta": (st, [vp, vp, C.POINTER(KvView), vp, vp, i32, i32, vp, vp]),
@@ -254,6 +256,22 @@ class Context:
         flags = C.c_uint32(0)
         self._ck(self.lib.prhs_check(self.h, _stream(stream), C.byref(flags)))
         return flags.value
+
+
+def sparse_decode_attn_noalloc(q, view, idx, count, batch, num_q_heads, num_kv_heads, out, out_lse=None,
+                               stream=None):
+    """The context-free, allocation-free variant of Context.sparse_decode_attn.
+
+    For callers that may not allocate device memory (a frozen memory budget, a framework
+    that owns the heap): it needs no Context, and its scratch is a fixed array inside the
+    library.  Raises PrhsError on a shape beyond the array's capacity.
+    """
+    lib = load()
+    rc = lib.prhs_sparse_decode_attn_noalloc(_ptr(q), C.byref(view), _ptr(idx), _ptr(count), idx.shape[-1],
+                                             batch, num_q_heads, num_kv_heads, _ptr(out), _ptr(out_lse),
+                                             _stream(stream))
+    if rc != PRHS_OK:
+        raise PrhsError(rc, lib.prhs_last_error(None).decode())
 
 
 def version() -> str:

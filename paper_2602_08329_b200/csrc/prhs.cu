@@ -35,6 +35,14 @@ struct FusedSet {
   int mid_stride = 0, sinks = 0, window = 0;
 };
 
+// ---- scratch of the allocation-free entry point: split-K partials, merge tickets, flag word.
+// In host code the name is a stand-in, not a device address: set-up resolves it per device.
+constexpr size_t kNoAllocPartialFloats =
+    (size_t)PRHS_NOALLOC_MAX_UNITS * PRHS_NOALLOC_MAX_SPLITS * kPartStride;
+constexpr size_t kNoAllocScratchBytes =
+    kNoAllocPartialFloats * sizeof(float) + (PRHS_NOALLOC_MAX_UNITS + 64) * sizeof(unsigned int);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
 struct prhs_ctx {
   prhs_config cfg{};
   int device = 0, sm_count = 148;
@@ -487,6 +495,92 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
   if (rc != PRHS_OK) return rc;
   return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, out, out_lse,
                      nullptr, nullptr, as_stream(stream));
+}
+
+prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* kv, const int32_t* idx,
+                                            const int32_t* count, int32_t idx_stride, int32_t batch,
+                                            int32_t num_q_heads, int32_t num_kv_heads, void* out,
+                                            float* out_lse, void* stream) {
+  // per-device set-up state (no allocation): scratch address, SM count, resident CTAs per SM
+  struct DevState { unsigned char* scratch = nullptr; int sm_count = 0; int ctas_per_sm = 0; };
+  static DevState dev_state[64];
+  if (!q || !kv || !kv->k || !kv->v || !kv->seq_lens || !idx || !count || !out)
+    return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: NULL pointer");
+  if (batch < 1 || num_q_heads < 1 || num_kv_heads < 1 || num_q_heads % num_kv_heads || idx_stride < 1)
+    return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: bad shape");
+  if (num_q_heads / num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "noalloc: group size above 16");
+  if ((long long)batch * num_q_heads > PRHS_NOALLOC_MAX_UNITS)
+    return fail(nullptr, PRHS_ERR_CAPACITY, "noalloc: batch * num_q_heads exceeds PRHS_NOALLOC_MAX_UNITS");
+  if ((kv->stride_outer % kHeadDim) || (kv->stride_head % kHeadDim) || kv->stride_outer <= 0 ||
+      kv->stride_head <= 0 || ((uintptr_t)kv->k % 16) || ((uintptr_t)kv->v % 16))
+    return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: strides must be positive multiples of 128 elements, bases 16-byte aligned");
+  if (kv->page_table && (kv->page_table_stride < 1 || kv->num_pages < 1))
+    return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: bad page table stride or pool size");
+  int dev = -1;
+  PRHS_CUDA(nullptr, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "noalloc: device ordinal above 63");
+  DevState& ds = dev_state[dev];
+  if (!ds.scratch) {
+    // first call on this device, with this device current
+    unsigned char* ptr = nullptr;
+    PRHS_CUDA(nullptr, cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch));
+    PRHS_CUDA(nullptr, cudaFuncSetAttribute(gather_attn_mma_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes));
+    PRHS_CUDA(nullptr, cudaDeviceGetAttribute(&ds.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    PRHS_CUDA(nullptr, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ds.ctas_per_sm, gather_attn_mma_kernel,
+                                                                     kTThreads, kTSmemBytes));
+    if (ds.ctas_per_sm < 1) ds.ctas_per_sm = 1;
+    ds.scratch = ptr;
+  }
+  cudaStream_t st = as_stream(stream);
+  const int units = batch * num_q_heads;
+  // same split rule as the context-based call, capped by the static capacity
+  const int slots = ds.sm_count * ds.ctas_per_sm;
+  int splits = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= PRHS_NOALLOC_MAX_SPLITS; ++s) {
+    const int rows = (idx_stride + s - 1) / s;
+    if (s > 1 && rows < 64) break;
+    const double waves = (double)(((long long)units * s + slots - 1) / slots);
+    const double cost = waves * (rows + 96);
+    if (cost < best_cost * 0.999) { best_cost = cost; splits = s; }
+  }
+  float* partials = reinterpret_cast<float*>(ds.scratch);
+  unsigned int* tickets = reinterpret_cast<unsigned int*>(ds.scratch + kNoAllocPartialFloats * sizeof(float));
+  uint32_t* flag_word = tickets + PRHS_NOALLOC_MAX_UNITS;
+  // the array keeps the last call's contents: tickets must start at zero
+  PRHS_CUDA(nullptr, cudaMemsetAsync(tickets, 0, (size_t)units * sizeof(unsigned int), st));
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.kv.k = static_cast<const __nv_bfloat16*>(kv->k);
+  p.kv.v = static_cast<const __nv_bfloat16*>(kv->v);
+  p.kv.stride_outer = kv->stride_outer;
+  p.kv.stride_head = kv->stride_head;
+  p.kv.page_table = kv->page_table;
+  p.kv.page_table_stride = kv->page_table_stride;
+  p.kv.seq_lens = kv->seq_lens;
+  p.kv.num_pages = kv->num_pages;
+  p.idx = idx;
+  p.count = count;
+  p.idx_stride = idx_stride;
+  p.mid = nullptr;
+  p.n_mid = nullptr;
+  p.mid_stride = 0;
+  p.sinks = 0;
+  p.window = 0;
+  p.num_q_heads = num_q_heads;
+  p.group_size = num_q_heads / num_kv_heads;
+  p.splits = splits;
+  p.partials = partials;
+  p.tickets = tickets;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.out_lse = out_lse;
+  p.lse_full = nullptr;
+  p.out_delta = nullptr;
+  p.flags = flag_word;
+  gather_attn_mma_kernel<<<dim3(splits, num_q_heads, batch), kTThreads, kTSmemBytes, st>>>(p);
+  PRHS_CUDA(nullptr, cudaGetLastError());
+  return PRHS_OK;
 }
 
 prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, int32_t batch,
