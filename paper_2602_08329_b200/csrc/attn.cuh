@@ -412,12 +412,15 @@ __global__ void delta_kernel(const float* __restrict__ lse_c, const float* __res
 }
 
 // Reduce the scoring pass' per-chunk (m, l) partials to lse_full (used when no selection runs).
-__global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunks,
+__global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunks, int chunk_rows,
+                                  const int* __restrict__ seq_lens, int num_q_heads,
                                   float* __restrict__ lse_full, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
+  const int t = __ldg(seq_lens + i / num_q_heads);
+  const int nch = min(nchunks, (t + chunk_rows - 1) / chunk_rows);   // later chunks were never written
   float mm = -INFINITY, ll = 0.f;
-  for (int c = 0; c < nchunks; ++c) {
+  for (int c = 0; c < nch; ++c) {
     const float2 x = part_ml[(long long)i * nchunks + c];
     ml_combine(mm, ll, x.x, x.y);
   }

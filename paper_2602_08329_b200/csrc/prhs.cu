@@ -52,7 +52,6 @@ struct prhs_ctx {
   // workspaces (device)
   float* scores = nullptr;
   float2* part_ml = nullptr;
-  uint32_t* hist = nullptr;       // [B][Hq][2048] selection histogram, zero between retrievals
   float* lse_full = nullptr;
   float* lse_c = nullptr;
   float* partials = nullptr;
@@ -167,17 +166,17 @@ struct LaunchScope {
 prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
                          const prhs_schedule* sched, cudaStream_t st, int* nchunks_out) {
   const int write_scores = sched != nullptr;
-  uint32_t* hist = sched ? c->hist : nullptr;
-  const int sinks = sched ? sched->sinks : 0, window = sched ? sched->window : 0;
   const int nchunks = std::max(1, (max_t + kChunkRows - 1) / kChunkRows);
   const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
   {
     LaunchScope ls(c, PRHS_KIND_SCORE, st);
-    dim3 grid(nchunks, c->cfg.num_kv_heads, batch);
-    const size_t smem = hist ? (size_t)c->gq * kScoreHistWordsPerHead * sizeof(uint32_t) : 0;
+    const size_t smem = (size_t)(batch + 1) * sizeof(int);
+    const long long max_items = (long long)batch * c->cfg.num_kv_heads * nchunks;
+    const int grid = (int)std::max<long long>(1, std::min<long long>(max_items, (long long)c->sm_count * 2));
     score_mma_kernel<<<grid, kScoreThreads, smem, st>>>(qq, kv, c->scores, c->ld, c->part_ml, nchunks,
-                                                        kChunkRows, c->cfg.num_q_heads, c->gq,
-                                                        write_scores, hist, sinks, window, c->flags);
+                                                        kChunkRows, c->cfg.num_q_heads,
+                                                        c->cfg.num_kv_heads, batch, write_scores,
+                                                        c->flags);
   }
   *nchunks_out = nchunks;
   PRHS_CUDA(c, cudaGetLastError());
@@ -253,6 +252,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.ld = c->ld;
   p.part_ml = c->part_ml;
   p.nchunks = nchunks;
+  p.chunk_rows = kChunkRows;
   p.seq_lens = kv.seq_lens;
   p.k_per_seq = s->top_k_per_seq;
   p.k = s->top_k;
@@ -275,7 +275,6 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.out_lse_full = out_lse_full;
   p.flags = c->flags;
   p.sort_cap = c->sort_cap;
-  p.hist = c->hist;
   {
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
     select_kernel<<<batch * c->cfg.num_q_heads, kSelThreads, c->sel_smem, st>>>(p);
@@ -362,6 +361,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   c->ld = (cfg->max_context + 63) & ~63;
   c->max_chunks = (cfg->max_context + kChunkRows - 1) / kChunkRows;
   while (c->sort_cap < cfg->max_k) c->sort_cap <<= 1;
+  c->sort_cap <<= 1;   // room for a tie group that straddles the k-th place
   c->anchor_step.assign(c->num_groups, -1);
 
   cudaError_t e = cudaGetDevice(&c->device);
@@ -382,7 +382,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             16 * kScoreHistWordsPerHead * (int)sizeof(uint32_t));
+                             std::max(1024, (cfg->max_batch + 1) * (int)sizeof(int)));
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess) {
@@ -394,7 +394,6 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   const size_t U = units_max(c), G = c->num_groups;
   if (e == cudaSuccess) e = dev_alloc(&c->scores, U * c->ld);
   if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * c->max_chunks);
-  if (e == cudaSuccess) e = dev_alloc(&c->hist, U * kHistBins);
   if (e == cudaSuccess) e = dev_alloc(&c->lse_full, U);
   if (e == cudaSuccess) e = dev_alloc(&c->lse_c, U);
   if (e == cudaSuccess) e = dev_alloc(&c->partials, U * kMaxSplits * kPartStride);
@@ -415,7 +414,6 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->st_v, (size_t)cfg->max_batch * cfg->num_kv_heads * kHeadDim);
   if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, U * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(c->flags, 0, sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMemset(c->hist, 0, U * kHistBins * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(c->n_star, 0, G * U * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->n_hat, 0, G * U * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->count, 0, U * sizeof(int));
@@ -432,7 +430,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
 
 prhs_status prhs_destroy(prhs_ctx* c) {
   if (!c) return PRHS_OK;
-  void* ptrs[] = {c->scores, c->part_ml, c->hist, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
+  void* ptrs[] = {c->scores, c->part_ml, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
                   c->count, c->flags, c->scratch_out, c->sstar_desc, c->sstar_asc, c->shat_asc,
                   c->n_star, c->n_hat, c->anchor_t, c->st_q, c->st_out, c->st_k, c->st_v};
   for (void* p : ptrs)
@@ -621,7 +619,8 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
     const int n = batch * ctx->cfg.num_q_heads;
     {
       LaunchScope ls(ctx, PRHS_KIND_MISC, st);
-      lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, ctx->lse_full, n);
+      lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, kChunkRows, dv.seq_lens,
+                                                         ctx->cfg.num_q_heads, ctx->lse_full, n);
     }
     PRHS_CUDA(ctx, cudaGetLastError());
   }
@@ -688,7 +687,8 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
   const int n = batch * ctx->cfg.num_q_heads;
   {
     LaunchScope ls(ctx, PRHS_KIND_MISC, st);
-    lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, ctx->lse_full, n);
+    lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, kChunkRows, dv.seq_lens,
+                                                         ctx->cfg.num_q_heads, ctx->lse_full, n);
   }
   PRHS_CUDA(ctx, cudaGetLastError());
   return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, ctx->scratch_out,

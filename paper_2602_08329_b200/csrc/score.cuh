@@ -1,6 +1,5 @@
 // Retrieval pass, part 1: dense logits a_i = q . k_i / sqrt(d) for every cached position
-// (Eq. 2), written as fp32 scores, plus per-chunk online log-sum-exp partials and the
-// histogram of the top 11 key bits that the selection kernel starts from.
+// (Eq. 2), written as fp32 scores, plus per-chunk online log-sum-exp partials.
 //
 // The K stream goes straight from global memory into tensor-core operand registers: with
 // keys as the N dimension of mma.sync m16n8k16 and the (up to 16) query heads of one KV
@@ -18,7 +17,6 @@ namespace prhs {
 constexpr int kScoreThreads = 256;
 constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kScoreTilesPerIter = 4;           // 4 n-tiles = 32 keys = 8 KB in flight per warp
-constexpr int kScoreHistWordsPerHead = 1024;    // 2048 bins, two 16-bit counters per word
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
                                                uint32_t b1) {
@@ -29,34 +27,60 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// grid (nchunks, Hkv, B); dynamic shared memory: group_size * 4 KB (histogram) when hist != NULL.
-// chunk_rows must be a multiple of 256 (8 warps x 32 keys) and at most 65535.
+// Persistent CTAs: grid.x CTAs share the work items (unit, chunk) -- unit = (b, kvh), chunk =
+// chunk_rows consecutive keys -- in unit-major order, each CTA taking one contiguous range, so
+// that the grid is exactly one wave and the query fragments are reloaded only when the unit
+// changes.  Dynamic shared memory: (batch + 1) ints.  chunk_rows: a multiple of 256 (8 warps
+// x 32 keys).
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restrict__ scores, int ld,
                  float2* __restrict__ part_ml, int nchunks, int chunk_rows, int num_q_heads,
-                 int group_size, int write_scores, uint32_t* __restrict__ hist, int sinks, int window,
-                 uint32_t* flags) {
-  extern __shared__ __align__(16) uint32_t sh_hist[];   // [group_size][1024]
-  const int b = blockIdx.z, kvh = blockIdx.y, chunk = blockIdx.x;
-  const int head0 = kvh * group_size;
-  const int t = __ldg(kv.seq_lens + b);
-  const int row0 = chunk * chunk_rows;
-  const int row1 = min(row0 + chunk_rows, t);
+                 int num_kv_heads, int batch, int write_scores, uint32_t* flags) {
+  extern __shared__ __align__(16) uint32_t sh_dyn[];
+  const int group_size = num_q_heads / num_kv_heads;
+  int* cum = reinterpret_cast<int*>(sh_dyn);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;
-  const int span = chunk_rows / kScoreWarps;
-  const int wrow0 = row0 + warp * span;
-  const int wrow1 = min(wrow0 + span, row1);
   const bool has0 = g < group_size, has1 = g + 8 < group_size;
-  const int mid_lo = min(sinks, t), mid_hi = t - window;
 
-  if (hist != nullptr) {
-    for (int i = tid; i < group_size * kScoreHistWordsPerHead; i += kScoreThreads) sh_hist[i] = 0u;
-    __syncthreads();
+  // items per sequence: Hkv * ceil(t_b / chunk_rows); exclusive prefix in cum[0..batch]
+  for (int b = tid; b < batch; b += kScoreThreads) {
+    const int t = __ldg(kv.seq_lens + b);
+    cum[b + 1] = num_kv_heads * ((max(t, 0) + chunk_rows - 1) / chunk_rows);
   }
+  __syncthreads();
+  if (tid == 0) {
+    cum[0] = 0;
+    for (int b = 0; b < batch; ++b) cum[b + 1] += cum[b];
+  }
+  __syncthreads();
+  const int total_items = cum[batch];
+  const int item0 = (int)(((long long)total_items * blockIdx.x) / gridDim.x);
+  const int item1 = (int)(((long long)total_items * (blockIdx.x + 1)) / gridDim.x);
 
-  // query fragments: k-step 2j uses elements 8c..8c+3 of chunk c = tg + 4j, k-step 2j+1 the rest
+  __shared__ float sm_m[kScoreWarps][16], sm_l[kScoreWarps][16];
+  int b = 0;
+  int cur_unit = -1;       // unit whose query fragments are loaded
   uint32_t a[8][4];
+
+  for (int item = item0; item < item1; ++item) {
+    while (cum[b + 1] <= item) ++b;
+    const int t = __ldg(kv.seq_lens + b);
+    const int nch_b = (t + chunk_rows - 1) / chunk_rows;
+    const int local = item - cum[b];
+    const int kvh = local / nch_b;
+    const int chunk = local - kvh * nch_b;
+    const int unit = b * num_kv_heads + kvh;
+    const int head0 = kvh * group_size;
+    const int row0 = chunk * chunk_rows;
+    const int row1 = min(row0 + chunk_rows, t);
+    const int span = chunk_rows / kScoreWarps;
+    const int wrow0 = row0 + warp * span;
+    const int wrow1 = min(wrow0 + span, row1);
+
+    if (unit != cur_unit) {
+      cur_unit = unit;
+  // query fragments: k-step 2j uses elements 8c..8c+3 of chunk c = tg + 4j, k-step 2j+1 the rest
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     uint4 x0 = make_uint4(0u, 0u, 0u, 0u), x1 = x0;
@@ -66,6 +90,7 @@ score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restric
     a[2 * j][0] = x0.x; a[2 * j][1] = x1.x; a[2 * j][2] = x0.y; a[2 * j][3] = x1.y;
     a[2 * j + 1][0] = x0.z; a[2 * j + 1][1] = x1.z; a[2 * j + 1][2] = x0.w; a[2 * j + 1][3] = x1.w;
   }
+    }   // unit change
 
   // paged cache: the 16 pages of this warp's span, one per lane
   int pg = 0;
@@ -129,24 +154,12 @@ score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restric
             l = l * exp2f(m - mn) + exp2f(x0 - mn);
             m = mn;
           }
-          if (hist != nullptr) {
-            uint32_t* hh_hist = sh_hist + (g + 8 * hh) * kScoreHistWordsPerHead;
-            if (key0 >= mid_lo && key0 < mid_hi) {
-              const uint32_t bin = float_to_key(s0) >> 21;
-              atomicAdd(&hh_hist[bin >> 1], 1u << ((bin & 1u) << 4));
-            }
-            if (key0 + 1 >= mid_lo && key0 + 1 < mid_hi) {
-              const uint32_t bin = float_to_key(s1) >> 21;
-              atomicAdd(&hh_hist[bin >> 1], 1u << ((bin & 1u) << 4));
-            }
-          }
         }
       }
     }
   }
 
   // ---- reduce (m, l) per head: over the 4 lanes of a group, then over the warps
-  __shared__ float sm_m[kScoreWarps][16], sm_l[kScoreWarps][16];
 #pragma unroll
   for (int off = 1; off <= 2; off <<= 1) {
     float m2 = __shfl_xor_sync(0xffffffffu, m0, off), l2 = __shfl_xor_sync(0xffffffffu, l0, off);
@@ -155,6 +168,7 @@ score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restric
     l2 = __shfl_xor_sync(0xffffffffu, l1, off);
     ml_combine(m1, l1, m2, l2);
   }
+  __syncthreads();           // the previous item's partials have been read
   if (tg == 0) {
     sm_m[warp][g] = m0; sm_l[warp][g] = l0;
     sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1;
@@ -165,16 +179,8 @@ score_mma_kernel(const __nv_bfloat16* __restrict__ q, KvDev kv, float* __restric
     for (int w = 0; w < kScoreWarps; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
     part_ml[((long long)b * num_q_heads + head0 + tid) * nchunks + chunk] = make_float2(mm, ll);
   }
-  if (hist != nullptr) {
-    for (int i = tid; i < group_size * kScoreHistWordsPerHead; i += kScoreThreads) {
-      const uint32_t w = sh_hist[i];
-      if (w) {
-        uint32_t* gh = hist + ((long long)b * num_q_heads + head0 + (i >> 10)) * 2048 + ((i & 1023) << 1);
-        if (w & 0xffffu) atomicAdd(gh, w & 0xffffu);
-        if (w >> 16) atomicAdd(gh + 1, w >> 16);
-      }
-    }
-  }
+  }   // items
+
 }
 
 }  // namespace prhs

@@ -2,13 +2,15 @@
 // Criteria"), descending-logit order with ties broken by lower position, then the
 // neighbour dilation of Eq. 10.  One CTA per (sequence, query head).
 //
-// Fast path: the scoring kernel has already histogrammed the top 11 bits of every middle
-// candidate's order-preserving key.  The histogram names the bin d1 that holds the k-th
-// largest key, so ONE pass over the logits splits them into definite winners (bin > d1) and
-// a short candidate list (bin == d1); the remaining 21 key bits are resolved on that list in
-// shared memory.  If the candidate list or the tie group does not fit (degenerate inputs such
-// as all-equal logits), a generic 4 x 8-bit radix select over the logits in global memory
-// takes over; it orders ties by position explicitly.
+// Fast path: a 1-in-16 sample of the unit's logits is histogrammed on the top 11 bits of the
+// order-preserving key; from it a conservative bin d_lo is chosen so that, with a wide
+// margin, at least k logits lie in bins >= d_lo.  ONE pass over all logits then collects those
+// into a short list in shared memory (about 1.5-2 k entries), and everything else -- the exact
+// bin of the k-th key, the remaining 21 key bits, ties -- is resolved on that list.  Small
+// problems (at most 8192 candidates) skip the sample and list every candidate.  If the list
+// comes out too short or too long (sampling bad luck, or degenerate inputs such as all-equal
+// logits), a generic 4 x 8-bit radix select over the logits in global memory takes over; it
+// orders ties by position explicitly.
 #pragma once
 #include "common.cuh"
 
@@ -20,13 +22,13 @@ constexpr int kHistBins = 1 << kHistBits;          // 2048
 constexpr int kHistShift = 32 - kHistBits;         // key >> 21
 constexpr int kSelMiscWords = 64;
 constexpr int kCandCap = 8192;                      // candidate list entries (8 bytes each)
+constexpr int kSampleStride = 16;
 
 struct SelectParams {
   const float* scores;      // [B][Hq][ld]
   int ld;
-  const float2* part_ml;    // [B][Hq][nchunks] (m, l) in the log2 domain
-  int nchunks;
-  uint32_t* hist;           // [B][Hq][kHistBins], filled by the scoring kernel; zeroed here
+  const float2* part_ml;    // [B][Hq][nchunks] (m, l) in the log2 domain; chunks past t are unset
+  int nchunks, chunk_rows;
   const int* seq_lens;
   const int* k_per_seq;     // or nullptr
   int k, sinks, window, r, m;
@@ -163,24 +165,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   const int m_eff = min(p.m < 0 ? k / 3 : p.m, kk);
   const float* g = p.scores + (long long)unit * p.ld + lo;
 
-  // histogram of the scoring pass -> shared memory; the global copy is zeroed for the next use.
-  // All loads are issued before the first store: a store followed by an L2 load in the same
-  // thread serialises on the store's acknowledgement.
-  {
-    uint32_t* gh = p.hist + (long long)unit * kHistBins;
-    uint32_t hv[kHistBins / kSelThreads];
-#pragma unroll
-    for (int x = 0; x < kHistBins / kSelThreads; ++x) hv[x] = __ldcg(gh + tid + x * kSelThreads);
-#pragma unroll
-    for (int x = 0; x < kHistBins / kSelThreads; ++x) {
-      hist[tid + x * kSelThreads] = hv[x];
-      gh[tid + x * kSelThreads] = 0u;
-    }
-  }
   // full-softmax log-sum-exp from the scoring pass' per-chunk partials
   if (warp == 1) {
     float mm = -INFINITY, ll = 0.f;
-    for (int c = lane; c < p.nchunks; c += 32) {
+    const int nch = min(p.nchunks, (t + p.chunk_rows - 1) / p.chunk_rows);
+    for (int c = lane; c < nch; c += 32) {
       const float2 x = p.part_ml[(long long)unit * p.nchunks + c];
       ml_combine(mm, ll, x.x, x.y);
     }
@@ -207,13 +196,26 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   bool fast_ok = false;
   if (kk > 0) {
     // ---------------- fast path
-    if (warp == 0) find_bin_from_top(hist, kHistBins, kk, misc);
-    __syncthreads();
-    const uint32_t d1 = misc[0];
-    const int rem1 = (int)misc[1];        // needed from bin d1
-    const int gt1 = kk - rem1;            // definite winners (bins above d1)
-    // one pass over the logits: 16 independent loads in flight per thread, then one warp scan
-    // and one pair of shared-memory atomics per warp and batch to place winners and candidates
+    // 1. conservative bin d_lo from a sample (or 0: list everything)
+    uint32_t d_lo = 0u;
+    if (n > kCandCap) {
+      for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0u;
+      __syncthreads();
+      const int ns = n / kSampleStride;
+      for (int j = tid; j < ns; j += kSelThreads) {
+        const uint32_t u = float_to_key(__ldcg(g + j * kSampleStride + (j & (kSampleStride - 1))));
+        atomicAdd(&hist[u >> kHistShift], 1u);
+      }
+      __syncthreads();
+      // want at least 1.5 k/16 + 16 sampled logits at or above d_lo (several sigma of margin)
+      const int want = min(ns, (3 * kk) / (2 * kSampleStride) + 16);
+      if (warp == 0) find_bin_from_top(hist, kHistBins, want, misc);
+      __syncthreads();
+      d_lo = misc[0];
+      __syncthreads();
+    }
+    // 2. one pass over the logits: 16 independent loads in flight per thread, then one warp
+    //    scan and one shared-memory atomic per warp and batch to place the listed entries
     const int nrounds = (n + kSelThreads - 1) / kSelThreads;
     for (int rd0 = 0; rd0 < nrounds; rd0 += 16) {
       uint32_t u16[16];
@@ -222,57 +224,47 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
         const int i = (rd0 + x) * kSelThreads + tid;
         u16[x] = i < n ? float_to_key(__ldcg(g + i)) : 0u;
       }
-      uint32_t wmask = 0u, cmask = 0u;
+      uint32_t cmask = 0u;
 #pragma unroll
       for (int x = 0; x < 16; ++x) {
         const int i = (rd0 + x) * kSelThreads + tid;
-        const uint32_t d = u16[x] >> kHistShift;
-        wmask |= (uint32_t)(i < n && d > d1) << x;
-        cmask |= (uint32_t)(i < n && d == d1) << x;
+        cmask |= (uint32_t)(i < n && (u16[x] >> kHistShift) >= d_lo) << x;
       }
-      const uint32_t mine = (uint32_t)__popc(wmask) | ((uint32_t)__popc(cmask) << 16);
+      const uint32_t mine = (uint32_t)__popc(cmask);
       uint32_t incl = mine;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         const uint32_t x = __shfl_up_sync(0xffffffffu, incl, off);
         if (lane >= off) incl += x;
       }
-      uint32_t bw = 0u, bc = 0u;
-      if (lane == 31) {
-        if (incl & 0xffffu) bw = atomicAdd(&misc[4], incl & 0xffffu);
-        if (incl >> 16) bc = atomicAdd(&misc[5], incl >> 16);
-      }
-      uint32_t ow = __shfl_sync(0xffffffffu, bw, 31) + (incl & 0xffffu) - (mine & 0xffffu);
-      uint32_t oc = __shfl_sync(0xffffffffu, bc, 31) + (incl >> 16) - (mine >> 16);
+      uint32_t bc = 0u;
+      if (lane == 31 && incl) bc = atomicAdd(&misc[5], incl);
+      uint32_t oc = __shfl_sync(0xffffffffu, bc, 31) + incl - mine;
 #pragma unroll
       for (int x = 0; x < 16; ++x) {
-        const int i = (rd0 + x) * kSelThreads + tid;
-        if ((wmask >> x) & 1u) {
-          if (ow < (uint32_t)p.sort_cap) wbuf[ow] = make_entry(u16[x], lo + i);
-          ++ow;
-        }
         if ((cmask >> x) & 1u) {
-          if (oc < (uint32_t)kCandCap) cand[oc] = make_entry(u16[x], lo + i);
+          if (oc < (uint32_t)kCandCap) cand[oc] = make_entry(u16[x], lo + (rd0 + x) * kSelThreads + tid);
           ++oc;
         }
       }
     }
     __syncthreads();
     const int ncand = (int)misc[5];
-    fast_ok = ((int)misc[4] == gt1) && ncand <= kCandCap && ncand >= rem1;
+    fast_ok = ncand >= kk && ncand <= kCandCap;
     if (fast_ok) {
-      if (rem1 == ncand) {
-        // every candidate is a winner
-        if (gt1 + ncand <= p.sort_cap) {
-          for (int i = tid; i < ncand; i += kSelThreads) wbuf[gt1 + i] = cand[i];
-          total = gt1 + ncand;
-        } else {
-          fast_ok = false;
-        }
-      } else {
-        // resolve the remaining 21 key bits on the candidate list: 3 passes of 7 bits
-        uint32_t prefix = d1 << kHistShift;
-        int rem = rem1, eq = ncand;
+      // 3. exact histogram of the list -> bin d1 of the kk-th largest key
+      for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0u;
+      __syncthreads();
+      for (int i = tid; i < ncand; i += kSelThreads)
+        atomicAdd(&hist[(uint32_t)(cand[i] >> 32) >> kHistShift], 1u);
+      __syncthreads();
+      if (warp == 0) find_bin_from_top(hist, kHistBins, kk, misc);
+      __syncthreads();
+      uint32_t prefix = misc[0] << kHistShift;
+      int rem = (int)misc[1], eq = (int)misc[2];
+      __syncthreads();
+      // 4. the remaining 21 key bits within that bin: 3 passes of 7 bits
+      if (rem < eq) {
         for (int pass = 0; pass < 3; ++pass) {
           const int shift = kHistShift - 7 * (pass + 1);
           const uint32_t mask = 0xffffffffu << (shift + 7);
@@ -288,24 +280,22 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
           prefix |= misc[0] << shift;
           rem = (int)misc[1];
           eq = (int)misc[2];
+          __syncthreads();
         }
-        const uint32_t T = prefix;            // the kk-th largest key
-        const int gt_total = kk - rem;        // keys strictly above T
-        // all keys equal to T go into the sort buffer; sorting orders them by position and
-        // the surplus falls behind the first kk entries
-        if (gt_total + eq <= p.sort_cap) {
-          const int crounds = (ncand + kSelThreads - 1) / kSelThreads;
-          for (int rd = 0; rd < crounds; ++rd) {
-            const int i = rd * kSelThreads + tid;
-            unsigned long long e = 0ull;
-            if (i < ncand) e = cand[i];
-            warp_append(i < ncand && (uint32_t)(e >> 32) >= T, e, wbuf, &misc[4], (uint32_t)p.sort_cap);
-          }
-          total = gt_total + eq;
-        } else {
-          fast_ok = false;
-        }
+      }   // else every key of bin d1 is needed: the threshold is the start of the bin
+      const uint32_t T = prefix;            // keys >= T: the winners plus the surplus ties at T
+      // 5. winners and ties into the sort buffer; sorting orders ties by position and the
+      //    surplus falls behind the first kk entries
+      const int crounds = (ncand + kSelThreads - 1) / kSelThreads;
+      for (int rd = 0; rd < crounds; ++rd) {
+        const int i = rd * kSelThreads + tid;
+        unsigned long long e = 0ull;
+        if (i < ncand) e = cand[i];
+        warp_append(i < ncand && (uint32_t)(e >> 32) >= T, e, wbuf, &misc[4], (uint32_t)p.sort_cap);
       }
+      __syncthreads();
+      total = (int)misc[4];
+      if (total > p.sort_cap || total < kk) fast_ok = false;
     }
     __syncthreads();
 

@@ -121,7 +121,7 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
     B, Hq = w.batch, w.q_heads
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=device)
     dlt = torch.empty(B, Hq, dtype=torch.float32, device=device)
-    stats = dict(max_y_err=0.0, max_delta_err=0.0, near_tie_sets=0, checked=0, deltas=[], set_sizes=[])
+    stats = dict(select_fallback=False, max_y_err=0.0, max_delta_err=0.0, near_tie_sets=0, checked=0, deltas=[], set_sizes=[])
     gq = w.q_heads // w.kv_heads
     for n in range(steps):
         t_host = W.seq_lens_at(w, n)
@@ -136,7 +136,9 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
             q = q_all[l, n].contiguous()
             ctx.decode_step(l, n, sched, q, view, B, out, dlt if want_delta else None)
             idx, cnt = ctx.get_index_set(B)
-            assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+            dev_flags = ctx.check()
+            assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+            stats["select_fallback"] = stats["select_fallback"] or bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK)
             y_gpu, d_gpu = np32(out), np32(dlt)
             retrieve = orc.is_retrieval(l, n)
             if retrieve:

@@ -136,6 +136,7 @@ def test_identical_keys_take_the_tie_path(cuda_device):
     ctx = H.make_ctx(w)
     view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
     ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), 1)
+    assert ctx.check() == P.PRHS_FLAG_SELECT_FALLBACK      # all-equal logits: the generic path ran
     s_star, n_star, s_hat, n_hat = ctx.get_shared_set(0, 1)
     for h in range(2):
         assert int(n_star[0, h]) == 100
@@ -313,6 +314,7 @@ def test_c2_full_size_sampled(cuda_device):
     units = [(0, 0), (3, 17), (7, 31), (5, 8)]
     st = H.run_schedule_parity(w, cuda_device, units)
     assert st["checked"] == 8 * len(units)
+    assert not st["select_fallback"]          # the sampled-threshold path handled every unit
 
 
 def test_c4_long_context_sampled(cuda_device):
