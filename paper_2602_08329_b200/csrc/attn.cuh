@@ -140,34 +140,6 @@ __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit
   return d;
 }
 
-// Row id (row offset / 128 elements) of list entry j for this lane, or kBadRow.
-__device__ __forceinline__ uint32_t fetch_row_id(const AttnParams& p, const ListDesc& d, int j, int end,
-                                                 int t, int b, int kvh, uint32_t outer_rows,
-                                                 uint32_t head_rows) {
-  if (j >= end) return kBadRow;
-  int pos;
-  if (d.fused) {
-    if (j < d.s0) pos = j;
-    else if (j < d.s0 + d.nmid) pos = __ldg(d.list + d.lo + (j - d.s0));
-    else pos = d.wlo + (j - d.s0 - d.nmid);
-  } else {
-    pos = d.list ? __ldg(d.list + j) : j;
-  }
-  if ((unsigned)pos >= (unsigned)t) {
-    atomicOr(p.flags, kFlagBadIndex);
-    return kBadRow;
-  }
-  if (p.kv.page_table != nullptr) {
-    const int page = __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
-    if ((unsigned)page >= (unsigned)p.kv.num_pages) {
-      atomicOr(p.flags, kFlagBadPage);
-      return kBadRow;
-    }
-    return (uint32_t)page * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)(pos & 15);
-  }
-  return (uint32_t)b * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)pos;
-}
-
 // ------------------------------------------- gathered attention, tensor-core pipeline (sm_100a)
 // The same warp-private cp.async pipeline, with the arithmetic moved to mma.sync m16n8k16
 // (bf16 in, fp32 accumulate) so that a gathered row costs about a dozen warp instructions
@@ -244,18 +216,64 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   float z0 = 0.f, z1 = 0.f;            // accumulator rows 8..15: always zero
   float m = -INFINITY, l = 0.f;
 
-  uint32_t rid_a = fetch_row_id(p, ld, start + lane, end, t, b, kvh, outer_rows, head_rows);
-  uint32_t rid_b = fetch_row_id(p, ld, start + 32 + lane, end, t, b, kvh, outer_rows, head_rows);
+  // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane.  Each level is
+  // produced one step before it is consumed, so that no load is waited for where it is issued:
+  //   pos2 : raw list entry of group G+2 (a load from the list, unchecked)
+  //   pos1 / pg1 : checked position of group G+1 and, for a paged cache, its raw page id (a load)
+  //   rid_a : final row id of group G, the one being issued
+  auto list_pos = [&](int grp) -> int {
+    const int j = start + grp * 32 + lane;
+    if (j >= end) return -1;
+    if (ld.fused) {
+      if (j < ld.s0) return j;
+      if (j < ld.s0 + ld.nmid) return __ldg(ld.list + ld.lo + (j - ld.s0));
+      return ld.wlo + (j - ld.s0 - ld.nmid);
+    }
+    return ld.list ? __ldg(ld.list + j) : j;
+  };
+  auto check_pos = [&](int pos, int grp) -> int {      // consumes the list load
+    if (start + grp * 32 + lane >= end) return -1;
+    if ((unsigned)pos >= (unsigned)t) {
+      atomicOr(p.flags, kFlagBadIndex);
+      return -1;
+    }
+    return pos;
+  };
+  const bool paged = p.kv.page_table != nullptr;
+  auto page_of = [&](int pos) -> int {                 // issues the page-table load
+    if (!paged || pos < 0) return 0;
+    return __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
+  };
+  auto row_id = [&](int pos, int page) -> uint32_t {   // consumes the page-table load
+    if (pos < 0) return kBadRow;
+    if (paged) {
+      if ((unsigned)page >= (unsigned)p.kv.num_pages) {
+        atomicOr(p.flags, kFlagBadPage);
+        return kBadRow;
+      }
+      return (uint32_t)page * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)(pos & 15);
+    }
+    return (uint32_t)b * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)pos;
+  };
+  int pos1 = check_pos(list_pos(0), 0);
+  int pg1 = page_of(pos1);
+  uint32_t rid_a = row_id(pos1, pg1);
+  pos1 = check_pos(list_pos(1), 1);
+  pg1 = page_of(pos1);
+  int pos2 = list_pos(2);
+
   const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
   const uint32_t dst_tile = (lane < 16 ? 0u : (uint32_t)kTTileBytes);
   unsigned long long vmask = 0ull;     // 16 validity bits per ring slot
 
   auto issue = [&](int j) {
     if (j < nstages) {
-      if (j > 0 && (j & 1) == 0) {
-        rid_a = rid_b;
-        rid_b = fetch_row_id(p, ld, start + (j + 2) * kTStageRows + lane, end, t, b, kvh, outer_rows,
-                             head_rows);
+      if (j > 0 && (j & 1) == 0) {     // step the row-id pipeline
+        const int grp = j >> 1;
+        rid_a = row_id(pos1, pg1);
+        pos1 = check_pos(pos2, grp + 1);
+        pg1 = page_of(pos1);
+        pos2 = list_pos(grp + 2);
       }
       const int slot_i = j % kTStages;
       const uint32_t slot = ring + (uint32_t)slot_i * kTStageBytes + dst_tile;
@@ -279,6 +297,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   const float sc = kScale * kLog2e;
   // ldmatrix lane roles
   const int lm_mi = lane >> 3, lm_r = lane & 7;
+  const int vrow = (lm_mi & 1) * 8 + lm_r;
   for (int i = 0; i < nstages; ++i) {
     cp_async_wait<kTStages - 2>();
     __syncwarp();
@@ -287,50 +306,66 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
     issue(i + kTStages - 1);
     const uint32_t kt = ring + (uint32_t)slot_i * kTStageBytes;
     const uint32_t vt = kt + kTTileBytes;
-    // ---- S = Q K^T
-    float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    // ---- S = Q K^T : all K fragments first, then the two accumulator chains interleaved
+    uint32_t bk[2][4][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
       const int row = nt * 8 + lm_r;
 #pragma unroll
-      for (int pp = 0; pp < 4; ++pp) {
-        uint32_t bk[4];
-        ldmatrix_x4(bk, kt + row * kRowBytes + (((4 * pp + lm_mi) ^ (row & 7)) << 4));
-        mma_bf16_row0(s[nt][0], s[nt][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[0], bk[1]);
-        mma_bf16_row0(s[nt][0], s[nt][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[2], bk[3]);
-      }
+      for (int pp = 0; pp < 4; ++pp)
+        ldmatrix_x4(bk[nt][pp], kt + row * kRowBytes + (((4 * pp + lm_mi) ^ (row & 7)) << 4));
     }
-    // ---- online softmax on the 16 logits held by lanes 0-3
-    float s0 = s[0][0] * sc, s1 = s[0][1] * sc, s2 = s[1][0] * sc, s3 = s[1][1] * sc;
-    if (!((vm >> (2 * tg)) & 1u)) s0 = -INFINITY;
-    if (!((vm >> (2 * tg + 1)) & 1u)) s1 = -INFINITY;
-    if (!((vm >> (8 + 2 * tg)) & 1u)) s2 = -INFINITY;
-    if (!((vm >> (9 + 2 * tg)) & 1u)) s3 = -INFINITY;
+    float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+    for (int pp = 0; pp < 4; ++pp) {
+      mma_bf16_row0(s[0][0], s[0][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[0][pp][0], bk[0][pp][1]);
+      mma_bf16_row0(s[1][0], s[1][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[1][pp][0], bk[1][pp][1]);
+      mma_bf16_row0(s[0][0], s[0][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[0][pp][2], bk[0][pp][3]);
+      mma_bf16_row0(s[1][0], s[1][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[1][pp][2], bk[1][pp][3]);
+    }
+    // the first half of the V fragments, fetched under the softmax arithmetic
+    uint32_t bv[4][4];
+#pragma unroll
+    for (int np = 0; np < 4; ++np)
+      ldmatrix_x4_trans(bv[np], vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
+    // ---- online softmax on the 16 logits held by lanes 0-3.  The reference exponent m only
+    // moves when a logit exceeds it by more than 8 (weights stay below 2^8): the common
+    // stage costs one warp vote instead of a cross-lane maximum.
+    float s0 = -INFINITY, s1 = -INFINITY, s2 = -INFINITY, s3 = -INFINITY;
+    if (g == 0) {
+      if ((vm >> (2 * tg)) & 1u) s0 = s[0][0] * sc;
+      if ((vm >> (2 * tg + 1)) & 1u) s1 = s[0][1] * sc;
+      if ((vm >> (8 + 2 * tg)) & 1u) s2 = s[1][0] * sc;
+      if ((vm >> (9 + 2 * tg)) & 1u) s3 = s[1][1] * sc;
+    }
     float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-    const float mn = fmaxf(m, __shfl_sync(0xffffffffu, mx, 0));
-    if (mn != -INFINITY) {             // warp-uniform
-      const float corr = exp2f(m - mn);
+    if (__any_sync(0xffffffffu, mx > m + 8.f)) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float mn = fmaxf(m, __shfl_sync(0xffffffffu, mx, 0));
+      const float corr = exp2f(m - mn);     // m = -inf on the first real stage: corr = 0
       m = mn;
-      float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
-      if (g == 0) {
-        p0 = exp2f(s0 - mn); p1 = exp2f(s1 - mn); p2 = exp2f(s2 - mn); p3 = exp2f(s3 - mn);
-      }
-      l = l * corr + ((p0 + p1) + (p2 + p3));
+      l *= corr;
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+    }
+    if (m != -INFINITY) {              // warp-uniform; false only while every row so far was invalid
+      const float p0 = exp2f(s0 - m), p1 = exp2f(s1 - m), p2 = exp2f(s2 - m), p3 = exp2f(s3 - m);
+      l += (p0 + p1) + (p2 + p3);
       const uint32_t ap0 = pack_bf16x2(p0, p1), ap2 = pack_bf16x2(p2, p3);
-      if (corr != 1.f) {
-#pragma unroll
-        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
-      }
       // ---- O += P V
-      const int vrow = (lm_mi & 1) * 8 + lm_r;
 #pragma unroll
-      for (int np = 0; np < 8; ++np) {
-        uint32_t bv[4];
-        ldmatrix_x4_trans(bv, vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
-        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[0], bv[1]);
-        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[2], bv[3]);
+      for (int np = 0; np < 4; ++np) {
+        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[np][0], bv[np][1]);
+        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[np][2], bv[np][3]);
+      }
+#pragma unroll
+      for (int np = 4; np < 8; ++np)
+        ldmatrix_x4_trans(bv[np - 4], vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
+#pragma unroll
+      for (int np = 4; np < 8; ++np) {
+        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[np - 4][0], bv[np - 4][1]);
+        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[np - 4][2], bv[np - 4][3]);
       }
     }
   }
