@@ -7,7 +7,9 @@
 A step is one pass of the whole hot path over one batch: one decode step of one layer
 (retrieval on the first step of every block of `refresh` steps, then index-set build and
 gathered attention).  The workload is the LLaMA-2-7B-shaped single layer at 32K context
-(batch 8, 32 MHA heads, k = 1024, window 128, 4 sinks, refresh every 4 steps), synthetic.
+(batch 8, 32 MHA heads, k = 1024, window 128, 4 sinks, refresh every 4 steps), synthetic;
+four independent copies of that layer's cache are visited round-robin so that no step finds
+its rows in L2.
 
 Prints ONE JSON line.  `value` is attention-only decode throughput in tokens/s (batch tokens
 per step / device time per step) with every input resident in HBM; `e2e` is the same metric
@@ -152,7 +154,7 @@ def workload_config(w: W.Workload, extra=None):
     cfg = {"workload": w.name, "layers": 1, "batch": w.batch, "q_heads": w.q_heads, "kv_heads": w.kv_heads,
            "head_dim": 128, "context": w.context, "top_k": w.top_k, "window": w.window, "sinks": w.sinks,
            "refresh_interval": w.refresh, "dilate_r": w.dilate_r, "dilate_m": "k/3",
-           "l2": "flushed between steps (256 MiB write outside the timed events); cache 4.3 GB >> L2"}
+           "l2": "no flush: inputs larger than L2 (each cache copy is 4.3 GB)"}
     cfg.update(extra or {})
     return cfg
 
@@ -194,39 +196,60 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     Wn, Kn = args.warmup, args.steps
-    total_steps = Wn + Kn
-    w = W.C2_LLAMA2_7B.scaled(steps=total_steps, seed=W.C2_LLAMA2_7B.seed + 97 * rank)
+    # Step i of the run is decode step i // L of cache i % L: L independent copies of the
+    # single-layer workload are visited round-robin, so every step finds its K/V rows cold in
+    # L2 (each copy is 4.3 GB) without a flush kernel between steps, and launches stay
+    # back to back as in a real decode loop.  L = 1 falls back to flushing L2 between steps.
+    L = max(1, args.rotate)
+    n_dec = (Wn + Kn + L - 1) // L
+    w = W.C2_LLAMA2_7B.scaled(steps=n_dec, layers=L, seed=W.C2_LLAMA2_7B.seed + 97 * rank)
     if args.batch:
         w = w.scaled(batch=args.batch)      # smaller case for profiler captures only
-    k, v = W.make_kv(w, dev)
-    q_all = W.make_queries(w, dev)[0]                     # [steps][B][Hq][128]
+    kv_layers = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
+    q_all = W.make_queries(w, dev)                        # [L][n_dec][B][Hq][128]
     B, Hq, Hkv = w.batch, w.q_heads, w.kv_heads
-    ctx = P.Context(1, B, Hq, Hkv, w.capacity, w.top_k, w.window, w.sinks, max_dilate_r=w.dilate_r)
+    ctx = P.Context(L, B, Hq, Hkv, w.capacity, w.top_k, w.window, w.sinks, max_dilate_r=w.dilate_r)
     sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r)
-    t_all = torch.stack([W.seq_lens_at(w, n) for n in range(total_steps)]).to(dev)   # [steps][B]
-    views = [P.make_view(k, v, t_all[n], max_seq_len=w.capacity) for n in range(total_steps)]
+    t_all = torch.stack([W.seq_lens_at(w, n) for n in range(n_dec)]).to(dev)        # [n_dec][B]
+    views = [[P.make_view(kv_layers[l][0], kv_layers[l][1], t_all[n], max_seq_len=w.capacity)
+              for n in range(n_dec)] for l in range(L)]
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev) if L == 1 else None
     stream = torch.cuda.current_stream()
 
-    def timed_steps(first, count, fn):
-        """Run `count` steps; per-step CUDA events on the launching stream; L2 flushed between."""
+    def timed_steps(first, count, fn, per_step=False):
+        """Run `count` steps and return their device times in ms (CUDA events on the launching
+        stream).  With cache rotation the region is bracketed once (or per step when asked);
+        with a single cache L2 is flushed before every step, outside the per-step events."""
+        if L > 1 and not per_step:
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(count):
+                fn(first + i)
+            b_.record(stream)
+            torch.cuda.synchronize()
+            return [a.elapsed_time(b_) / max(count, 1)] * count
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                for _ in range(count)]
         for i in range(count):
-            flush.zero_()
+            if flush is not None:
+                flush.zero_()
             evs[i][0].record(stream)
             fn(first + i)
             evs[i][1].record(stream)
         torch.cuda.synchronize()
-        return [a.elapsed_time(b) for a, b in evs]
+        return [a.elapsed_time(b_) for a, b_ in evs]
 
-    def step_device(n):
-        ctx.decode_step(0, n, sched, q_all[n], views[n], B, out)
+    def step_device(i):
+        l, n = i % L, i // L
+        ctx.decode_step(l, n, sched, q_all[l, n], views[l][n], B, out)
+
+    def is_refresh(i):
+        return (i // L) % w.refresh == 0
 
     # ---- warm-up, then the timed region
     timed_steps(0, Wn, step_device)
-    sampler = ClockSampler(local, uuid=str(torch.cuda.get_device_properties(dev).uuid))
+    sampler = ClockSampler(local, uuid=str(torch.cuda.get_device_properties(dev).uuid), period=0.002)
     sampler.start()
     launches0 = ctx.launch_count
     barrier()
@@ -235,24 +258,33 @@ def run_cuda(args):
     prof = ctx.profile_end()
     barrier()
     launches = ctx.launch_count - launches0
-    clocks = sampler.stop()
     dev_flags = ctx.check()
     assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
     total_ms = sum(ms)
     total_ms_max = reduce_max_ms(total_ms, dist, dev)
     value = job_throughput(world, B, Kn, total_ms_max)
 
-    refresh_ms = [m for i, m in enumerate(ms) if (Wn + i) % w.refresh == 0]
-    shared_ms = [m for i, m in enumerate(ms) if (Wn + i) % w.refresh != 0]
+    def rewind():
+        """Replay the warm-up steps so that the shared-set state is the one step Wn expects."""
+        for i in range(Wn):
+            step_device(i)
+
+    # per-step times of the same steps (event pair per step), to tell retrieval from sharing steps
+    rewind()
+    ms_each = timed_steps(Wn, Kn, step_device, per_step=True)
+
+    refresh_ms = [m for i, m in enumerate(ms_each) if is_refresh(Wn + i)]
+    shared_ms = [m for i, m in enumerate(ms_each) if not is_refresh(Wn + i)]
 
     # ---- algorithmic bytes: K once on retrieval steps, gathered K/V rows on every step
     counts = []
-    for n in range(Wn, Wn + Kn):                          # untimed replay to read the set sizes
-        step_device(n)
+    rewind()
+    for i in range(Wn, Wn + Kn):                          # untimed replay to read the set sizes
+        step_device(i)
         _, cnt = ctx.get_index_set(B)
         counts.append(int(cnt.sum()))
     t_cpu = t_all.cpu()
-    score_bytes = [int(t_cpu[n].sum()) * Hkv * 256 for n in range(Wn, Wn + Kn) if n % w.refresh == 0]
+    score_bytes = [int(t_cpu[i // L].sum()) * Hkv * 256 for i in range(Wn, Wn + Kn) if is_refresh(i)]
     gather_bytes = [c * 512 for c in counts]
     hbm_peak, peak_kind = load_peaks()
     kernels = {}
@@ -283,33 +315,40 @@ def run_cuda(args):
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "kernels": kernels,
                               "select_fallback": bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK),
                               "config": workload_config(w), "note": "path only (profiling run)"}))
+        sampler.stop()
         ctx.close()
         return 0
 
     # ---- in-library dense flash-decode baseline, same protocol
     nd = min(4, Kn)
-    dense_ms = timed_steps(Wn, nd, lambda n: ctx.dense_decode_attn(q_all[n], views[n], B, out))
+    dense_ms = timed_steps(Wn, nd, lambda i: ctx.dense_decode_attn(q_all[i % L, i // L], views[i % L][i // L],
+                                                                 B, out))
     dense_us = 1e3 * statistics.median(dense_ms[1:] or dense_ms)
-    dense_bytes = int(t_cpu[Wn + nd - 1].sum()) * Hkv * 512
+    dense_bytes = int(t_cpu[(Wn + nd - 1) // L].sum()) * Hkv * 512
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     bi = torch.arange(B)
     host = []
-    for n in range(Wn, Wn + Kn):
+    for i in range(Wn, Wn + Kn):
+        l, n = i % L, i // L
         pos = (t_cpu[n] - 1).long()
-        host.append((q_all[n].cpu().pin_memory(), k[bi, :, pos].cpu().contiguous().pin_memory(),
+        k, v = kv_layers[l]
+        host.append((q_all[l, n].cpu().pin_memory(), k[bi, :, pos].cpu().contiguous().pin_memory(),
                      v[bi, :, pos].cpu().contiguous().pin_memory(), t_cpu[n].contiguous().pin_memory()))
     host_out = torch.empty(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
     t_scratch = torch.zeros(B, dtype=torch.int32, device=dev)
-    view_h = P.make_view(k, v, t_scratch, max_seq_len=w.capacity)
+    views_h = [P.make_view(kv_layers[l][0], kv_layers[l][1], t_scratch, max_seq_len=w.capacity)
+               for l in range(L)]
 
-    def step_host(n):
-        hq, hk, hv, ht = host[n - Wn]
-        ctx.decode_step_host(0, n, sched, hq, hk, hv, ht, view_h, B, host_out)
+    def step_host(i):
+        hq, hk, hv, ht = host[i - Wn]
+        ctx.decode_step_host(i % L, i // L, sched, hq, hk, hv, ht, views_h[i % L], B, host_out)
 
+    rewind()
     barrier()
     e2e_ms = timed_steps(Wn, Kn, step_host)
     barrier()
+    clocks = sampler.stop()
     e2e_max_ms = reduce_max_ms(sum(e2e_ms), dist, dev)
     e2e_value = job_throughput(world, B, Kn, e2e_max_ms)
     h2d = B * Hq * 256 + 2 * B * Hkv * 256 + B * 4
@@ -332,7 +371,12 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": Kn, "warmup": Wn,
         "ms_per_step": total_ms_max / Kn, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
-        "config": workload_config(w, {"parallelism": f"replicas x{world} (no collective)"}),
+        "config": workload_config(w, {
+            "parallelism": f"replicas x{world} (no collective)",
+            "cache_copies": L,
+            "l2": (f"no flush: {L} independent copies of the layer's cache (4.3 GB each) visited round-robin, "
+                   "so every step's K/V rows are cold in L2; steps are launched back to back"
+                   if L > 1 else "flushed between steps (256 MiB write outside the per-step events)")}),
         "us_per_layer_step": 1e3 * total_ms_max / Kn,
         "refresh_step_us": 1e3 * statistics.median(refresh_ms) if refresh_ms else None,
         "shared_step_us": 1e3 * statistics.median(shared_ms) if shared_ms else None,
@@ -365,6 +409,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling captures)")
+    ap.add_argument("--rotate", type=int, default=4,
+                    help="independent copies of the layer cache visited round-robin (1 = flush L2 instead)")
     ap.add_argument("--path-only", action="store_true", help="skip the dense, e2e and CPU legs")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
