@@ -37,8 +37,8 @@ METRIC = "sparse_decode_attn_tokens_per_s_32k_ctx"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch (read + write) of the kernels, from the ncu captures summarised under
-# profiles/ (scaled to a full launch by the units processed); None until captured.
-NCU_TRAFFIC_BYTES = {"score": None, "attn_sparse": None}
+# profiles/ (captured at batch 2-4 and scaled to the full batch by the units processed).
+NCU_TRAFFIC_BYTES = {"score": 2.164e9, "attn_sparse": 2.39e8}
 
 
 def load_peaks():
