@@ -31,7 +31,7 @@ import numpy as np
 __all__ = [
     "dense_scores", "rank_logits", "softmax_full", "logsumexp", "dense_attention",
     "topk_middle", "dilate", "build_set", "attn_over_set", "retained_mass",
-    "dropped_mass", "delta_from_lse", "mi_bound_g", "coverage", "bf16_round",
+    "dropped_mass", "delta_from_lse", "mi_bound_g", "coverage", "bf16_round", "psaw_start",
     "Schedule", "PrhsOracle",
 ]
 
@@ -84,15 +84,32 @@ def dense_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, t: int):
 
 
 # ------------------------------------------------- Sec. 4.1: top-k over the middle range
-def topk_middle(a: np.ndarray, t: int, sinks: int, window: int, k: int) -> np.ndarray:
+def psaw_start(layer: int, num_layers: int, t: int, phi: float, alpha: float, layer_start: int) -> int:
+    """P_l(t) of the progressive sliding attention window (Eq. 11).
+
+    `layer` is 0-based; the paper's l is layer + 1 and runs to N = num_layers.  `layer_start`
+    is the paper's l_s (1-based; Sec. 5.1 default floor(3N/4)); 0 switches the window off.
+    P = 0 for l < l_s, else floor((1 - phi^(alpha (l - l_s) / (N - l_s))) t).  The result is
+    used as a 0-based position: positions [S0, P) are masked, [0, S0) and [P, t) stay visible.
+    """
+    ell = layer + 1
+    if layer_start <= 0 or ell < layer_start or num_layers <= layer_start:
+        return 0
+    expo = alpha * (ell - layer_start) / (num_layers - layer_start)
+    return int(math.floor((1.0 - phi ** expo) * t))
+
+
+def topk_middle(a: np.ndarray, t: int, sinks: int, window: int, k: int, psaw_lo: int = 0) -> np.ndarray:
     """S* = the k positions of largest logit among the middle candidates [S0, t-W).
+
+    With a sliding-window start `psaw_lo` (Eq. 11) the candidates are [max(S0, P), t-W).
 
     Returned in descending-logit order p_1, p_2, ... (Sec. 4.1: "sorted and selected in
     descending order of attention weight"); equal logits are ordered by lower position
     first.  Softmax is monotone in the logit, so ranking logits ranks attention weights.
     The ranking uses the float32-rounded logits (see module docstring).
     """
-    lo, hi = sinks, t - window
+    lo, hi = max(sinks, psaw_lo), t - window
     if hi <= lo or k <= 0:
         return np.zeros(0, dtype=np.int64)
     cand = np.arange(lo, hi, dtype=np.int64)
@@ -119,16 +136,18 @@ def dilate(s_star: np.ndarray, m: int, r: int, t_anchor: int) -> np.ndarray:
 
 
 # ---------------------------------------------------------------- Sec. 4.1: critical set
-def build_set(t: int, sinks: int, window: int, middle: np.ndarray) -> np.ndarray:
+def build_set(t: int, sinks: int, window: int, middle: np.ndarray, psaw_lo: int = 0) -> np.ndarray:
     """C = [0, S0) ∪ M ∪ [t-W, t) at the CURRENT length t; sorted, unique (Sec. 4.1).
 
     On a sharing step M is the anchor's (dilated) middle set (Def. 3.2); the sink and
-    local groups are positional and follow the current t.
+    local groups are positional and follow the current t.  With a sliding-window start
+    `psaw_lo` = P_l(t) (Sec. 4.2) only the visible positions [0, S0) ∪ [P, t) are kept.
     """
     out = set(range(0, min(sinks, t)))
     out.update(int(x) for x in middle if 0 <= int(x) < t)
     out.update(range(max(0, t - window), t))
-    return np.array(sorted(out), dtype=np.int64)
+    s0 = min(sinks, t)
+    return np.array(sorted(x for x in out if x < s0 or x >= psaw_lo), dtype=np.int64)
 
 
 # ------------------------------------------------------ Def. 3.1: token-sparse attention
@@ -197,12 +216,19 @@ class Schedule:
     dilate_m: int = -1             # -1 -> floor(k/3)
     dilate_anchor: bool = False    # True: the anchor's own attention also uses S^
     top_k_per_seq: np.ndarray | None = None
+    psaw_phi: float = 0.7          # Eq. 11 (defaults Sec. 5.1)
+    psaw_alpha: float = 1.0
+    psaw_layer_start: int = 0      # l_s, 1-based; 0 = no sliding window
+    num_layers: int = 1            # N of Eq. 11
 
     def k_for(self, b: int) -> int:
         return int(self.top_k_per_seq[b]) if self.top_k_per_seq is not None else self.top_k
 
     def m_for(self, b: int) -> int:
         return self.k_for(b) // 3 if self.dilate_m < 0 else self.dilate_m
+
+    def psaw_for(self, layer: int, t: int) -> int:
+        return psaw_start(layer, self.num_layers, t, self.psaw_phi, self.psaw_alpha, self.psaw_layer_start)
 
 
 @dataclass
@@ -240,7 +266,7 @@ class PrhsOracle:
             raise RuntimeError("group leader has not retrieved for this block")
         own = self.is_retrieval(layer, step) and not self.s.dilate_anchor
         M = sh.s_star[(b, h)] if own else sh.s_hat[(b, h)]
-        return build_set(t, self.s.sinks, self.s.window, M)
+        return build_set(t, self.s.sinks, self.s.window, M, self.s.psaw_for(layer, t))
 
     def decode_step(self, layer, step, q, K, V, seq_lens, units=None, want_delta=True):
         """q [B][Hq][d]; K, V [B][Hkv][cap][d]; seq_lens [B].
@@ -266,7 +292,8 @@ class PrhsOracle:
             a = None
             if retrieve:
                 a = dense_scores(q[b, h], K[b, kv], t)
-                s_star = topk_middle(a, t, self.s.sinks, self.s.window, self.s.k_for(b))
+                s_star = topk_middle(a, t, self.s.sinks, self.s.window, self.s.k_for(b),
+                                     self.s.psaw_for(layer, t))
                 sh = self.groups[g]
                 sh.s_star[(b, h)] = s_star
                 sh.s_hat[(b, h)] = dilate(s_star, self.s.m_for(b), self.s.dilate_r, t)

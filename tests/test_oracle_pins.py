@@ -184,6 +184,7 @@ def test_paper_defaults_fixture():
     s = O.Schedule(top_k=432, window=64, sinks=16)
     assert s.dilate_r == int(kv["dilate_r"])
     assert s.m_for(0) == 432 // int(kv["dilate_m_divisor"]) == 144
+    assert s.psaw_phi == float(kv["psaw_phi"]) and s.psaw_alpha == float(kv["psaw_alpha"])
 
 
 def test_build_set_union_and_bounds():
@@ -345,6 +346,58 @@ def test_dilated_set_covers_next_topk_on_clustered_keys():
     s_hat = O.dilate(s1, n_c, 1, t)
     assert O.coverage(s_hat, s2) == 1.0
     assert O.coverage(np.sort(s1), s2) == 0.0
+
+
+# ------------------------------------------------------- sliding attention window, Eq. 11
+def test_psaw_window_start_worked_values():
+    with open(os.path.join(GOLDEN, "psaw_window_start.txt")) as f:
+        rows = [l.split("#")[0].split() for l in f if l.split("#")[0].strip()]
+    assert len(rows) >= 9
+    for phi, alpha, ell, t, want in rows:
+        got = O.psaw_start(int(ell) - 1, 32, int(t), float(phi), float(alpha), 24)
+        assert got == int(want), (phi, alpha, ell, t)
+    # off switch, monotone in depth, never reaches t, alpha = 0 prunes nothing
+    assert O.psaw_start(31, 32, 32768, 0.7, 1.0, 0) == 0
+    ps = [O.psaw_start(l, 32, 50000, 0.7, 1.0, 24) for l in range(32)]
+    assert ps[:24] == [0] * 24 and all(a <= b for a, b in zip(ps, ps[1:])) and ps[-1] < 50000
+    assert all(O.psaw_start(l, 32, 50000, 0.7, 0.0, 24) == 0 for l in range(32))
+
+
+def test_psaw_clips_retrieval_range_and_set():
+    g = rng(30)
+    t, S0, W, k, P = 400, 4, 16, 24, 150
+    a = g.standard_normal(t)
+    s_star = O.topk_middle(a, t, S0, W, k, psaw_lo=P)
+    # brute force on the clipped range
+    cand = np.arange(P, t - W)
+    want = cand[np.argsort(-a[P:t - W], kind="stable")[:k]]
+    assert np.array_equal(s_star, want) and s_star.min() >= P
+    # the set keeps sinks, drops everything else below P
+    M = O.dilate(O.topk_middle(a, t, S0, W, k), k // 3, 1, t)       # an unclipped shared set
+    C0, C1 = O.build_set(t, S0, W, M), O.build_set(t, S0, W, M, psaw_lo=P)
+    assert set(C1) == {x for x in C0 if x < S0 or x >= P}
+    assert O.dropped_mass(a, C1) >= O.dropped_mass(a, C0) - 1e-15      # a subset retains less
+    # a window start beyond t - W clips the local window too, sinks always stay
+    C2 = O.build_set(t, S0, W, M, psaw_lo=t - 5)
+    assert np.array_equal(C2, list(range(S0)) + list(range(t - 5, t)))
+    assert np.array_equal(O.build_set(t, S0, W, M, psaw_lo=0), C0)
+
+
+def test_schedule_with_psaw_layers():
+    q, K, V = _stack(24, layers=4)
+    s = O.Schedule(top_k=16, window=8, sinks=2, refresh_interval=2, layer_group=2, psaw_phi=0.5,
+                   psaw_alpha=1.0, psaw_layer_start=2, num_layers=4)
+    orc = O.PrhsOracle(s, 4, 2)
+    for n in range(2):
+        t = np.array([210 + n + 1, 190 + n + 1])
+        for l in range(4):
+            out = orc.decode_step(l, n, q[l, n], K[l], V[l], t)
+            for (b, h), C in out["set"].items():
+                P = O.psaw_start(l, 4, int(t[b]), 0.5, 1.0, 2)
+                assert P == (0 if l < 2 else int((1 - 0.5 ** ((l - 1) / 2)) * int(t[b])))
+                assert all(x < 2 or x >= P for x in C)
+                if l == 3:
+                    assert P == int(t[b]) // 2 and C[2] >= P
 
 
 # ------------------------------------------------------------------------- MI bound, Eq. 4
