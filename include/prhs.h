@@ -103,6 +103,13 @@ typedef struct {
   int32_t dilate_r;             /* r of Eq. 10 */
   int32_t dilate_m;             /* m of Eq. 10; -1 = floor(k / 3) per sequence                  */
   uint32_t flags;
+  /* Progressive sliding attention window in decode (Sec. 4.2, Eq. 11): for the paper's layer
+   * number l = layer + 1 >= l_s, positions [S0, P) with P = floor((1 - phi^(alpha (l - l_s) /
+   * (N - l_s))) t_b) are masked: they are neither retrieval candidates nor attended (sinks
+   * stay).  N = prhs_config.num_layers.  psaw_layer_start = l_s (1-based); 0 = off. */
+  float psaw_phi;               /* phi in (0, 1); default 0.7 (Sec. 5.1)                        */
+  float psaw_alpha;             /* alpha >= 0; default 1                                        */
+  int32_t psaw_layer_start;     /* l_s; default floor(3 N / 4); 0 disables the window           */
 } prhs_schedule;
 
 /* Create / destroy a context on the current CUDA device.  prhs_create allocates every

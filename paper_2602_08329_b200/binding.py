@@ -56,7 +56,8 @@ class KvView(C.Structure):
 class Schedule(C.Structure):
     _fields_ = [("refresh_interval", C.c_int32), ("layer_group", C.c_int32), ("top_k", C.c_int32),
                 ("top_k_per_seq", C.c_void_p), ("window", C.c_int32), ("sinks", C.c_int32),
-                ("dilate_r", C.c_int32), ("dilate_m", C.c_int32), ("flags", C.c_uint32)]
+                ("dilate_r", C.c_int32), ("dilate_m", C.c_int32), ("flags", C.c_uint32),
+                ("psaw_phi", C.c_float), ("psaw_alpha", C.c_float), ("psaw_layer_start", C.c_int32)]
 
 
 _lib = None
@@ -119,9 +120,9 @@ def _stream(stream=None):
 
 
 def make_schedule(top_k, window, sinks, refresh_interval=1, layer_group=1, dilate_r=1, dilate_m=-1,
-                  top_k_per_seq=None, flags=0) -> Schedule:
+                  top_k_per_seq=None, flags=0, psaw_phi=0.7, psaw_alpha=1.0, psaw_layer_start=0) -> Schedule:
     s = Schedule(refresh_interval, layer_group, top_k, _ptr(top_k_per_seq), window, sinks,
-                 dilate_r, dilate_m, flags)
+                 dilate_r, dilate_m, flags, psaw_phi, psaw_alpha, psaw_layer_start)
     s._keep = top_k_per_seq
     return s
 

@@ -11,7 +11,7 @@ namespace prhs {
 // One CTA per (sequence, query head).
 __global__ void __launch_bounds__(128)
 build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int mid_stride,
-                 const int* __restrict__ seq_lens, int sinks, int window, int num_q_heads,
+                 const int* __restrict__ seq_lens, int sinks, int window, double psaw_c, int num_q_heads,
                  int* __restrict__ out_idx, int idx_stride, int* __restrict__ out_count) {
   const int unit = blockIdx.x;
   const int b = unit / num_q_heads;
@@ -19,7 +19,8 @@ build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int
   const int* M = mid + (long long)unit * mid_stride;
   const int nm = __ldg(n_mid + unit);
   const int s0 = min(sinks, t);
-  const int wlo = max(max(t - window, 0), s0);
+  const int vis_lo = max(s0, psaw_start(psaw_c, t));      // first visible non-sink position
+  const int wlo = max(max(t - window, 0), vis_lo);
   // M is ascending: the number of entries below a bound is the position of the bound.  Count
   // in parallel (one coalesced pass) instead of a binary search of dependent cold loads.
   __shared__ int sh_lo, sh_hi;
@@ -28,7 +29,7 @@ build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int
   int c0 = 0, c1 = 0;
   for (int i = threadIdx.x; i < nm; i += blockDim.x) {
     const int x = __ldg(M + i);
-    c0 += x < s0;
+    c0 += x < vis_lo;
     c1 += x < wlo;
   }
 #pragma unroll
@@ -66,6 +67,7 @@ struct AttnParams {
   const int* mid;
   const int* n_mid;
   int mid_stride, sinks, window;
+  double psaw_c;            // sliding-window factor of this layer (0 = off), fused mode only
   // idx == nullptr and mid == nullptr: all positions [0, t) (dense baseline)
   int num_q_heads, group_size;
   int splits;
@@ -99,8 +101,9 @@ struct ListDesc {
 };
 
 // Per-warp set-up of the list descriptor (all 32 lanes call it).  In fused mode the bounds of
-// M inside [s0, wlo) are found by looking at its two ends: dilation can push at most r
-// entries below S0 or into the window; a longer overlap falls back to a full scan.
+// M inside [vis_lo, wlo) are found by looking at its two ends: dilation can push at most r
+// entries below S0 or into the window; a longer overlap (a sliding window start that moved
+// past many entries, a schedule change inside a block) falls back to a full scan.
 __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit, int t) {
   ListDesc d;
   const int lane = threadIdx.x & 31;
@@ -112,15 +115,16 @@ __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit
     const int* M = p.mid + (long long)unit * p.mid_stride;
     const int nm = min(__ldg(p.n_mid + unit), p.mid_stride);
     const int s0 = min(p.sinks, t);
-    const int wlo = max(max(t - p.window, 0), s0);
-    int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && __ldg(M + min(lane, max(nm - 1, 0))) < s0));
+    const int vis_lo = max(s0, psaw_start(p.psaw_c, t));
+    const int wlo = max(max(t - p.window, 0), vis_lo);
+    int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && __ldg(M + min(lane, max(nm - 1, 0))) < vis_lo));
     const int i1 = nm - 32 + lane;
     int above = __popc(__ballot_sync(0xffffffffu, i1 >= 0 && __ldg(M + max(i1, 0)) >= wlo));
     if (lo == 32 || above == 32) {      // unusual schedule change inside a block: count everything
       int c0 = 0, c1 = 0;
       for (int i = lane; i < nm; i += 32) {
         const int x = __ldg(M + i);
-        c0 += x < s0;
+        c0 += x < vis_lo;
         c1 += x >= wlo;
       }
 #pragma unroll

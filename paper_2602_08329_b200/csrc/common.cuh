@@ -44,6 +44,14 @@ __device__ __forceinline__ long long row_offset(const KvDev& kv, int b, int kvh,
   return (long long)b * kv.stride_outer + (long long)kvh * kv.stride_head + (long long)i * kHeadDim;
 }
 
+// Start of the progressive sliding attention window (Eq. 11): P = floor(c * t) with
+// c = 1 - phi^(alpha (l - l_s) / (N - l_s)) computed on the host in double (0 = no window).
+__device__ __forceinline__ int psaw_start(double c, int t) {
+  if (c <= 0.0) return 0;
+  const int p = (int)floor(c * (double)t);
+  return max(0, min(p, t));
+}
+
 // bf16 pair (packed in 32 bits) -> two floats; exact.
 __device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }

@@ -3,6 +3,7 @@
 #include "../../include/prhs.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -33,6 +34,7 @@ struct FusedSet {
   const int* mid = nullptr;
   const int* n_mid = nullptr;
   int mid_stride = 0, sinks = 0, window = 0;
+  double psaw_c = 0.0;
 };
 
 // ---- scratch of the allocation-free entry point: split-K partials, merge tickets, flag word.
@@ -137,6 +139,9 @@ prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
     return fail(ctx, PRHS_ERR_CAPACITY, "schedule: layer_group below min_layer_group");
   if (s->top_k < 0 || s->window < 0 || s->sinks < 0 || s->dilate_r < 0 || s->dilate_m < -1)
     return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: negative budget");
+  if (s->psaw_layer_start < 0 ||
+      (s->psaw_layer_start > 0 && !(s->psaw_phi > 0.f && s->psaw_phi < 1.f && s->psaw_alpha >= 0.f)))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: sliding window needs 0 < phi < 1, alpha >= 0, l_s >= 0");
   if (s->top_k > ctx->cfg.max_k || s->window > ctx->cfg.max_window || s->sinks > ctx->cfg.max_sinks ||
       s->dilate_r > ctx->cfg.max_dilate_r || (s->dilate_m >= 0 && s->dilate_m > ctx->max_m))
     return fail(ctx, PRHS_ERR_CAPACITY, "schedule: budget exceeds the configured maximum");
@@ -215,6 +220,7 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.mid_stride = fs.mid_stride;
   p.sinks = fs.sinks;
   p.window = fs.window;
+  p.psaw_c = fs.psaw_c;
   p.num_q_heads = c->cfg.num_q_heads;
   p.group_size = c->gq;
   p.splits = pick_splits(c, batch * c->cfg.num_q_heads, max_count);
@@ -235,6 +241,14 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
 }
 
 int group_of(const prhs_schedule* s, int layer) { return layer / s->layer_group; }
+
+// Sliding-window factor c of Eq. 11 for a 0-based layer: P_l(t) = floor(c t); 0 = no window.
+double psaw_factor(const prhs_ctx* c, const prhs_schedule* s, int layer) {
+  const int N = c->cfg.num_layers, ls = s->psaw_layer_start, ell = layer + 1;
+  if (ls <= 0 || ell < ls || N <= ls) return 0.0;
+  const double expo = (double)s->psaw_alpha * (double)(ell - ls) / (double)(N - ls);
+  return 1.0 - std::pow((double)s->psaw_phi, expo);
+}
 
 size_t state_off(const prhs_ctx* c, int group, size_t per_unit) {
   return (size_t)group * units_max(c) * per_unit;
@@ -260,6 +274,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.window = s->window;
   p.r = s->dilate_r;
   p.m = s->dilate_m;
+  p.psaw_c = psaw_factor(c, s, layer);
   p.max_k = c->cfg.max_k;
   p.shat_cap = c->shat_cap;
   p.num_q_heads = c->cfg.num_q_heads;
@@ -298,6 +313,7 @@ prhs_status pick_middle(prhs_ctx* c, int layer, int step, const prhs_schedule* s
   fs->mid_stride = own ? c->cfg.max_k : c->shat_cap;
   fs->sinks = s->sinks;
   fs->window = s->window;
+  fs->psaw_c = psaw_factor(c, s, layer);
   return PRHS_OK;
 }
 
@@ -306,8 +322,8 @@ prhs_status launch_build(prhs_ctx* c, const FusedSet& fs, const int* seq_lens, i
   {
     LaunchScope ls(c, PRHS_KIND_BUILD, st);
     build_set_kernel<<<batch * c->cfg.num_q_heads, 128, 0, st>>>(
-        fs.mid, fs.n_mid, fs.mid_stride, seq_lens, fs.sinks, fs.window, c->cfg.num_q_heads, out_idx,
-        idx_stride, out_count);
+        fs.mid, fs.n_mid, fs.mid_stride, seq_lens, fs.sinks, fs.window, fs.psaw_c, c->cfg.num_q_heads,
+        out_idx, idx_stride, out_count);
   }
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
@@ -566,6 +582,7 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
   p.mid_stride = 0;
   p.sinks = 0;
   p.window = 0;
+  p.psaw_c = 0.0;
   p.num_q_heads = num_q_heads;
   p.group_size = num_q_heads / num_kv_heads;
   p.splits = splits;

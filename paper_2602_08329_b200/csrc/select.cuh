@@ -32,6 +32,7 @@ struct SelectParams {
   const int* seq_lens;
   const int* k_per_seq;     // or nullptr
   int k, sinks, window, r, m;
+  double psaw_c;            // sliding-window factor of this layer (0 = off)
   int max_k, shat_cap, num_q_heads;
   int* sstar_desc;          // [B][Hq][max_k]
   int* sstar_asc;           // [B][Hq][max_k]
@@ -159,7 +160,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   const int t = __ldg(p.seq_lens + b);
   int k = p.k_per_seq ? __ldg(p.k_per_seq + b) : p.k;
   k = max(0, min(k, p.max_k));
-  const int lo = min(p.sinks, t);
+  const int lo = max(min(p.sinks, t), psaw_start(p.psaw_c, t));   // first middle candidate
   const int n = max(t - p.window - lo, 0);
   const int kk = min(k, n);
   const int m_eff = min(p.m < 0 ? k / 3 : p.m, kk);

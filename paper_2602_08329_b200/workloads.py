@@ -59,6 +59,9 @@ class Workload:
     page_size: int = 0      # 0 = contiguous cache, 16 = paged
     min_context: int = 0    # > 0: ragged contexts uniform in [min_context, context]
     k_frac: float = 0.0     # > 0: per-sequence k = floor(k_frac * N_b)
+    psaw_layer_start: int = 0   # l_s of the sliding attention window (1-based); 0 = off
+    psaw_phi: float = 0.7
+    psaw_alpha: float = 1.0
 
     @property
     def capacity(self) -> int:

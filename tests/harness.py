@@ -65,7 +65,8 @@ def make_sched(w: W.Workload, device, flags=0, **over):
     kps_dev = kps.to(device) if kps is not None else None
     kw = dict(top_k=w.top_k, window=w.window, sinks=w.sinks, refresh_interval=w.refresh,
               layer_group=w.layer_group, dilate_r=w.dilate_r, dilate_m=-1, top_k_per_seq=kps_dev,
-              flags=flags)
+              flags=flags, psaw_phi=w.psaw_phi, psaw_alpha=w.psaw_alpha,
+              psaw_layer_start=w.psaw_layer_start)
     kw.update(over)
     return P.make_schedule(**kw)
 
@@ -74,7 +75,10 @@ def oracle_sched(w: W.Workload, **over) -> O.Schedule:
     kps = W.top_k_per_seq(w)
     kw = dict(top_k=w.top_k, window=w.window, sinks=w.sinks, refresh_interval=w.refresh,
               layer_group=w.layer_group, dilate_r=w.dilate_r, dilate_m=-1,
-              top_k_per_seq=None if kps is None else kps.numpy())
+              top_k_per_seq=None if kps is None else kps.numpy(),
+              # the C ABI carries phi and alpha as fp32: give the oracle the same values
+              psaw_phi=float(np.float32(w.psaw_phi)), psaw_alpha=float(np.float32(w.psaw_alpha)),
+              psaw_layer_start=w.psaw_layer_start, num_layers=w.layers)
     kw.update(over)
     return O.Schedule(**kw)
 
@@ -153,7 +157,7 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                 if retrieve:
                     a = O.dense_scores(qh[b, h], Kh, t)
                     a32 = O.rank_logits(a)
-                    want = O.topk_middle(a, t, w.sinks, w.window, osched.k_for(b))
+                    want = O.topk_middle(a, t, w.sinks, w.window, osched.k_for(b), osched.psaw_for(l, t))
                     got = s_star[b, h, : int(n_star[b, h])].numpy().astype(np.int64)
                     before = len(np.setxor1d(got, want))
                     check_topk_legal(a32, got, want, where)

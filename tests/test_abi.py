@@ -37,8 +37,9 @@ def test_version_and_struct_layout(lib):
     # the ctypes mirrors must have the C layout the header implies (LP64)
     assert ctypes.sizeof(P.Config) == 13 * 4
     assert ctypes.sizeof(P.KvView) == 64
-    assert ctypes.sizeof(P.Schedule) == 48
+    assert ctypes.sizeof(P.Schedule) == 56
     assert P.KvView.seq_lens.offset == 48 and P.Schedule.top_k_per_seq.offset == 16
+    assert P.Schedule.psaw_phi.offset == 44 and P.Schedule.psaw_layer_start.offset == 52
 
 
 def test_create_validates_before_touching_the_device(lib):

@@ -274,6 +274,17 @@ def test_schedule_cross_layer_groups(cuda_device):
     assert st["checked"] == 4 * 4 * w.batch * w.q_heads
 
 
+@pytest.mark.parametrize("phi,alpha,ls", [(0.7, 1.0, 3), (0.5, 2.0, 1), (0.9, 0.5, 4)])
+def test_schedule_with_sliding_window(cuda_device, phi, alpha, ls):
+    # progressive sliding attention window on the upper layers, with cross-layer groups:
+    # followers clip the leader's shared set by their own, larger window start
+    w = small(layers=4, layer_group=2, steps=4, refresh=2, q_heads=4, kv_heads=2, context=2600, seed=14,
+              psaw_layer_start=ls, psaw_phi=phi, psaw_alpha=alpha)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w))
+    assert st["checked"] == 4 * 4 * w.batch * w.q_heads
+    assert min(st["set_sizes"]) < max(st["set_sizes"])         # deeper layers attend over fewer rows
+
+
 def test_schedule_paged_and_ragged(cuda_device):
     w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=5, q_heads=8, kv_heads=2,
               context=3000, min_context=300, page_size=16, top_k=0, k_frac=0.03, seed=13)
@@ -330,6 +341,14 @@ def test_c3_stack_slice_sampled(cuda_device):
     w = W.C3_MISTRAL.scaled(layers=8, steps=5, batch=4)
     units = [(0, 0), (2, 21), (3, 31)]
     st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3, 4, 7])
+    assert st["checked"] == 5 * 5 * len(units)
+
+
+def test_c3_top_layers_with_sliding_window_sampled(cuda_device):
+    # layers 25..32 of a 32-layer stack prune with the paper's defaults (phi 0.7, alpha 1, l_s 24)
+    w = W.C3_MISTRAL.scaled(steps=5, batch=2, psaw_layer_start=24)
+    units = [(0, 3), (1, 30)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[24, 25, 27, 28, 31])
     assert st["checked"] == 5 * 5 * len(units)
 
 
