@@ -443,6 +443,237 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   }
 }
 
+// ---------------------------------------------------- dense flash-decode baseline (Eq. 2)
+// Attention over every position [0, t): K and V of a KV head are read ONCE for all the
+// query heads of its group, which sit on the 16 rows of the MMA tile (head j of the group =
+// row j).  Same warp-private cp.async ring, swizzle and fragment plumbing as the gathered
+// kernel; rows are consecutive, so the copies need no index list, and a 16-row stage that
+// starts on a multiple of 16 lies in one page of a paged cache.
+// grid (splits, Hkv, B).  Partials, tickets and outputs are per query head, as above.
+__device__ __forceinline__ void mma_bf16_full(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                              uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p) {
+  extern __shared__ __align__(128) unsigned char g_smem[];
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int gq = p.group_size;
+  const int head0 = kvh * gq;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  const int t = __ldg(p.kv.seq_lens + b);
+  int per = (t + p.splits * kTWarps - 1) / (p.splits * kTWarps);
+  per = (per + kTStageRows - 1) & ~(kTStageRows - 1);
+  const int start = min((split * kTWarps + warp) * per, t);
+  const int end = min(start + per, t);
+  const int nstages = (end - start + kTStageRows - 1) / kTStageRows;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(g_smem) + warp * (kTStages * kTStageBytes);
+  const bool has0 = g < gq, has1 = g + 8 < gq;
+
+  // A fragments of the group's queries: rows g and g + 8
+  uint32_t aq[8][4];
+  {
+    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + ((long long)b * p.num_q_heads + head0 + g) * kHeadDim);
+    const uint32_t* q1 = q0 + 8 * (kHeadDim / 2);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      aq[ks][0] = has0 ? __ldg(q0 + ks * 8 + tg) : 0u;
+      aq[ks][1] = has1 ? __ldg(q1 + ks * 8 + tg) : 0u;
+      aq[ks][2] = has0 ? __ldg(q0 + ks * 8 + 4 + tg) : 0u;
+      aq[ks][3] = has1 ? __ldg(q1 + ks * 8 + 4 + tg) : 0u;
+    }
+  }
+  float o[16][4];
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; o[nt][2] = 0.f; o[nt][3] = 0.f; }
+  float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // rows g and g + 8
+
+  const bool paged = p.kv.page_table != nullptr;
+  const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
+  const uint32_t dst_tile = (lane < 16 ? 0u : (uint32_t)kTTileBytes);
+  const long long lin_off = (long long)b * p.kv.stride_outer + (long long)kvh * p.kv.stride_head;
+  // paged: page id of the stage issued next, prefetched one stage ahead (start is a multiple of 16)
+  auto page_of_stage = [&](int j) -> int {
+    const int pos = start + j * kTStageRows;
+    if (!paged || pos >= end) return 0;
+    return __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
+  };
+  int pg_next = page_of_stage(0);
+
+  auto issue = [&](int j) {
+    if (j < nstages) {
+      const int pos0 = start + j * kTStageRows;
+      long long row_off = lin_off + (long long)pos0 * kHeadDim;
+      bool page_ok = true;
+      if (paged) {
+        const int page = pg_next;
+        pg_next = page_of_stage(j + 1);
+        page_ok = (unsigned)page < (unsigned)p.kv.num_pages;
+        if (!page_ok) atomicOr(p.flags, kFlagBadPage);
+        row_off = (long long)page * p.kv.stride_outer + (long long)kvh * p.kv.stride_head;
+      }
+      const uint32_t slot = ring + (uint32_t)(j % kTStages) * kTStageBytes + dst_tile;
+#pragma unroll
+      for (int r = 0; r < kTStageRows; ++r) {
+        const bool ok = page_ok && (pos0 + r < end);
+        const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
+        cp_async_16(dst, src_base + (ok ? row_off + (long long)r * kHeadDim : 0ll), ok ? 16 : 0);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int j = 0; j < kTStages - 1; ++j) issue(j);
+
+  const float sc = kScale * kLog2e;
+  const int lm_mi = lane >> 3, lm_r = lane & 7;
+  const int vrow = (lm_mi & 1) * 8 + lm_r;
+  for (int i = 0; i < nstages; ++i) {
+    cp_async_wait<kTStages - 2>();
+    __syncwarp();
+    issue(i + kTStages - 1);
+    const uint32_t kt = ring + (uint32_t)(i % kTStages) * kTStageBytes;
+    const uint32_t vt = kt + kTTileBytes;
+    const int pos0 = start + i * kTStageRows;
+    // ---- S = Q K^T for the whole group
+    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int pp = 0; pp < 4; ++pp) {
+      uint32_t bk0[4], bk1[4];
+      ldmatrix_x4(bk0, kt + lm_r * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+      ldmatrix_x4(bk1, kt + (8 + lm_r) * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+      mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
+      mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
+      mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
+      mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
+    }
+    // keys of this lane: pos0 + 2tg, +1 (n-tile 0) and pos0 + 8 + 2tg, +1 (n-tile 1)
+    const bool v0 = pos0 + 2 * tg < end, v1 = pos0 + 2 * tg + 1 < end;
+    const bool v2 = pos0 + 8 + 2 * tg < end, v3 = pos0 + 9 + 2 * tg < end;
+    float x[2][4];   // [row half][key]
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      x[hh][0] = v0 ? s[0][2 * hh] * sc : -INFINITY;
+      x[hh][1] = v1 ? s[0][2 * hh + 1] * sc : -INFINITY;
+      x[hh][2] = v2 ? s[1][2 * hh] * sc : -INFINITY;
+      x[hh][3] = v3 ? s[1][2 * hh + 1] * sc : -INFINITY;
+    }
+    // ---- online softmax per row (lazy reference exponent, as in the gathered kernel)
+    float mx0 = fmaxf(fmaxf(x[0][0], x[0][1]), fmaxf(x[0][2], x[0][3]));
+    float mx1 = fmaxf(fmaxf(x[1][0], x[1][1]), fmaxf(x[1][2], x[1][3]));
+    if (__any_sync(0xffffffffu, mx0 > m0 + 8.f || mx1 > m1 + 8.f)) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);
+      const float c0 = (n0 == -INFINITY) ? 1.f : exp2f(m0 - n0);
+      const float c1 = (n1 == -INFINITY) ? 1.f : exp2f(m1 - n1);
+      m0 = n0; m1 = n1;
+      l0 *= c0; l1 *= c1;
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c1; o[nt][3] *= c1; }
+    }
+    float pw[2][4];
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+      pw[0][k4] = (m0 == -INFINITY) ? 0.f : exp2f(x[0][k4] - m0);
+      pw[1][k4] = (m1 == -INFINITY) ? 0.f : exp2f(x[1][k4] - m1);
+    }
+    l0 += (pw[0][0] + pw[0][1]) + (pw[0][2] + pw[0][3]);
+    l1 += (pw[1][0] + pw[1][1]) + (pw[1][2] + pw[1][3]);
+    const uint32_t a0 = pack_bf16x2(pw[0][0], pw[0][1]), a1 = pack_bf16x2(pw[1][0], pw[1][1]);
+    const uint32_t a2 = pack_bf16x2(pw[0][2], pw[0][3]), a3 = pack_bf16x2(pw[1][2], pw[1][3]);
+    // ---- O += P V
+#pragma unroll
+    for (int np = 0; np < 8; ++np) {
+      uint32_t bv[4];
+      ldmatrix_x4_trans(bv, vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
+      mma_bf16_full(o[2 * np], a0, a1, a2, a3, bv[0], bv[1]);
+      mma_bf16_full(o[2 * np + 1], a0, a1, a2, a3, bv[2], bv[3]);
+    }
+  }
+  cp_async_wait<0>();
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+
+  // ---- combine the warps of this CTA; the ring is free now and holds [warp][head][128] floats
+  __syncthreads();
+  float* sm_o = reinterpret_cast<float*>(g_smem);                       // 4 x 16 x 128 floats = 32 KB
+  float* sm_m = sm_o + kTWarps * 16 * kHeadDim;                         // [warp][16]
+  float* sm_l = sm_m + kTWarps * 16;
+  __shared__ bool is_last;
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt) {
+    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
+    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g + 8) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][2], o[nt][3]);
+  }
+  if (tg == 0) {
+    sm_m[warp * 16 + g] = m0; sm_l[warp * 16 + g] = l0;
+    sm_m[warp * 16 + g + 8] = m1; sm_l[warp * 16 + g + 8] = l1;
+  }
+  __syncthreads();
+  for (int j = 0; j < gq; ++j) {
+    const int unit = b * p.num_q_heads + head0 + j;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w * 16 + j]);
+    float acc = 0.f, L = 0.f;
+    if (M != -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < kTWarps; ++w) {
+        const float scw = exp2f(sm_m[w * 16 + j] - M);
+        acc = fmaf(sm_o[(w * 16 + j) * kHeadDim + tid], scw, acc);
+        L = fmaf(sm_l[w * 16 + j], scw, L);
+      }
+    }
+    if (p.splits == 1) {
+      p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+      if (tid == 0 && p.out_lse) p.out_lse[unit] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    } else {
+      float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
+      part[tid] = acc;
+      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
+    }
+  }
+  if (p.splits == 1) return;
+  // ---- the last CTA of this (b, kvh) merges the split partials of the group's heads
+  __threadfence();
+  __syncthreads();
+  const int tunit = b * p.num_q_heads + head0;      // ticket slot: the group's first head
+  if (tid == 0) {
+    const unsigned int ticket = atomicAdd(p.tickets + tunit, 1u);
+    is_last = (ticket == (unsigned int)p.splits - 1u);
+    if (is_last) p.tickets[tunit] = 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int j = 0; j < gq; ++j) {
+    const int unit = tunit + j;
+    const float* base = p.partials + (long long)unit * p.splits * kPartStride;
+    float M = -INFINITY;
+    for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
+    float acc = 0.f, L = 0.f;
+    if (M != -INFINITY) {
+      for (int sp = 0; sp < p.splits; ++sp) {
+        const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
+        acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
+        L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
+      }
+    }
+    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+    if (tid == 0 && p.out_lse) p.out_lse[unit] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
+}
+
 // delta = 1 - exp(lse_C - lse_full)  (Sec. 2.3), one thread per (b, h).
 __global__ void delta_kernel(const float* __restrict__ lse_c, const float* __restrict__ lse_full,
                              float* __restrict__ out, int n) {

@@ -231,9 +231,15 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.lse_full = lse_full;
   p.out_delta = lse_full ? out_delta : nullptr;
   p.flags = c->flags;
-  dim3 grid(p.splits, c->cfg.num_q_heads, batch);
-  {
-    LaunchScope ls(c, (idx || fs.mid) ? PRHS_KIND_ATTN_SPARSE : PRHS_KIND_ATTN_DENSE, st);
+  if (!idx && !fs.mid) {
+    // dense baseline: one CTA column per KV head, the group's heads share the K/V stream
+    p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
+    dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
+    LaunchScope ls(c, PRHS_KIND_ATTN_DENSE, st);
+    dense_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
+  } else {
+    dim3 grid(p.splits, c->cfg.num_q_heads, batch);
+    LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
     gather_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   }
   PRHS_CUDA(c, cudaGetLastError());
@@ -401,6 +407,8 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
                              std::max(1024, (cfg->max_batch + 1) * (int)sizeof(int)));
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(dense_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess) {
     int nb = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, gather_attn_mma_kernel, kTThreads, kTSmemBytes);

@@ -1,0 +1,115 @@
+"""Attention-operator latency of the library on the shapes of the paper's efficiency study.
+
+    python -m paper_2602_08329_b200.operator_latency            # Table-3 shapes
+    python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C4 shapes
+
+The paper (Sec. 5.4, Table 3) times one attention layer of LLaMA-2-7B-Chat (32 MHA heads,
+head_dim 128) in decode at batch 8 / 16 and 1k-4k cached tokens, token sparsity 1/8, block
+size s = 8 / 16, against a dense FlashAttention-2 call, on an A100.  This script times the same
+shapes here: the in-library dense flash-decode kernel, a sharing step, a retrieval step, and the
+amortised per-step latency for s = 8 and 16.  Budgets follow Sec. 5.3.2 scaled to the length
+(C_sink 16, C_local 64, k = N/8 - 80).  Data are synthetic (`workloads.py`).
+
+Each figure is the median of per-step CUDA-event times over independent cache copies visited
+round-robin (so that no step finds its rows in L2).  Prints a markdown table.
+"""
+from __future__ import annotations
+
+import argparse
+import statistics
+
+import torch
+
+from . import binding as P
+from . import workloads as W
+
+PAPER_TABLE3_MS = {  # (batch, seqlen): (Flash, CPE-8, CPE-16) in ms on an A100 (Table 3)
+    (8, 1024): (0.230, 0.092, 0.078), (8, 2048): (0.830, 0.144, 0.095), (8, 4096): (1.630, 0.506, 0.469),
+    (16, 1024): (0.440, 0.089, 0.075), (16, 2048): (1.630, 0.196, 0.165), (16, 4096): (3.230, 0.904, 0.821),
+}
+
+
+def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6):
+    """Median device time (us) of a dense step, a retrieval step and a sharing step."""
+    w = w.scaled(layers=copies, steps=max(w.refresh, 2) + 1)
+    kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
+    q = W.make_queries(w, dev)
+    B, Hq = w.batch, w.q_heads
+    kps = W.top_k_per_seq(w)
+    max_k = max(w.top_k, int(w.k_frac * w.context))
+    ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
+                    page_size=0)
+    sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
+                            top_k_per_seq=None if kps is None else kps.to(dev))
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    t0, t1 = W.seq_lens_at(w, 0).to(dev), W.seq_lens_at(w, 1).to(dev)
+    views0 = [P.make_view(kv[l][0], kv[l][1], t0, max_seq_len=w.capacity) for l in range(copies)]
+    views1 = [P.make_view(kv[l][0], kv[l][1], t1, max_seq_len=w.capacity) for l in range(copies)]
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        ts = []
+        for r in range(reps):
+            evs = []
+            for l in range(copies):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn(l)
+                b.record(stream)
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            if r > 0:
+                ts += [a.elapsed_time(b) * 1e3 for a, b in evs]
+        return statistics.median(ts)
+
+    dense = timed(lambda l: ctx.dense_decode_attn(q[l, 0], views0[l], B, out))
+    refresh = timed(lambda l: ctx.decode_step(l, 0, sched, q[l, 0], views0[l], B, out))
+    shared = timed(lambda l: ctx.decode_step(l, 1, sched, q[l, 1], views1[l], B, out))
+    _, cnt = ctx.get_index_set(B)
+    ctx.close()
+    return {"dense_us": dense, "refresh_us": refresh, "shared_us": shared,
+            "set_size": float(cnt.float().mean())}
+
+
+def table3(dev):
+    print("| BS | seqlen | k | dense us | retrieval step us | sharing step us | amortised s=8 us | amortised s=16 us "
+          "| dense / s=16 | paper Flash / CPE-8 / CPE-16 ms (A100) |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
+    for batch in (8, 16):
+        for n in (1024, 2048, 4096):
+            k = n // 8 - 80
+            w = W.Workload(f"table3_b{batch}_{n}", layers=1, batch=batch, q_heads=32, kv_heads=32, context=n,
+                           steps=4, top_k=k, window=64, sinks=16, refresh=8, heavy_hitters=16,
+                           decay_span=min(512, n // 8), seed=100 + batch + n)
+            r = time_workload(w, dev)
+            am = {s: (r["refresh_us"] + (s - 1) * r["shared_us"]) / s for s in (8, 16)}
+            pf, p8, p16 = PAPER_TABLE3_MS[(batch, n)]
+            print(f"| {batch} | {n} | {k} | {r['dense_us']:.1f} | {r['refresh_us']:.1f} | {r['shared_us']:.1f} | "
+                  f"{am[8]:.1f} | {am[16]:.1f} | {r['dense_us'] / am[16]:.2f}x | {pf} / {p8} / {p16} |")
+
+
+def configs(dev):
+    print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
+          "mean set size | dense / amortised |")
+    print("|---|---|---|---|---|---|---|")
+    for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K):
+        r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 100000 else 2)
+        period = w.refresh * w.layer_group      # layer-steps per retrieval
+        am = (r["refresh_us"] + (period - 1) * r["shared_us"]) / period
+        print(f"| {w.name} | {r['dense_us']:.1f} | {r['refresh_us']:.1f} | {r['shared_us']:.1f} | {am:.1f} | "
+              f"{r['set_size']:.0f} | {r['dense_us'] / am:.2f}x |")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C4 shapes instead")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    (configs if args.configs else table3)(dev)
+
+
+if __name__ == "__main__":
+    main()

@@ -72,9 +72,9 @@ def test_sparse_attention_over_given_sets(cuda_device, gq):
     ctx.close()
 
 
-@pytest.mark.parametrize("gq", [1, 4])
+@pytest.mark.parametrize("gq", [1, 4, 8, 16])
 def test_dense_baseline_matches_oracle(cuda_device, gq):
-    w = small(q_heads=4, kv_heads=4 // gq, context=5000, seed=30 + gq)
+    w = small(q_heads=max(4, gq), kv_heads=max(4, gq) // gq, context=5000, seed=30 + gq)
     k, v = W.make_kv(w, cuda_device)
     q = W.make_queries(w, cuda_device)[0, 1].contiguous()
     t_host = torch.tensor([5003, 777], dtype=torch.int32)
@@ -307,10 +307,13 @@ def test_paged_identity_equals_contiguous(cuda_device):
         out = torch.empty(2, 4, 128, dtype=torch.bfloat16, device=cuda_device)
         ctx.decode_step(0, 0, H.make_sched(w, cuda_device), q, view, 2, out)
         idx, cnt = ctx.get_index_set(2)
-        outs.append((out.cpu(), idx, cnt))
+        dense = torch.empty_like(out)
+        ctx.dense_decode_attn(q, view, 2, dense)
+        outs.append((out.cpu(), idx, cnt, dense.cpu()))
         assert ctx.check() == 0
         ctx.close()
     assert torch.equal(outs[0][2], outs[1][2]) and torch.equal(outs[0][0], outs[1][0])
+    assert torch.equal(outs[0][3], outs[1][3])                 # the dense baseline through pages
 
 
 def test_c1_tiny_exactly_as_specified(cuda_device):
