@@ -674,6 +674,161 @@ __global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p)
   }
 }
 
+// ------------------------------------------------------- retrieval scoring, ring variant
+// Logits a_i = q . k_i / sqrt(d) for all i < t (Eq. 2) with the K stream staged like the dense
+// baseline's: warp-private cp.async ring (K tiles only, 6 stages of 16 rows), ldmatrix, one
+// MMA tile for all heads of the KV group.  Writes fp32 logits [B][Hq][ld] and per-(head, split)
+// online log-sum-exp partials part_ml[unit][split] in the log2 domain.
+// grid (splits, Hkv, B).
+constexpr int kSRStages = 6;
+constexpr int kSRSmemBytes = kTWarps * kSRStages * kTTileBytes;      // 96 KB
+
+struct ScoreParams {
+  const __nv_bfloat16* q;
+  KvDev kv;
+  float* scores;          // [B][Hq][ld] or nullptr (log-sum-exp only)
+  int ld;
+  float2* part_ml;        // [B][Hq][splits]
+  int splits, num_q_heads, group_size;
+  uint32_t* flags;
+};
+
+__global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
+  extern __shared__ __align__(128) unsigned char g_smem[];
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int gq = p.group_size;
+  const int head0 = kvh * gq;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  const int t = __ldg(p.kv.seq_lens + b);
+  int per = (t + p.splits * kTWarps - 1) / (p.splits * kTWarps);
+  per = (per + kTStageRows - 1) & ~(kTStageRows - 1);
+  const int start = min((split * kTWarps + warp) * per, t);
+  const int end = min(start + per, t);
+  const int nstages = (end - start + kTStageRows - 1) / kTStageRows;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(g_smem) + warp * (kSRStages * kTTileBytes);
+  const bool has0 = g < gq, has1 = g + 8 < gq;
+
+  uint32_t aq[8][4];
+  {
+    const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + ((long long)b * p.num_q_heads + head0 + g) * kHeadDim);
+    const uint32_t* q1 = q0 + 8 * (kHeadDim / 2);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      aq[ks][0] = has0 ? __ldg(q0 + ks * 8 + tg) : 0u;
+      aq[ks][1] = has1 ? __ldg(q1 + ks * 8 + tg) : 0u;
+      aq[ks][2] = has0 ? __ldg(q0 + ks * 8 + 4 + tg) : 0u;
+      aq[ks][3] = has1 ? __ldg(q1 + ks * 8 + 4 + tg) : 0u;
+    }
+  }
+  float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+
+  const bool paged = p.kv.page_table != nullptr;
+  // each lane copies 16 bytes; a K row is 16 lanes, so one instruction moves two rows
+  const __nv_bfloat16* src_base = p.kv.k + (lane & 15) * 8;
+  const int rsel = lane >> 4;                       // which of the two rows of a pair
+  const long long lin_off = (long long)b * p.kv.stride_outer + (long long)kvh * p.kv.stride_head;
+  auto page_of_stage = [&](int j) -> int {
+    const int pos = start + j * kTStageRows;
+    if (!paged || pos >= end) return 0;
+    return __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
+  };
+  int pg_next = page_of_stage(0);
+  auto issue = [&](int j) {
+    if (j < nstages) {
+      const int pos0 = start + j * kTStageRows;
+      long long row_off = lin_off + (long long)pos0 * kHeadDim;
+      bool page_ok = true;
+      if (paged) {
+        const int page = pg_next;
+        pg_next = page_of_stage(j + 1);
+        page_ok = (unsigned)page < (unsigned)p.kv.num_pages;
+        if (!page_ok) atomicOr(p.flags, kFlagBadPage);
+        row_off = (long long)page * p.kv.stride_outer + (long long)kvh * p.kv.stride_head;
+      }
+      const uint32_t slot = ring + (uint32_t)(j % kSRStages) * kTTileBytes;
+#pragma unroll
+      for (int rp = 0; rp < kTStageRows / 2; ++rp) {
+        const int r = 2 * rp + rsel;
+        const bool ok = page_ok && (pos0 + r < end);
+        const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
+        cp_async_16(dst, src_base + (ok ? row_off + (long long)r * kHeadDim : 0ll), ok ? 16 : 0);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int j = 0; j < kSRStages - 1; ++j) issue(j);
+
+  const int lm_mi = lane >> 3, lm_r = lane & 7;
+  for (int i = 0; i < nstages; ++i) {
+    cp_async_wait<kSRStages - 2>();
+    __syncwarp();
+    issue(i + kSRStages - 1);
+    const uint32_t kt = ring + (uint32_t)(i % kSRStages) * kTTileBytes;
+    const int pos0 = start + i * kTStageRows;
+    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int pp = 0; pp < 4; ++pp) {
+      uint32_t bk0[4], bk1[4];
+      ldmatrix_x4(bk0, kt + lm_r * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+      ldmatrix_x4(bk1, kt + (8 + lm_r) * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+      mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
+      mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
+      mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
+      mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
+    }
+    // lane (g, tg): head g -> s[nt][0..1], head g + 8 -> s[nt][2..3]; keys pos0 + 8 nt + 2 tg, +1
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      if (hh == 0 ? has0 : has1) {
+        float& m = hh == 0 ? m0 : m1;
+        float& l = hh == 0 ? l0 : l1;
+        float* dst = p.scores ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          const int key0 = pos0 + 8 * nt + 2 * tg;
+          const float s0 = s[nt][2 * hh] * kScale, s1 = s[nt][2 * hh + 1] * kScale;
+          if (key0 + 1 < end) {
+            if (dst) *reinterpret_cast<float2*>(dst + key0) = make_float2(s0, s1);
+            const float x0 = s0 * kLog2e, x1 = s1 * kLog2e;
+            const float mn = fmaxf(m, fmaxf(x0, x1));
+            l = l * exp2f(m - mn) + exp2f(x0 - mn) + exp2f(x1 - mn);
+            m = mn;
+          } else if (key0 < end) {
+            if (dst) dst[key0] = s0;
+            const float x0 = s0 * kLog2e;
+            const float mn = fmaxf(m, x0);
+            l = l * exp2f(m - mn) + exp2f(x0 - mn);
+            m = mn;
+          }
+        }
+      }
+    }
+  }
+  cp_async_wait<0>();
+  // ---- (m, l) per head: over the 4 lanes of a group, then over the warps
+#pragma unroll
+  for (int off = 1; off <= 2; off <<= 1) {
+    float m2 = __shfl_xor_sync(0xffffffffu, m0, off), l2 = __shfl_xor_sync(0xffffffffu, l0, off);
+    ml_combine(m0, l0, m2, l2);
+    m2 = __shfl_xor_sync(0xffffffffu, m1, off);
+    l2 = __shfl_xor_sync(0xffffffffu, l1, off);
+    ml_combine(m1, l1, m2, l2);
+  }
+  __shared__ float sm_m[kTWarps][16], sm_l[kTWarps][16];
+  if (tg == 0) {
+    sm_m[warp][g] = m0; sm_l[warp][g] = l0;
+    sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1;
+  }
+  __syncthreads();
+  if (tid < gq) {
+    float mm = -INFINITY, ll = 0.f;
+    for (int w = 0; w < kTWarps; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
+    p.part_ml[((long long)b * p.num_q_heads + head0 + tid) * p.splits + split] = make_float2(mm, ll);
+  }
+}
+
 // delta = 1 - exp(lse_C - lse_full)  (Sec. 2.3), one thread per (b, h).
 __global__ void delta_kernel(const float* __restrict__ lse_c, const float* __restrict__ lse_full,
                              float* __restrict__ out, int n) {
@@ -688,7 +843,8 @@ __global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunk
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int t = __ldg(seq_lens + i / num_q_heads);
-  const int nch = min(nchunks, (t + chunk_rows - 1) / chunk_rows);   // later chunks were never written
+  // chunk_rows > 0: chunks past t were never written; 0: every partial is valid
+  const int nch = chunk_rows > 0 ? min(nchunks, (t + chunk_rows - 1) / chunk_rows) : nchunks;
   float mm = -INFINITY, ll = 0.f;
   for (int c = 0; c < nch; ++c) {
     const float2 x = part_ml[(long long)i * nchunks + c];

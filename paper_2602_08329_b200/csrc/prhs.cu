@@ -12,14 +12,12 @@
 
 #include "attn.cuh"
 #include "common.cuh"
-#include "score.cuh"
 #include "select.cuh"
 
 using namespace prhs;
 
 namespace {
 
-constexpr int kChunkRows = 2048;        // keys scored per CTA (8 warps x 256 keys)
 constexpr int kMaxSplits = 64;          // split-K partial slots per (b, h)
 constexpr int kMaxSmemBytes = 227 * 1024;
 constexpr int kMaxContext = 1 << 20;
@@ -167,27 +165,6 @@ struct LaunchScope {
 };
 
 // ---- launchers -----------------------------------------------------------------------
-// `sched` != nullptr: a retrieval pass (logits are written and the selection histogram filled).
-prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
-                         const prhs_schedule* sched, cudaStream_t st, int* nchunks_out) {
-  const int write_scores = sched != nullptr;
-  const int nchunks = std::max(1, (max_t + kChunkRows - 1) / kChunkRows);
-  const __nv_bfloat16* qq = static_cast<const __nv_bfloat16*>(q);
-  {
-    LaunchScope ls(c, PRHS_KIND_SCORE, st);
-    const size_t smem = (size_t)(batch + 1) * sizeof(int);
-    const long long max_items = (long long)batch * c->cfg.num_kv_heads * nchunks;
-    const int grid = (int)std::max<long long>(1, std::min<long long>(max_items, (long long)c->sm_count * 2));
-    score_mma_kernel<<<grid, kScoreThreads, smem, st>>>(qq, kv, c->scores, c->ld, c->part_ml, nchunks,
-                                                        kChunkRows, c->cfg.num_q_heads,
-                                                        c->cfg.num_kv_heads, batch, write_scores,
-                                                        c->flags);
-  }
-  *nchunks_out = nchunks;
-  PRHS_CUDA(c, cudaGetLastError());
-  return PRHS_OK;
-}
-
 // Split count for the gathered attention: minimise (waves of CTAs) x (rows per CTA plus a
 // fixed per-CTA cost), so that the grid fills an integer number of waves of resident CTAs.
 int pick_splits(const prhs_ctx* c, int units, int max_count) {
@@ -204,6 +181,30 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
     if (cost < best_cost * 0.999) { best_cost = cost; best = s; }
   }
   return best;
+}
+
+// `sched` != nullptr: a retrieval pass (logits are written and the selection histogram filled).
+prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
+                         const prhs_schedule* sched, cudaStream_t st, int* nchunks_out) {
+  const int write_scores = sched != nullptr;
+  ScoreParams sp;
+  sp.q = static_cast<const __nv_bfloat16*>(q);
+  sp.kv = kv;
+  sp.scores = write_scores ? c->scores : nullptr;
+  sp.ld = c->ld;
+  sp.part_ml = c->part_ml;
+  sp.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_t);
+  sp.num_q_heads = c->cfg.num_q_heads;
+  sp.group_size = c->gq;
+  sp.flags = c->flags;
+  {
+    LaunchScope ls(c, PRHS_KIND_SCORE, st);
+    score_ring_kernel<<<dim3(sp.splits, c->cfg.num_kv_heads, batch), kTThreads, kSRSmemBytes, st>>>(sp);
+  }
+  const int nchunks = sp.splits;
+  *nchunks_out = nchunks;
+  PRHS_CUDA(c, cudaGetLastError());
+  return PRHS_OK;
 }
 
 prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
@@ -272,7 +273,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.ld = c->ld;
   p.part_ml = c->part_ml;
   p.nchunks = nchunks;
-  p.chunk_rows = kChunkRows;
+  p.chunk_rows = 0;          // every split partial is written
   p.seq_lens = kv.seq_lens;
   p.k_per_seq = s->top_k_per_seq;
   p.k = s->top_k;
@@ -381,7 +382,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   c->shat_cap = cfg->max_k + 2 * cfg->max_dilate_r * c->max_m;
   c->idx_cap = cfg->max_sinks + c->shat_cap + cfg->max_window;
   c->ld = (cfg->max_context + 63) & ~63;
-  c->max_chunks = (cfg->max_context + kChunkRows - 1) / kChunkRows;
+  c->max_chunks = kMaxSplits;
   while (c->sort_cap < cfg->max_k) c->sort_cap <<= 1;
   c->sort_cap <<= 1;   // room for a tie group that straddles the k-th place
   c->anchor_step.assign(c->num_groups, -1);
@@ -403,10 +404,9 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   }
   e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             std::max(1024, (cfg->max_batch + 1) * (int)sizeof(int)));
-  if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSRSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(dense_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess) {
@@ -417,7 +417,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
 
   const size_t U = units_max(c), G = c->num_groups;
   if (e == cudaSuccess) e = dev_alloc(&c->scores, U * c->ld);
-  if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * c->max_chunks);
+  if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * std::max(c->max_chunks, kMaxSplits));
   if (e == cudaSuccess) e = dev_alloc(&c->lse_full, U);
   if (e == cudaSuccess) e = dev_alloc(&c->lse_c, U);
   if (e == cudaSuccess) e = dev_alloc(&c->partials, U * kMaxSplits * kPartStride);
@@ -644,7 +644,7 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
     const int n = batch * ctx->cfg.num_q_heads;
     {
       LaunchScope ls(ctx, PRHS_KIND_MISC, st);
-      lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, kChunkRows, dv.seq_lens,
+      lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, 0, dv.seq_lens,
                                                          ctx->cfg.num_q_heads, ctx->lse_full, n);
     }
     PRHS_CUDA(ctx, cudaGetLastError());
@@ -712,7 +712,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
   const int n = batch * ctx->cfg.num_q_heads;
   {
     LaunchScope ls(ctx, PRHS_KIND_MISC, st);
-    lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, kChunkRows, dv.seq_lens,
+    lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, nchunks, 0, dv.seq_lens,
                                                          ctx->cfg.num_q_heads, ctx->lse_full, n);
   }
   PRHS_CUDA(ctx, cudaGetLastError());

@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   // full-softmax log-sum-exp from the scoring pass' per-chunk partials
   if (warp == 1) {
     float mm = -INFINITY, ll = 0.f;
-    const int nch = min(p.nchunks, (t + p.chunk_rows - 1) / p.chunk_rows);
+    const int nch = p.chunk_rows > 0 ? min(p.nchunks, (t + p.chunk_rows - 1) / p.chunk_rows) : p.nchunks;
     for (int c = lane; c < nch; c += 32) {
       const float2 x = p.part_ml[(long long)unit * p.nchunks + c];
       ml_combine(mm, ll, x.x, x.y);
