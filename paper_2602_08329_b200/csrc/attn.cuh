@@ -87,6 +87,9 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, int s
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
                : "memory");
 }
+__device__ __forceinline__ void cp_async_16_full(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -262,6 +265,10 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   int pos1 = check_pos(list_pos(0), 0);
   int pg1 = page_of(pos1);
   uint32_t rid_a = row_id(pos1, pg1);
+  // validity of the 32 entries of the group being issued, one bit per lane; invalid entries
+  // point at row 0 (a valid address) and are copied with size 0 (zero fill)
+  uint32_t valid_a = __ballot_sync(0xffffffffu, rid_a != kBadRow);
+  if (rid_a == kBadRow) rid_a = 0u;
   pos1 = check_pos(list_pos(1), 1);
   pg1 = page_of(pos1);
   int pos2 = list_pos(2);
@@ -275,20 +282,29 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
       if (j > 0 && (j & 1) == 0) {     // step the row-id pipeline
         const int grp = j >> 1;
         rid_a = row_id(pos1, pg1);
+        valid_a = __ballot_sync(0xffffffffu, rid_a != kBadRow);
+        if (rid_a == kBadRow) rid_a = 0u;
         pos1 = check_pos(pos2, grp + 1);
         pg1 = page_of(pos1);
         pos2 = list_pos(grp + 2);
       }
       const int slot_i = j % kTStages;
       const uint32_t slot = ring + (uint32_t)slot_i * kTStageBytes + dst_tile;
-      uint32_t vm = 0u;
+      const uint32_t vm = (valid_a >> ((j & 1) * kTStageRows)) & 0xffffu;
+      if (vm == 0xffffu) {             // the common case: 16 real rows
 #pragma unroll
-      for (int r = 0; r < kTStageRows; ++r) {
-        const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
-        const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
-        const bool ok = rid != kBadRow;
-        vm |= (ok ? 1u : 0u) << r;
-        cp_async_16(dst, src_base + (ok ? (long long)rid * kHeadDim : 0ll), ok ? 16 : 0);
+        for (int r = 0; r < kTStageRows; ++r) {
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
+          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
+          cp_async_16_full(dst, src_base + (size_t)rid * kHeadDim);
+        }
+      } else {
+#pragma unroll
+        for (int r = 0; r < kTStageRows; ++r) {
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
+          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
+          cp_async_16(dst, src_base + (size_t)rid * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
+        }
       }
       vmask = (vmask & ~(0xffffull << (16 * slot_i))) | ((unsigned long long)vm << (16 * slot_i));
     }
