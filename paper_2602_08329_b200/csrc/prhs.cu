@@ -385,6 +385,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   c->max_chunks = kMaxSplits;
   while (c->sort_cap < cfg->max_k) c->sort_cap <<= 1;
   c->sort_cap <<= 1;   // room for a tie group that straddles the k-th place
+  c->sort_cap = std::max(c->sort_cap, 64);   // the block sort works on 64-entry blocks
   c->anchor_step.assign(c->num_groups, -1);
 
   cudaError_t e = cudaGetDevice(&c->device);

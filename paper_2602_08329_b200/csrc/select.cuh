@@ -122,8 +122,8 @@ __device__ __forceinline__ unsigned long long make_entry(uint32_t key, int pos) 
 __device__ __forceinline__ void find_bin_from_top(const uint32_t* hist, int nb, int rem, uint32_t* misc) {
   const int lane = threadIdx.x & 31;
   const int per = nb >> 5;
-  int s = 0;
-  for (int j = 0; j < per; ++j) s += (int)hist[lane * per + j];
+  int s = 0;   // lane's bins are read in a rotated order: per is a multiple of 32 for large nb
+  for (int j = 0; j < per; ++j) s += (int)hist[lane * per + ((j + lane) % per)];
   int incl = s;   // sum over lanes >= lane
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
@@ -143,6 +143,64 @@ __device__ __forceinline__ void find_bin_from_top(const uint32_t* hist, int nb, 
       }
       c += hc;
     }
+  }
+}
+
+// ---- block-wide bitonic sort, descending, of P (a power of two >= 64) 64-bit entries in
+// shared memory.  Compare-exchange steps with a stride below 64 stay inside one 64-entry
+// block, which a warp holds in registers (two entries per lane) and resolves with shuffles;
+// only strides >= 64 go through shared memory with a CTA barrier.  All threads call it.
+__device__ __forceinline__ void warp_sort_steps(unsigned long long& a, unsigned long long& b, int pos_a,
+                                                int size, int first_stride) {
+  const int lane = threadIdx.x & 31;
+  const int pos_b = pos_a + 32;
+  for (int stride = first_stride; stride > 0; stride >>= 1) {
+    if (stride == 32) {
+      const bool desc = (pos_a & size) == 0;
+      if ((a < b) == desc) { const unsigned long long x = a; a = b; b = x; }
+    } else {
+      const unsigned long long oa = __shfl_xor_sync(0xffffffffu, a, stride);
+      const unsigned long long ob = __shfl_xor_sync(0xffffffffu, b, stride);
+      const bool lower = (lane & stride) == 0;
+      const bool da = (pos_a & size) == 0, db = (pos_b & size) == 0;
+      a = (lower == da) ? (a > oa ? a : oa) : (a < oa ? a : oa);
+      b = (lower == db) ? (b > ob ? b : ob) : (b < ob ? b : ob);
+    }
+  }
+}
+
+__device__ __forceinline__ void block_sort_desc(unsigned long long* buf, int P) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nwarps = blockDim.x >> 5;
+  const int nblocks = P >> 6;
+  // sizes 2 .. 64: entirely inside 64-entry blocks
+  for (int blk = warp; blk < nblocks; blk += nwarps) {
+    const int pos_a = blk * 64 + lane;
+    unsigned long long a = buf[pos_a], b = buf[pos_a + 32];
+    for (int size = 2; size <= 64; size <<= 1) warp_sort_steps(a, b, pos_a, size, size >> 1);
+    buf[pos_a] = a;
+    buf[pos_a + 32] = b;
+  }
+  __syncthreads();
+  for (int size = 128; size <= P; size <<= 1) {
+    for (int stride = size >> 1; stride >= 64; stride >>= 1) {
+      for (int x = tid; x < (P >> 1); x += blockDim.x) {
+        const int i = 2 * x - (x & (stride - 1));
+        const int j = i + stride;
+        const bool desc = ((i & size) == 0);
+        const unsigned long long a = buf[i], c = buf[j];
+        if ((a < c) == desc) { buf[i] = c; buf[j] = a; }
+      }
+      __syncthreads();
+    }
+    for (int blk = warp; blk < nblocks; blk += nwarps) {
+      const int pos_a = blk * 64 + lane;
+      unsigned long long a = buf[pos_a], b = buf[pos_a + 32];
+      warp_sort_steps(a, b, pos_a, size, 32);
+      buf[pos_a] = a;
+      buf[pos_a + 32] = b;
+    }
+    __syncthreads();
   }
 }
 
@@ -203,9 +261,16 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
       for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0u;
       __syncthreads();
       const int ns = n / kSampleStride;
-      for (int j = tid; j < ns; j += kSelThreads) {
-        const uint32_t u = float_to_key(__ldcg(g + j * kSampleStride + (j & (kSampleStride - 1))));
-        atomicAdd(&hist[u >> kHistShift], 1u);
+      for (int j0 = 0; j0 < ns; j0 += 8 * kSelThreads) {     // 8 independent loads in flight
+        uint32_t u8[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          const int j = j0 + x * kSelThreads + tid;
+          u8[x] = j < ns ? float_to_key(__ldcg(g + j * kSampleStride + (j & (kSampleStride - 1)))) : 0u;
+        }
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+          if (j0 + x * kSelThreads + tid < ns) atomicAdd(&hist[u8[x] >> kHistShift], 1u);
       }
       __syncthreads();
       // want at least 1.5 k/16 + 16 sampled logits at or above d_lo (several sigma of margin)
@@ -362,22 +427,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   }
 
   // ---- sort: descending key, ascending position among equal keys
-  int P = 2;
+  int P = 64;
   while (P < total) P <<= 1;
   for (int i = total + tid; i < P; i += kSelThreads) wbuf[i] = 0ull;
-  for (int size = 2; size <= P; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      __syncthreads();
-      for (int x = tid; x < (P >> 1); x += kSelThreads) {
-        const int i = 2 * x - (x & (stride - 1));
-        const int j = i + stride;
-        const bool desc = ((i & size) == 0);
-        const unsigned long long a = wbuf[i], c = wbuf[j];
-        if ((a < c) == desc) { wbuf[i] = c; wbuf[j] = a; }
-      }
-    }
-  }
   __syncthreads();
+  block_sort_desc(wbuf, P);
 
   // ---- S* in descending-logit order
   int* sd = p.sstar_desc + (long long)unit * p.max_k;
