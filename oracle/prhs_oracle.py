@@ -32,7 +32,7 @@ __all__ = [
     "dense_scores", "rank_logits", "softmax_full", "logsumexp", "dense_attention",
     "topk_middle", "dilate", "build_set", "attn_over_set", "retained_mass",
     "dropped_mass", "delta_from_lse", "mi_bound_g", "coverage", "bf16_round", "psaw_start",
-    "Schedule", "PrhsOracle",
+    "Schedule", "PrhsOracle", "cosine", "gate_decision",
 ]
 
 
@@ -216,6 +216,7 @@ class Schedule:
     dilate_m: int = -1             # -1 -> floor(k/3)
     dilate_anchor: bool = False    # True: the anchor's own attention also uses S^
     top_k_per_seq: np.ndarray | None = None
+    sim_threshold: float | None = None   # tau of the cosine gate (Eq. 9; Sec. 5.1 default 0.8); None = fixed schedule
     psaw_phi: float = 0.7          # Eq. 11 (defaults Sec. 5.1)
     psaw_alpha: float = 1.0
     psaw_layer_start: int = 0      # l_s, 1-based; 0 = no sliding window
@@ -231,75 +232,137 @@ class Schedule:
         return psaw_start(layer, self.num_layers, t, self.psaw_phi, self.psaw_alpha, self.psaw_layer_start)
 
 
+def cosine(q1: np.ndarray, q2: np.ndarray) -> float:
+    """sim(i, j) = q_i . q_j / (|q_i| |q_j|)  (Eq. 9), float64."""
+    a, b = q1.astype(np.float64), q2.astype(np.float64)
+    return float(a @ b / (math.sqrt(float(a @ a)) * math.sqrt(float(b @ b))))
+
+
+def gate_decision(q: np.ndarray, earlier: list, tau: float):
+    """Cosine gate of CIS (Sec. 4.1 "Similarity Criteria").
+
+    `earlier` lists the queries of the earlier steps of the block, oldest first.  Returns
+    (ref, sims): ref = index into `earlier` of the MOST RECENT query with sim > tau, or -1
+    if none (the head must retrieve); sims = the similarities, aligned with `earlier`.
+    """
+    sims = [cosine(q, e) for e in earlier]
+    for j in range(len(earlier) - 1, -1, -1):
+        if sims[j] > tau:
+            return j, sims
+    return -1, sims
+
+
 @dataclass
-class _Shared:
-    step: int = -1
-    s_star: dict = field(default_factory=dict)   # (b, h) -> S* (descending weight)
-    s_hat: dict = field(default_factory=dict)    # (b, h) -> S^ (ascending)
+class _Block:
+    """What one (layer group, sequence, head) remembers inside the current block."""
+    start: int = -1                                     # first step of the block
+    queries: list = field(default_factory=list)         # q of every step so far, by position
+    set_of_pos: list = field(default_factory=list)      # which set each step attended over
+    sets: list = field(default_factory=list)            # (s_star, s_hat) per retrieval, in order
+    own_at: int = -1                                    # step of the latest retrieval
 
 
 class PrhsOracle:
     """Runs the decode-step schedule one (layer, step) at a time.
 
-    A (layer, step) retrieves iff the layer is the first of its group and the step is the
-    first of its block (step % s == 0).  The retrieving call stores S* and its dilation
-    S^ (Eq. 10) per (sequence, query head).  Every other (layer, step) of the same block
-    and group attends over C built from the stored S^ (Def. 3.2) with its own q, K, V.
-    The retrieving call itself attends over C built from the undilated S* unless
-    `dilate_anchor` is set (dilation costs budget "during sharing", Sec. 5.2.2).
+    Blocks of `refresh_interval` steps (Sec. 4.1): the first step of a block retrieves.  A later
+    step of the block, on the first layer of its layer group,
+      * without a similarity threshold shares the block's first set (fixed schedule);
+      * with `sim_threshold` = tau applies the cosine gate per head: it shares the set used by
+        the most recent earlier step of the block whose query has cosine similarity > tau,
+        and retrieves a new set if there is none.
+    A retrieval stores S* and its dilation S^ (Eq. 10).  The retrieving call attends over C
+    built from the undilated S* unless `dilate_anchor` is set (dilation costs budget "during
+    sharing", Sec. 5.2.2); every sharer attends over C built from S^ (Def. 3.2) with its own
+    q, K, V.  The other layers of a group follow the decision and the set of its first layer.
+
+    `override_ref` / `override_s_star` (per (b, h)) let a test substitute a decision or a
+    retrieved S* that it has checked to be legal (a similarity within rounding of tau, a
+    near-tie at the k-th logit), so that everything downstream can be compared exactly.
     """
 
     def __init__(self, sched: Schedule, num_q_heads: int, num_kv_heads: int):
         self.s = sched
         self.hq, self.hkv = num_q_heads, num_kv_heads
         self.gq = num_q_heads // num_kv_heads
-        self.groups: dict[int, _Shared] = {}
+        self.blocks: dict = {}          # (group, b, h) -> _Block
+        self.last: dict = {}            # (group, b, h) -> (step, set id, own) of the latest leader call
+        self.retrievals = 0             # head-level retrievals so far (for the retrieval ratio)
+        self.calls = 0                  # head-level (layer, step) calls so far
 
     def is_retrieval(self, layer: int, step: int) -> bool:
+        """True where the FIXED schedule retrieves (first layer of a group, first step of a block)."""
         return layer % self.s.layer_group == 0 and step % self.s.refresh_interval == 0
 
-    def index_set(self, layer: int, step: int, b: int, h: int, t: int) -> np.ndarray:
+    def _plan(self, layer, step, b, h, q_bh, override_ref):
+        """Decide what (layer, step) does for head (b, h): returns (block, set id, own, ref)."""
         g = layer // self.s.layer_group
-        sh = self.groups.get(g)
-        anchor = step - step % self.s.refresh_interval
-        if sh is None or sh.step != anchor:
+        key = (g, b, h)
+        if layer % self.s.layer_group != 0:           # follower: the leader's decision of this step
+            if key not in self.last or self.last[key][0] != step:
+                raise RuntimeError("group leader has not been called for this step")
+            return self.blocks[key], self.last[key][1], False, None
+        pos = step % self.s.refresh_interval
+        blk = self.blocks.get(key)
+        if pos == 0:
+            blk = self.blocks[key] = _Block(start=step)
+        elif blk is None or blk.start != step - pos or len(blk.queries) != pos:
             raise RuntimeError("group leader has not retrieved for this block")
-        own = self.is_retrieval(layer, step) and not self.s.dilate_anchor
-        M = sh.s_star[(b, h)] if own else sh.s_hat[(b, h)]
-        return build_set(t, self.s.sinks, self.s.window, M, self.s.psaw_for(layer, t))
+        if pos == 0:
+            ref = -1
+        elif override_ref is not None and (b, h) in override_ref:
+            ref = int(override_ref[(b, h)])
+        elif self.s.sim_threshold is None:
+            ref = 0
+        else:
+            ref, _ = gate_decision(q_bh, blk.queries, self.s.sim_threshold)
+        own = ref < 0
+        set_id = len(blk.sets) if own else blk.set_of_pos[ref]
+        return blk, set_id, own, ref
 
-    def decode_step(self, layer, step, q, K, V, seq_lens, units=None, want_delta=True):
+    def decode_step(self, layer, step, q, K, V, seq_lens, units=None, want_delta=True,
+                    override_ref=None, override_s_star=None):
         """q [B][Hq][d]; K, V [B][Hkv][cap][d]; seq_lens [B].
 
         `units` optionally restricts the work to a list of (b, h) pairs (sampled parity).
-        Returns dict with per-unit 'y' (float64), 'lse', 'delta', 'set', and on retrieval
-        steps 's_star', 'lse_full', 'scores32'.
+        Returns dict with per-unit 'y' (float64), 'lse', 'delta', 'set', 'retrieved' (bool),
+        'ref' (position in the block shared from, -1 = retrieved) and, where retrieved,
+        's_star', 's_hat', 'lse_full', 'scores32'.
         """
         B = q.shape[0]
         if units is None:
             units = [(b, h) for b in range(B) for h in range(self.hq)]
-        g = layer // self.s.layer_group
-        retrieve = self.is_retrieval(layer, step)
-        if retrieve:
-            sh = self.groups.setdefault(g, _Shared())
-            if sh.step != step:
-                sh.step, sh.s_star, sh.s_hat = step, {}, {}
+        leader = layer % self.s.layer_group == 0
         out = {"y": {}, "lse": {}, "delta": {}, "set": {}, "s_star": {}, "lse_full": {},
-               "scores32": {}}
+               "scores32": {}, "retrieved": {}, "ref": {}, "s_hat": {}}
         for (b, h) in units:
             t = int(seq_lens[b])
             kv = h // self.gq
+            blk, set_id, own, ref = self._plan(layer, step, b, h, q[b, h], override_ref)
             a = None
-            if retrieve:
+            if own:
                 a = dense_scores(q[b, h], K[b, kv], t)
-                s_star = topk_middle(a, t, self.s.sinks, self.s.window, self.s.k_for(b),
-                                     self.s.psaw_for(layer, t))
-                sh = self.groups[g]
-                sh.s_star[(b, h)] = s_star
-                sh.s_hat[(b, h)] = dilate(s_star, self.s.m_for(b), self.s.dilate_r, t)
+                if override_s_star is not None and (b, h) in override_s_star:
+                    s_star = np.asarray(override_s_star[(b, h)], dtype=np.int64)
+                else:
+                    s_star = topk_middle(a, t, self.s.sinks, self.s.window, self.s.k_for(b),
+                                         self.s.psaw_for(layer, t))
+                blk.sets.append((s_star, dilate(s_star, self.s.m_for(b), self.s.dilate_r, t)))
                 out["s_star"][(b, h)] = s_star
+                out["s_hat"][(b, h)] = blk.sets[-1][1]
                 out["scores32"][(b, h)] = rank_logits(a)
-            C = self.index_set(layer, step, b, h, t)
+                self.retrievals += 1
+            if leader:
+                g = layer // self.s.layer_group
+                blk.queries.append(np.array(q[b, h], dtype=np.float64))
+                blk.set_of_pos.append(set_id)
+                out["ref"][(b, h)] = ref
+                self.last[(g, b, h)] = (step, set_id, own)
+            self.calls += 1
+            out["retrieved"][(b, h)] = own
+            s_star, s_hat = blk.sets[set_id]
+            M = s_star if (own and not self.s.dilate_anchor) else s_hat
+            C = build_set(t, self.s.sinks, self.s.window, M, self.s.psaw_for(layer, t))
             y, lse_c = attn_over_set(q[b, h], K[b, kv], V[b, kv], C)
             out["set"][(b, h)], out["y"][(b, h)], out["lse"][(b, h)] = C, y, lse_c
             if want_delta:
@@ -309,3 +372,7 @@ class PrhsOracle:
                 out["lse_full"][(b, h)] = lse_full
                 out["delta"][(b, h)] = delta_from_lse(lse_c, lse_full)
         return out
+
+    def retrieval_ratio(self) -> float:
+        """rho-hat of Sec. 5.1: head-level retrievals / head-level (layer, step) calls so far."""
+        return self.retrievals / max(1, self.calls)

@@ -348,6 +348,75 @@ def test_dilated_set_covers_next_topk_on_clustered_keys():
     assert O.coverage(np.sort(s1), s2) == 0.0
 
 
+# -------------------------------------------------------------- cosine gate, Eq. 9 / Sec. 4.1
+def test_cosine_similarity_against_library_and_closed_forms():
+    g = rng(40)
+    a, b = g.standard_normal(128), g.standard_normal(128)
+    want = torch.nn.functional.cosine_similarity(torch.from_numpy(a)[None], torch.from_numpy(b)[None]).item()
+    assert O.cosine(a, b) == pytest.approx(want, rel=1e-12)
+    assert O.cosine(a, 3.5 * a) == pytest.approx(1.0, abs=1e-15)          # scale invariant
+    assert O.cosine(a, -a) == pytest.approx(-1.0, abs=1e-15)
+    e0, e1 = np.eye(128)[0], np.eye(128)[1]
+    assert O.cosine(e0, e1) == 0.0
+    assert O.cosine(e0, e0 + e1) == pytest.approx(math.sqrt(0.5), rel=1e-15)
+
+
+def test_gate_picks_the_most_recent_similar_query():
+    e = np.eye(128)
+    q = e[0] + 0.1 * e[1]
+    earlier = [e[0], e[1], e[0] + 0.2 * e[1], e[2]]      # sims: .995, .0995, .995.., 0
+    ref, sims = O.gate_decision(q, earlier, 0.8)
+    assert ref == 2 and sims[0] > 0.8 and sims[2] > 0.8 and sims[3] == 0.0   # 0 also passes; 2 is later
+    assert O.gate_decision(q, earlier, 0.9999)[0] == -1                     # none similar enough
+    assert O.gate_decision(q, [], 0.8)[0] == -1
+    assert O.gate_decision(q, earlier, -1.0)[0] == 3                         # everything passes
+
+
+def test_gated_schedule_limits():
+    q, K, V = _stack(25, layers=1)
+    t = lambda n: np.array([200 + n + 1, 150 + n + 1])
+    base = dict(top_k=20, window=8, sinks=2, refresh_interval=4)
+    fixed = O.PrhsOracle(O.Schedule(**base), 4, 2)
+    always = O.PrhsOracle(O.Schedule(**base, sim_threshold=-1.0), 4, 2)     # gate always passes
+    never = O.PrhsOracle(O.Schedule(**base, sim_threshold=1.0), 4, 2)       # gate never passes
+    every = O.PrhsOracle(O.Schedule(**{**base, "refresh_interval": 1}), 4, 2)
+    for n in range(6):
+        a = fixed.decode_step(0, n, q[0, n], K[0], V[0], t(n))
+        b = always.decode_step(0, n, q[0, n], K[0], V[0], t(n))
+        c = never.decode_step(0, n, q[0, n], K[0], V[0], t(n))
+        d = every.decode_step(0, n, q[0, n], K[0], V[0], t(n))
+        for u in a["set"]:
+            assert np.array_equal(a["set"][u], b["set"][u])       # tau = -1 is the fixed schedule
+            assert np.array_equal(c["set"][u], d["set"][u])       # tau = 1 retrieves every step
+            assert c["retrieved"][u] and (a["retrieved"][u] == (n % 4 == 0))
+            assert b["ref"][u] == (-1 if n % 4 == 0 else n % 4 - 1)   # shares from the most recent step
+    assert fixed.retrieval_ratio() == pytest.approx(2 / 6) and never.retrieval_ratio() == 1.0
+
+
+def test_gated_schedule_mixed_heads():
+    # head 0 keeps its query, head 1 jumps at step 2: only head 1 retrieves there, and step 3
+    # shares from the most recent similar step (2 for head 1, still the block's first set for head 0)
+    g = rng(41)
+    K = bf16(g.standard_normal((1, 1, 300, 128)))
+    V = bf16(g.standard_normal((1, 1, 300, 128)))
+    base_q = bf16(g.standard_normal((2, 128)) * 2)
+    other = bf16(g.standard_normal(128) * 2)
+    orc = O.PrhsOracle(O.Schedule(top_k=16, window=8, sinks=2, refresh_interval=4, sim_threshold=0.8), 2, 1)
+    outs = []
+    for n in range(4):
+        q = np.array(base_q, copy=True)[None]
+        if n >= 2:
+            q[0, 1] = other
+        outs.append(orc.decode_step(0, n, q, K, V, np.array([280 + n])))
+    assert [o["retrieved"][(0, 0)] for o in outs] == [True, False, False, False]
+    assert [o["retrieved"][(0, 1)] for o in outs] == [True, False, True, False]
+    assert [o["ref"][(0, 1)] for o in outs] == [-1, 0, -1, 2]
+    s2 = outs[2]["s_star"][(0, 1)]
+    want3 = O.build_set(283, 2, 8, O.dilate(s2, 16 // 3, 1, 282))
+    assert np.array_equal(outs[3]["set"][(0, 1)], want3)
+    assert orc.retrieval_ratio() == pytest.approx(3 / 8)
+
+
 # ------------------------------------------------------- sliding attention window, Eq. 11
 def test_psaw_window_start_worked_values():
     with open(os.path.join(GOLDEN, "psaw_window_start.txt")) as f:
@@ -491,6 +560,8 @@ def test_schedule_cross_layer_followers_use_the_leader_set():
             assert np.array_equal(p["set"][u], outs[0]["set"][u])
     with pytest.raises(RuntimeError):
         O.PrhsOracle(s, 4, 2).decode_step(1, 0, q[1, 0], K[1], V[1], np.array([211, 191]))
+    with pytest.raises(RuntimeError):
+        O.PrhsOracle(s, 4, 2).decode_step(0, 1, q[0, 1], K[0], V[0], np.array([211, 191]))
 
 
 def test_schedule_sampled_units_match_full_run():
