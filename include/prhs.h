@@ -65,6 +65,8 @@ typedef struct {
   int32_t max_dilate_r;  /* largest dilation radius r */
   int32_t max_dilate_m;  /* largest number of dilated winners m; -1 = floor(max_k / 3) */
   int32_t min_layer_group; /* smallest layer_group that will be used (sizes the state); >= 1 */
+  int32_t max_block_sets;  /* sets kept per (b, h) and block, 1..64; 1 unless the cosine gate is
+                              used, which needs max_block_sets >= refresh_interval              */
 } prhs_config;
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
@@ -110,6 +112,14 @@ typedef struct {
   float psaw_phi;               /* phi in (0, 1); default 0.7 (Sec. 5.1)                        */
   float psaw_alpha;             /* alpha >= 0; default 1                                        */
   int32_t psaw_layer_start;     /* l_s; default floor(3 N / 4); 0 disables the window           */
+  /* Cosine gate of CIS (Sec. 4.1 "Similarity Criteria", Eq. 9).  With sim_threshold = tau > -1
+   * a step that is not the first of its block shares, per head, the set used by the MOST RECENT
+   * earlier step of the block whose query has cosine similarity > tau with the current query,
+   * and retrieves a new set only if there is none (paper default tau = 0.8).  The decision is
+   * taken on the device by the group's first layer; the other layers of the group follow it.
+   * Within a block the steps must then be run in order.  sim_threshold <= -1: gate off, every
+   * step of a block shares the block's first set (the fixed schedule). */
+  float sim_threshold;
 } prhs_schedule;
 
 /* Create / destroy a context on the current CUDA device.  prhs_create allocates every
@@ -238,10 +248,17 @@ prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx,
 
 /* Copy the stored shared sets of `layer`'s group to the host: host_s_star (descending
  * logit) [batch][Hq][max_k], host_s_hat (ascending) [batch][Hq][max_k + 2*r*m], their
- * counts [batch][Hq] each.  Any pointer may be NULL.  Synchronous. */
+ * counts [batch][Hq] each; per head, the set it attended over in the group's latest step.
+ * Any pointer may be NULL.  Synchronous. */
 prhs_status prhs_get_shared_set(prhs_ctx* ctx, int32_t layer, int32_t batch, int32_t* host_s_star,
                                 int32_t* host_n_star, int32_t* host_s_hat, int32_t* host_n_hat,
                                 void* stream);
+
+/* Decision of the cosine gate in the latest gated step of `layer`'s group: host_need int32
+ * [batch][Hq] (1 = the head retrieved), host_ref int32 [batch][Hq] (position in the block of
+ * the step it shares from, -1 = retrieved).  Either pointer may be NULL.  Synchronous. */
+prhs_status prhs_get_gate(prhs_ctx* ctx, int32_t layer, int32_t batch, int32_t* host_need,
+                          int32_t* host_ref, void* stream);
 
 /* Copy the logits of the last retrieval pass to the host: fp32 [batch][Hq][ld] with
  * ld = prhs_scores_ld().  Synchronous; for tests. */

@@ -28,7 +28,7 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_decode_step_host", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
            "prhs_launch_count", "prhs_last_error", "prhs_version", "prhs_profile_begin",
-           "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc"]
+           "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate"]
 NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
 
@@ -43,7 +43,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_layers", "max_batch", "num_q_heads", "num_kv_heads", "head_dim", "max_context",
         "page_size", "max_k", "max_window", "max_sinks", "max_dilate_r", "max_dilate_m",
-        "min_layer_group")]
+        "min_layer_group", "max_block_sets")]
 
 
 class KvView(C.Structure):
@@ -57,7 +57,8 @@ class Schedule(C.Structure):
     _fields_ = [("refresh_interval", C.c_int32), ("layer_group", C.c_int32), ("top_k", C.c_int32),
                 ("top_k_per_seq", C.c_void_p), ("window", C.c_int32), ("sinks", C.c_int32),
                 ("dilate_r", C.c_int32), ("dilate_m", C.c_int32), ("flags", C.c_uint32),
-                ("psaw_phi", C.c_float), ("psaw_alpha", C.c_float), ("psaw_layer_start", C.c_int32)]
+                ("psaw_phi", C.c_float), ("psaw_alpha", C.c_float), ("psaw_layer_start", C.c_int32),
+                ("sim_threshold", C.c_float)]
 
 
 _lib = None
@@ -88,6 +89,7 @@ def load() -> C.CDLL:
         "prhs_get_index_set": (st, [vp, i32, vp, vp, vp]),
         "prhs_get_shared_set": (st, [vp, i32, i32, vp, vp, vp, vp, vp]),
         "prhs_get_scores": (st, [vp, i32, vp, vp]),
+        "prhs_get_gate": (st, [vp, i32, i32, vp, vp, vp]),
         "prhs_scores_ld": (i32, [vp]),
         "prhs_check": (st, [vp, vp, C.POINTER(C.c_uint32)]),
         "prhs_profile_begin": (st, [vp, i32]),
@@ -120,9 +122,10 @@ def _stream(stream=None):
 
 
 def make_schedule(top_k, window, sinks, refresh_interval=1, layer_group=1, dilate_r=1, dilate_m=-1,
-                  top_k_per_seq=None, flags=0, psaw_phi=0.7, psaw_alpha=1.0, psaw_layer_start=0) -> Schedule:
+                  top_k_per_seq=None, flags=0, psaw_phi=0.7, psaw_alpha=1.0, psaw_layer_start=0,
+                  sim_threshold=-1.0) -> Schedule:
     s = Schedule(refresh_interval, layer_group, top_k, _ptr(top_k_per_seq), window, sinks,
-                 dilate_r, dilate_m, flags, psaw_phi, psaw_alpha, psaw_layer_start)
+                 dilate_r, dilate_m, flags, psaw_phi, psaw_alpha, psaw_layer_start, sim_threshold)
     s._keep = top_k_per_seq
     return s
 
@@ -144,11 +147,11 @@ class Context:
 
     def __init__(self, num_layers, max_batch, num_q_heads, num_kv_heads, max_context, max_k,
                  max_window, max_sinks, max_dilate_r=1, max_dilate_m=-1, page_size=0,
-                 min_layer_group=1, head_dim=128):
+                 min_layer_group=1, head_dim=128, max_block_sets=1):
         self.lib = load()
         self.cfg = Config(num_layers, max_batch, num_q_heads, num_kv_heads, head_dim, max_context,
                           page_size, max_k, max_window, max_sinks, max_dilate_r, max_dilate_m,
-                          min_layer_group)
+                          min_layer_group, max_block_sets)
         h = C.c_void_p()
         rc = self.lib.prhs_create(C.byref(self.cfg), C.byref(h))
         if rc != PRHS_OK:
@@ -236,6 +239,12 @@ class Context:
         self._ck(self.lib.prhs_get_shared_set(self.h, layer, batch, s_star.data_ptr(), n_star.data_ptr(),
                                               s_hat.data_ptr(), n_hat.data_ptr(), _stream(stream)))
         return s_star, n_star, s_hat, n_hat
+
+    def get_gate(self, layer, batch, stream=None):
+        need = torch.empty(batch, self.cfg.num_q_heads, dtype=torch.int32)
+        ref = torch.empty(batch, self.cfg.num_q_heads, dtype=torch.int32)
+        self._ck(self.lib.prhs_get_gate(self.h, layer, batch, need.data_ptr(), ref.data_ptr(), _stream(stream)))
+        return need, ref
 
     def get_scores(self, batch, stream=None):
         out = torch.empty(batch, self.cfg.num_q_heads, self.scores_ld, dtype=torch.float32)

@@ -10,17 +10,16 @@ namespace prhs {
 // unique already, so the union is: the sink run, M clipped to [S0', wlo), the window run.
 // One CTA per (sequence, query head).
 __global__ void __launch_bounds__(128)
-build_set_kernel(const int* __restrict__ mid, const int* __restrict__ n_mid, int mid_stride,
-                 const int* __restrict__ seq_lens, int sinks, int window, double psaw_c, int num_q_heads,
+build_set_kernel(SetRef ref, const int* __restrict__ seq_lens, int num_q_heads,
                  int* __restrict__ out_idx, int idx_stride, int* __restrict__ out_count) {
   const int unit = blockIdx.x;
   const int b = unit / num_q_heads;
   const int t = __ldg(seq_lens + b);
-  const int* M = mid + (long long)unit * mid_stride;
-  const int nm = __ldg(n_mid + unit);
-  const int s0 = min(sinks, t);
-  const int vis_lo = max(s0, psaw_start(psaw_c, t));      // first visible non-sink position
-  const int wlo = max(max(t - window, 0), vis_lo);
+  int nm, mstride;
+  const int* M = middle_of(ref, unit, &nm, &mstride);
+  const int s0 = min(ref.sinks, t);
+  const int vis_lo = max(s0, psaw_start(ref.psaw_c, t));  // first visible non-sink position
+  const int wlo = max(max(t - ref.window, 0), vis_lo);
   // M is ascending: the number of entries below a bound is the position of the bound.  Count
   // in parallel (one coalesced pass) instead of a binary search of dependent cold loads.
   __shared__ int sh_lo, sh_hi;
@@ -62,13 +61,10 @@ struct AttnParams {
   const int* idx;           // [B][Hq][idx_stride] or nullptr
   const int* count;         // [B][Hq] (with idx)
   int idx_stride;
-  // fused index-set builder (used when idx == nullptr and mid != nullptr): the list is
-  // [0, s0) ++ M clipped to [s0, wlo) ++ [wlo, t) with M = mid[unit][0..n_mid[unit]) ascending
-  const int* mid;
-  const int* n_mid;
-  int mid_stride, sinks, window;
-  double psaw_c;            // sliding-window factor of this layer (0 = off), fused mode only
-  // idx == nullptr and mid == nullptr: all positions [0, t) (dense baseline)
+  // fused index-set builder (used when idx == nullptr and set.star != nullptr): the list is
+  // [0, s0) ++ M clipped to [vis_lo, wlo) ++ [wlo, t) with M the unit's stored middle set
+  SetRef set;
+  // idx == nullptr and set.star == nullptr: all positions [0, t) (dense baseline)
   int num_q_heads, group_size;
   int splits;
   float* partials;          // [B][Hq][splits][kPartStride]
@@ -114,12 +110,12 @@ __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit
   if (p.idx) {
     d.list = p.idx + (long long)unit * p.idx_stride;
     d.count = min(__ldg(p.count + unit), p.idx_stride);
-  } else if (p.mid) {
-    const int* M = p.mid + (long long)unit * p.mid_stride;
-    const int nm = min(__ldg(p.n_mid + unit), p.mid_stride);
-    const int s0 = min(p.sinks, t);
-    const int vis_lo = max(s0, psaw_start(p.psaw_c, t));
-    const int wlo = max(max(t - p.window, 0), vis_lo);
+  } else if (p.set.star) {
+    int nm, mstride;
+    const int* M = middle_of(p.set, unit, &nm, &mstride);
+    const int s0 = min(p.set.sinks, t);
+    const int vis_lo = max(s0, psaw_start(p.set.psaw_c, t));
+    const int wlo = max(max(t - p.set.window, 0), vis_lo);
     int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && __ldg(M + min(lane, max(nm - 1, 0))) < vis_lo));
     const int i1 = nm - 32 + lane;
     int above = __popc(__ballot_sync(0xffffffffu, i1 >= 0 && __ldg(M + max(i1, 0)) >= wlo));
@@ -706,6 +702,7 @@ struct ScoreParams {
   int ld;
   float2* part_ml;        // [B][Hq][splits]
   int splits, num_q_heads, group_size;
+  const int* need;        // [B][Hq] or nullptr: score only KV heads with a query head that retrieves
   uint32_t* flags;
 };
 
@@ -714,6 +711,11 @@ __global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int gq = p.group_size;
   const int head0 = kvh * gq;
+  if (p.need != nullptr) {              // cosine-gated step: nothing to do if no head of the group retrieves
+    bool any = false;
+    for (int j = 0; j < gq; ++j) any |= __ldg(p.need + b * p.num_q_heads + head0 + j) != 0;
+    if (!any) return;
+  }
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;
   const int t = __ldg(p.kv.seq_lens + b);
@@ -842,6 +844,58 @@ __global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
     float mm = -INFINITY, ll = 0.f;
     for (int w = 0; w < kTWarps; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
     p.part_ml[((long long)b * p.num_q_heads + head0 + tid) * p.splits + split] = make_float2(mm, ll);
+  }
+}
+
+// ------------------------------------------------------------------- cosine gate (Eq. 9)
+// One warp per (b, h).  `pos` = step % s is the position of this step in its block.  At
+// pos == 0 the head retrieves into slot 0.  Later it shares the slot of the MOST RECENT earlier
+// step of the block whose query has cosine similarity > tau with the current one, or, if
+// there is none, retrieves into the next free slot (Sec. 4.1 "Similarity Criteria").
+// Updates the block history (queries, slot per position, number of sets) and writes the
+// decision: need (1 = retrieve now), slot (set to attend over), ref (position shared from, -1).
+__global__ void __launch_bounds__(128)
+gate_kernel(const __nv_bfloat16* __restrict__ q, int units, int pos, float tau, int slots,
+            __nv_bfloat16* __restrict__ qhist, int* __restrict__ set_of_pos, int* __restrict__ nsets,
+            int* __restrict__ need, int* __restrict__ slot_out, int* __restrict__ ref_out) {
+  const int unit = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (unit >= units) return;
+  const uint2 qx = *reinterpret_cast<const uint2*>(q + (long long)unit * kHeadDim + lane * 4);
+  const float q0 = bf_lo(qx.x), q1 = bf_hi(qx.x), q2 = bf_lo(qx.y), q3 = bf_hi(qx.y);
+  __nv_bfloat16* hist = qhist + (long long)unit * slots * kHeadDim;
+  int ref = -1;
+  if (pos > 0) {
+    float qq = q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) qq += __shfl_xor_sync(0xffffffffu, qq, off);
+    for (int j = pos - 1; j >= 0; --j) {
+      const uint2 ex = *reinterpret_cast<const uint2*>(hist + (long long)j * kHeadDim + lane * 4);
+      const float e0 = bf_lo(ex.x), e1 = bf_hi(ex.x), e2 = bf_lo(ex.y), e3 = bf_hi(ex.y);
+      float dot = q0 * e0 + q1 * e1 + q2 * e2 + q3 * e3;
+      float ee = e0 * e0 + e1 * e1 + e2 * e2 + e3 * e3;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        dot += __shfl_xor_sync(0xffffffffu, dot, off);
+        ee += __shfl_xor_sync(0xffffffffu, ee, off);
+      }
+      const float cs = dot / (sqrtf(qq) * sqrtf(ee));
+      if (cs > tau) { ref = j; break; }      // uniform over the warp
+    }
+  }
+  int slot;
+  if (ref >= 0) {
+    slot = set_of_pos[(long long)unit * slots + ref];
+  } else {
+    slot = pos == 0 ? 0 : min(nsets[unit], slots - 1);
+  }
+  *reinterpret_cast<uint2*>(hist + (long long)pos * kHeadDim + lane * 4) = qx;
+  if (lane == 0) {
+    if (ref < 0) nsets[unit] = slot + 1;
+    set_of_pos[(long long)unit * slots + pos] = slot;
+    need[unit] = ref < 0 ? 1 : 0;
+    slot_out[unit] = slot;
+    ref_out[unit] = ref;
   }
 }
 

@@ -44,6 +44,36 @@ __device__ __forceinline__ long long row_offset(const KvDev& kv, int b, int kvh,
   return (long long)b * kv.stride_outer + (long long)kvh * kv.stride_head + (long long)i * kHeadDim;
 }
 
+// Which stored middle set a (b, h) unit attends over.  Sets live in slots: [unit][slot][stride]
+// for S* (ascending) and for the dilated S^; a unit uses S* only on the step that retrieved
+// it (and not even then with PRHS_DILATE_ANCHOR), else S^ (Def. 3.2).
+struct SetRef {
+  const int* star;        // S* ascending, [U][slots][star_stride]; nullptr = no fused set
+  const int* n_star;      // [U][slots]
+  const int* hat;         // S^ ascending, [U][slots][hat_stride]
+  const int* n_hat;       // [U][slots]
+  const int* slot_of;     // [U] slot each unit uses this step, or nullptr = slot 0
+  const int* own_of;      // [U] != 0 where the unit retrieved this step, or nullptr = own_all
+  int star_stride, hat_stride, slots, own_all;
+  int sinks, window;
+  double psaw_c;          // sliding-window factor of this layer (0 = off)
+};
+
+// The unit's middle set M (ascending, unique) and its length.
+__device__ __forceinline__ const int* middle_of(const SetRef& r, int unit, int* n, int* stride) {
+  const int slot = r.slot_of ? __ldg(r.slot_of + unit) : 0;
+  const bool own = r.own_of ? (__ldg(r.own_of + unit) != 0) : (r.own_all != 0);
+  const long long e = (long long)unit * r.slots + slot;
+  if (own) {
+    *n = min(__ldg(r.n_star + e), r.star_stride);
+    *stride = r.star_stride;
+    return r.star + e * r.star_stride;
+  }
+  *n = min(__ldg(r.n_hat + e), r.hat_stride);
+  *stride = r.hat_stride;
+  return r.hat + e * r.hat_stride;
+}
+
 // Start of the progressive sliding attention window (Eq. 11): P = floor(c * t) with
 // c = 1 - phi^(alpha (l - l_s) / (N - l_s)) computed on the host in double (0 = no window).
 __device__ __forceinline__ int psaw_start(double c, int t) {

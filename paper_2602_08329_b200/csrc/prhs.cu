@@ -26,14 +26,8 @@ std::string g_create_error;
 
 }  // namespace
 
-// The list of a unit is given explicitly (idx/count), by the fused builder (mid/n_mid plus the
-// sink and window sizes) or, with both NULL, is every position (dense baseline).
-struct FusedSet {
-  const int* mid = nullptr;
-  const int* n_mid = nullptr;
-  int mid_stride = 0, sinks = 0, window = 0;
-  double psaw_c = 0.0;
-};
+// The list of a unit is given explicitly (idx/count), by the fused builder (a SetRef: stored
+// middle set plus the sink and window sizes) or, with neither, is every position (dense).
 
 // ---- scratch of the allocation-free entry point: split-K partials, merge tickets, flag word.
 // In host code the name is a stand-in, not a device address: set-up resolves it per device.
@@ -63,11 +57,18 @@ struct prhs_ctx {
   // shared-set state (device), per layer group
   int *sstar_desc = nullptr, *sstar_asc = nullptr, *shat_asc = nullptr;
   int *n_star = nullptr, *n_hat = nullptr, *anchor_t = nullptr;
+  // cosine gate (per layer group): block history and the decision of the latest step
+  int slots = 1;                    // sets kept per (b, h) and block (= max_block_sets)
+  __nv_bfloat16* qhist = nullptr;   // [G][U][slots][128] queries of the block so far
+  int *set_of_pos = nullptr;        // [G][U][slots] slot each step of the block attended over
+  int *nsets = nullptr;             // [G][U] sets retrieved so far in the block
+  int *g_need = nullptr, *g_slot = nullptr, *g_ref = nullptr;   // [G][U] decision of the latest step
+  std::vector<int> gate_step;       // host: step of each group's latest gate decision, -1 = never
   std::vector<int> anchor_step;     // host: step at which each group last retrieved, -1 = never
   // staging for the host-buffer entry point (device)
   __nv_bfloat16 *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_out = nullptr;
-  int last_batch = 0, last_layer_group = 1;
-  FusedSet last_set;                // what the last decode step attended over (for diagnostics)
+  int last_batch = 0, last_layer_group = 1, last_nchunks = 1;
+  SetRef last_set{};                // what the last decode step attended over (for diagnostics)
   const int* last_seq_lens = nullptr;
   long long launches = 0;
   // optional per-launch event timing
@@ -137,6 +138,8 @@ prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
     return fail(ctx, PRHS_ERR_CAPACITY, "schedule: layer_group below min_layer_group");
   if (s->top_k < 0 || s->window < 0 || s->sinks < 0 || s->dilate_r < 0 || s->dilate_m < -1)
     return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: negative budget");
+  if (!(s->sim_threshold <= 1.f))
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: sim_threshold must be <= 1 (<= -1 switches the gate off)");
   if (s->psaw_layer_start < 0 ||
       (s->psaw_layer_start > 0 && !(s->psaw_phi > 0.f && s->psaw_phi < 1.f && s->psaw_alpha >= 0.f)))
     return fail(ctx, PRHS_ERR_INVALID_ARG, "schedule: sliding window needs 0 < phi < 1, alpha >= 0, l_s >= 0");
@@ -185,7 +188,7 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
 
 // `sched` != nullptr: a retrieval pass (logits are written and the selection histogram filled).
 prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
-                         const prhs_schedule* sched, cudaStream_t st, int* nchunks_out) {
+                         const prhs_schedule* sched, const int* need, cudaStream_t st, int* nchunks_out) {
   const int write_scores = sched != nullptr;
   ScoreParams sp;
   sp.q = static_cast<const __nv_bfloat16*>(q);
@@ -196,19 +199,21 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_t);
   sp.num_q_heads = c->cfg.num_q_heads;
   sp.group_size = c->gq;
+  sp.need = need;
   sp.flags = c->flags;
   {
     LaunchScope ls(c, PRHS_KIND_SCORE, st);
     score_ring_kernel<<<dim3(sp.splits, c->cfg.num_kv_heads, batch), kTThreads, kSRSmemBytes, st>>>(sp);
   }
   const int nchunks = sp.splits;
+  c->last_nchunks = nchunks;
   *nchunks_out = nchunks;
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
 }
 
 prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
-                        int idx_stride, const FusedSet& fs, int max_count, int batch, void* out,
+                        int idx_stride, const SetRef& fs, int max_count, int batch, void* out,
                         float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st) {
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -216,12 +221,8 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.idx = idx;
   p.count = count;
   p.idx_stride = idx ? idx_stride : 0x7fffffff;
-  p.mid = idx ? nullptr : fs.mid;
-  p.n_mid = fs.n_mid;
-  p.mid_stride = fs.mid_stride;
-  p.sinks = fs.sinks;
-  p.window = fs.window;
-  p.psaw_c = fs.psaw_c;
+  p.set = fs;
+  if (idx) p.set.star = nullptr;
   p.num_q_heads = c->cfg.num_q_heads;
   p.group_size = c->gq;
   p.splits = pick_splits(c, batch * c->cfg.num_q_heads, max_count);
@@ -232,7 +233,7 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.lse_full = lse_full;
   p.out_delta = lse_full ? out_delta : nullptr;
   p.flags = c->flags;
-  if (!idx && !fs.mid) {
+  if (!idx && !fs.star) {
     // dense baseline: one CTA column per KV head, the group's heads share the K/V stream
     p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
     dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
@@ -257,16 +258,23 @@ double psaw_factor(const prhs_ctx* c, const prhs_schedule* s, int layer) {
   return 1.0 - std::pow((double)s->psaw_phi, expo);
 }
 
-size_t state_off(const prhs_ctx* c, int group, size_t per_unit) {
-  return (size_t)group * units_max(c) * per_unit;
+// Offset of a layer group's block in a state array with `per_slot` elements per (unit, slot).
+size_t state_off(const prhs_ctx* c, int group, size_t per_slot) {
+  return (size_t)group * units_max(c) * c->slots * per_slot;
 }
+// Offset of a layer group's block in a per-unit array (gate decisions, set counters).
+size_t unit_off(const prhs_ctx* c, int group) { return (size_t)group * units_max(c); }
 
+// `need` / `slot_of` (device, per unit) restrict the retrieval to the heads the cosine gate
+// sent here and name the slot of the new set; nullptr = every head, slot 0.  `score_all`
+// scores every head even so (the delta diagnostic wants every head's full log-sum-exp).
 prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const KvDev& kv, int max_t,
                          const prhs_schedule* s, int batch, int32_t* out_idx, int32_t* out_count,
-                         float* out_lse_full, cudaStream_t st) {
+                         float* out_lse_full, const int* need, const int* slot_of, bool score_all,
+                         cudaStream_t st) {
   const int g = group_of(s, layer);
   int nchunks = 1;
-  prhs_status rc = launch_score(c, q, kv, batch, max_t, s, st, &nchunks);
+  prhs_status rc = launch_score(c, q, kv, batch, max_t, s, score_all ? nullptr : need, st, &nchunks);
   if (rc != PRHS_OK) return rc;
   SelectParams p;
   p.scores = c->scores;
@@ -290,6 +298,9 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.shat_asc = c->shat_asc + state_off(c, g, c->shat_cap);
   p.n_star = c->n_star + state_off(c, g, 1);
   p.n_hat = c->n_hat + state_off(c, g, 1);
+  p.need = need;
+  p.slot_of = slot_of;
+  p.slots = c->slots;
   p.anchor_t = c->anchor_t + (size_t)g * c->cfg.max_batch;
   p.out_idx = out_idx;
   p.out_count = out_count;
@@ -302,35 +313,53 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
     select_kernel<<<batch * c->cfg.num_q_heads, kSelThreads, c->sel_smem, st>>>(p);
   }
   PRHS_CUDA(c, cudaGetLastError());
-  c->anchor_step[g] = step;
+  if (!need) c->anchor_step[g] = step;
   c->last_layer_group = s->layer_group;
   return PRHS_OK;
 }
 
-// The middle set (layer, step) attends over: S* for the retrieving call itself (unless
-// PRHS_DILATE_ANCHOR), else the dilated S^ of the group's anchor (Def. 3.2).
-prhs_status pick_middle(prhs_ctx* c, int layer, int step, const prhs_schedule* s, FusedSet* fs) {
+bool gated(const prhs_schedule* s) { return s->sim_threshold > -1.f; }
+
+// The middle set (layer, step) attends over: S* for the call that retrieved it (unless
+// PRHS_DILATE_ANCHOR), else the dilated S^ (Def. 3.2).  Fixed schedule: the block's first
+// step on the group's first layer retrieves into slot 0.  Cosine gate: the group's first
+// layer decided per head this step (need / slot), the other layers follow it.
+prhs_status pick_middle(prhs_ctx* c, int layer, int step, const prhs_schedule* s, SetRef* fs) {
   const int g = group_of(s, layer);
   const int anchor = step - step % s->refresh_interval;
-  if (c->anchor_step[g] != anchor)
-    return fail(c, PRHS_ERR_STATE, "no shared set for this block: the group's first layer has not retrieved");
-  const bool own = (layer % s->layer_group == 0) && (step == anchor) && !(s->flags & PRHS_DILATE_ANCHOR);
-  fs->mid = own ? c->sstar_asc + state_off(c, g, c->cfg.max_k) : c->shat_asc + state_off(c, g, c->shat_cap);
-  fs->n_mid = (own ? c->n_star : c->n_hat) + state_off(c, g, 1);
-  fs->mid_stride = own ? c->cfg.max_k : c->shat_cap;
+  const bool leader = layer % s->layer_group == 0;
+  if (gated(s)) {
+    if (c->gate_step[g] != step)
+      return fail(c, PRHS_ERR_STATE, "no gate decision for this step: the group's first layer has not been called");
+    fs->slot_of = c->g_slot + unit_off(c, g);
+    fs->own_of = (leader && !(s->flags & PRHS_DILATE_ANCHOR)) ? c->g_need + unit_off(c, g) : nullptr;
+    fs->own_all = 0;
+  } else {
+    if (c->anchor_step[g] != anchor)
+      return fail(c, PRHS_ERR_STATE, "no shared set for this block: the group's first layer has not retrieved");
+    fs->slot_of = nullptr;
+    fs->own_of = nullptr;
+    fs->own_all = (leader && step == anchor && !(s->flags & PRHS_DILATE_ANCHOR)) ? 1 : 0;
+  }
+  fs->star = c->sstar_asc + state_off(c, g, c->cfg.max_k);
+  fs->n_star = c->n_star + state_off(c, g, 1);
+  fs->hat = c->shat_asc + state_off(c, g, c->shat_cap);
+  fs->n_hat = c->n_hat + state_off(c, g, 1);
+  fs->star_stride = c->cfg.max_k;
+  fs->hat_stride = c->shat_cap;
+  fs->slots = c->slots;
   fs->sinks = s->sinks;
   fs->window = s->window;
   fs->psaw_c = psaw_factor(c, s, layer);
   return PRHS_OK;
 }
 
-prhs_status launch_build(prhs_ctx* c, const FusedSet& fs, const int* seq_lens, int batch, int32_t* out_idx,
+prhs_status launch_build(prhs_ctx* c, const SetRef& fs, const int* seq_lens, int batch, int32_t* out_idx,
                          int idx_stride, int32_t* out_count, cudaStream_t st) {
   {
     LaunchScope ls(c, PRHS_KIND_BUILD, st);
-    build_set_kernel<<<batch * c->cfg.num_q_heads, 128, 0, st>>>(
-        fs.mid, fs.n_mid, fs.mid_stride, seq_lens, fs.sinks, fs.window, fs.psaw_c, c->cfg.num_q_heads,
-        out_idx, idx_stride, out_count);
+    build_set_kernel<<<batch * c->cfg.num_q_heads, 128, 0, st>>>(fs, seq_lens, c->cfg.num_q_heads, out_idx,
+                                                                 idx_stride, out_count);
   }
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
@@ -366,7 +395,8 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     return fail(nullptr, PRHS_ERR_UNSUPPORTED, "page_size must be 0 or 16");
   if (cfg->num_layers < 1 || cfg->max_batch < 1 || cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 ||
       cfg->max_context < 1 || cfg->max_k < 0 || cfg->max_window < 0 || cfg->max_sinks < 0 ||
-      cfg->max_dilate_r < 0 || cfg->max_dilate_m < -1 || cfg->min_layer_group < 1)
+      cfg->max_dilate_r < 0 || cfg->max_dilate_m < -1 || cfg->min_layer_group < 1 ||
+      cfg->max_block_sets < 1 || cfg->max_block_sets > 64)
     return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: non-positive size");
   if (cfg->num_q_heads % cfg->num_kv_heads) return fail(nullptr, PRHS_ERR_INVALID_ARG, "Hkv must divide Hq");
   if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
@@ -387,6 +417,8 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   c->sort_cap <<= 1;   // room for a tie group that straddles the k-th place
   c->sort_cap = std::max(c->sort_cap, 64);   // the block sort works on 64-entry blocks
   c->anchor_step.assign(c->num_groups, -1);
+  c->gate_step.assign(c->num_groups, -1);
+  c->slots = cfg->max_block_sets;
 
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
@@ -427,11 +459,18 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->count, U);
   if (e == cudaSuccess) e = dev_alloc(&c->flags, 1);
   if (e == cudaSuccess) e = dev_alloc(&c->scratch_out, U * kHeadDim);
-  if (e == cudaSuccess) e = dev_alloc(&c->sstar_desc, G * U * cfg->max_k);
-  if (e == cudaSuccess) e = dev_alloc(&c->sstar_asc, G * U * cfg->max_k);
-  if (e == cudaSuccess) e = dev_alloc(&c->shat_asc, G * U * c->shat_cap);
-  if (e == cudaSuccess) e = dev_alloc(&c->n_star, G * U);
-  if (e == cudaSuccess) e = dev_alloc(&c->n_hat, G * U);
+  const size_t SL = (size_t)c->slots;
+  if (e == cudaSuccess) e = dev_alloc(&c->sstar_desc, G * U * SL * cfg->max_k);
+  if (e == cudaSuccess) e = dev_alloc(&c->sstar_asc, G * U * SL * cfg->max_k);
+  if (e == cudaSuccess) e = dev_alloc(&c->shat_asc, G * U * SL * c->shat_cap);
+  if (e == cudaSuccess) e = dev_alloc(&c->n_star, G * U * SL);
+  if (e == cudaSuccess) e = dev_alloc(&c->n_hat, G * U * SL);
+  if (e == cudaSuccess) e = dev_alloc(&c->qhist, G * U * SL * kHeadDim);
+  if (e == cudaSuccess) e = dev_alloc(&c->set_of_pos, G * U * SL);
+  if (e == cudaSuccess) e = dev_alloc(&c->nsets, G * U);
+  if (e == cudaSuccess) e = dev_alloc(&c->g_need, G * U);
+  if (e == cudaSuccess) e = dev_alloc(&c->g_slot, G * U);
+  if (e == cudaSuccess) e = dev_alloc(&c->g_ref, G * U);
   if (e == cudaSuccess) e = dev_alloc(&c->anchor_t, G * cfg->max_batch);
   if (e == cudaSuccess) e = dev_alloc(&c->st_q, U * kHeadDim);
   if (e == cudaSuccess) e = dev_alloc(&c->st_out, U * kHeadDim);
@@ -439,8 +478,13 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->st_v, (size_t)cfg->max_batch * cfg->num_kv_heads * kHeadDim);
   if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, U * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(c->flags, 0, sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMemset(c->n_star, 0, G * U * sizeof(int));
-  if (e == cudaSuccess) e = cudaMemset(c->n_hat, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->n_star, 0, G * U * SL * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->n_hat, 0, G * U * SL * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->set_of_pos, 0, G * U * SL * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->nsets, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->g_need, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->g_slot, 0, G * U * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->g_ref, 0xff, G * U * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->count, 0, U * sizeof(int));
   if (e != cudaSuccess) {
     std::string msg = std::string("prhs_create: ") + cudaGetErrorString(e);
@@ -457,7 +501,8 @@ prhs_status prhs_destroy(prhs_ctx* c) {
   if (!c) return PRHS_OK;
   void* ptrs[] = {c->scores, c->part_ml, c->lse_full, c->lse_c, c->partials, c->tickets, c->idx,
                   c->count, c->flags, c->scratch_out, c->sstar_desc, c->sstar_asc, c->shat_asc,
-                  c->n_star, c->n_hat, c->anchor_t, c->st_q, c->st_out, c->st_k, c->st_v};
+                  c->n_star, c->n_hat, c->anchor_t, c->qhist, c->set_of_pos, c->nsets, c->g_need,
+                  c->g_slot, c->g_ref, c->st_q, c->st_out, c->st_k, c->st_v};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   for (auto& r : c->prof) {
@@ -483,7 +528,7 @@ prhs_status prhs_score_topk(prhs_ctx* ctx, int32_t layer, int32_t step, const vo
   rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
   return do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, out_idx, out_count, out_lse_full,
-                      as_stream(stream));
+                      nullptr, nullptr, false, as_stream(stream));
 }
 
 prhs_status prhs_build_index_set(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
@@ -500,7 +545,7 @@ prhs_status prhs_build_index_set(prhs_ctx* ctx, int32_t layer, int32_t step, con
   int max_t;
   rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  FusedSet fs;
+  SetRef fs{};
   rc = pick_middle(ctx, layer, step, sched, &fs);
   if (rc != PRHS_OK) return rc;
   return launch_build(ctx, fs, dv.seq_lens, batch, out_idx, idx_stride, out_count, as_stream(stream));
@@ -516,7 +561,7 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
   int max_t;
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, out, out_lse,
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, SetRef{}, idx_stride, batch, out, out_lse,
                      nullptr, nullptr, as_stream(stream));
 }
 
@@ -586,12 +631,7 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
   p.idx = idx;
   p.count = count;
   p.idx_stride = idx_stride;
-  p.mid = nullptr;
-  p.n_mid = nullptr;
-  p.mid_stride = 0;
-  p.sinks = 0;
-  p.window = 0;
-  p.psaw_c = 0.0;
+  p.set = SetRef{};
   p.num_q_heads = num_q_heads;
   p.group_size = num_q_heads / num_kv_heads;
   p.splits = splits;
@@ -615,7 +655,7 @@ prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_v
   int max_t;
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
-  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, FusedSet(), max_t, batch, out, out_lse, nullptr,
+  return launch_attn(ctx, q, dv, nullptr, nullptr, 0, SetRef{}, max_t, batch, out, out_lse, nullptr,
                      nullptr, as_stream(stream));
 }
 
@@ -634,13 +674,51 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
   if (rc != PRHS_OK) return rc;
   cudaStream_t st = as_stream(stream);
   const bool want_delta = (sched->flags & PRHS_WANT_DELTA) && out_delta;
-  const bool retrieve = (layer % sched->layer_group == 0) && (step % sched->refresh_interval == 0);
-  if (retrieve) {
-    rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, st);
+  const bool leader = layer % sched->layer_group == 0;
+  const int g = group_of(sched, layer);
+  bool scored = false;                       // lse_full of every head is fresh
+  if (gated(sched)) {
+    // cosine gate (Eq. 9): the group's first layer decides per head, on the device, whether it
+    // shares or retrieves; scoring and selection are launched every step and skip the heads
+    // (and KV heads) that share
+    if (sched->refresh_interval > ctx->slots)
+      return fail(ctx, PRHS_ERR_CAPACITY, "cosine gate needs max_block_sets >= refresh_interval");
+    if (leader) {
+      const int units = batch * ctx->cfg.num_q_heads;
+      const int pos = step % sched->refresh_interval;
+      if (pos > 0 && ctx->gate_step[g] != step - 1)
+        return fail(ctx, PRHS_ERR_STATE, "cosine gate: the previous step of this block was not run");
+      int* need = ctx->g_need + unit_off(ctx, g);
+      int* slot = ctx->g_slot + unit_off(ctx, g);
+      {
+        LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+        gate_kernel<<<(units + 3) / 4, 128, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(q), units, pos, sched->sim_threshold, ctx->slots,
+            ctx->qhist + state_off(ctx, g, kHeadDim), ctx->set_of_pos + state_off(ctx, g, 1),
+            ctx->nsets + unit_off(ctx, g), need, slot, ctx->g_ref + unit_off(ctx, g));
+      }
+      PRHS_CUDA(ctx, cudaGetLastError());
+      ctx->gate_step[g] = step;
+      rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, need, slot,
+                        want_delta, st);
+      if (rc != PRHS_OK) return rc;
+      if (want_delta) {        // every head was scored; heads that share still need their lse_full
+        const int n = batch * ctx->cfg.num_q_heads;
+        LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+        lse_reduce_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctx->part_ml, ctx->last_nchunks, 0, dv.seq_lens,
+                                                           ctx->cfg.num_q_heads, ctx->lse_full, n);
+        scored = true;
+      }
+    }
+  } else if (leader && step % sched->refresh_interval == 0) {
+    rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, nullptr, nullptr,
+                      false, st);
     if (rc != PRHS_OK) return rc;
-  } else if (want_delta) {
+    scored = true;
+  }
+  if (want_delta && !scored) {
     int nchunks = 1;
-    rc = launch_score(ctx, q, dv, batch, max_t, nullptr, st, &nchunks);
+    rc = launch_score(ctx, q, dv, batch, max_t, nullptr, nullptr, st, &nchunks);
     if (rc != PRHS_OK) return rc;
     const int n = batch * ctx->cfg.num_q_heads;
     {
@@ -651,7 +729,7 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
     PRHS_CUDA(ctx, cudaGetLastError());
   }
   // the index set is built inside the attention kernel from the stored middle set
-  FusedSet fs;
+  SetRef fs{};
   rc = pick_middle(ctx, layer, step, sched, &fs);
   if (rc != PRHS_OK) return rc;
   ctx->last_set = fs;
@@ -708,7 +786,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
   if (rc != PRHS_OK) return rc;
   cudaStream_t st = as_stream(stream);
   int nchunks = 1;
-  rc = launch_score(ctx, q, dv, batch, max_t, nullptr, st, &nchunks);
+  rc = launch_score(ctx, q, dv, batch, max_t, nullptr, nullptr, st, &nchunks);
   if (rc != PRHS_OK) return rc;
   const int n = batch * ctx->cfg.num_q_heads;
   {
@@ -717,7 +795,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
                                                          ctx->cfg.num_q_heads, ctx->lse_full, n);
   }
   PRHS_CUDA(ctx, cudaGetLastError());
-  return launch_attn(ctx, q, dv, idx, count, idx_stride, FusedSet(), idx_stride, batch, ctx->scratch_out,
+  return launch_attn(ctx, q, dv, idx, count, idx_stride, SetRef{}, idx_stride, batch, ctx->scratch_out,
                      ctx->lse_c, ctx->lse_full, out_delta, st);
 }
 
@@ -727,7 +805,7 @@ prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx, 
   if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
   cudaStream_t st = as_stream(stream);
   const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
-  if (!ctx->last_set.mid || batch != ctx->last_batch)
+  if (!ctx->last_set.star || batch != ctx->last_batch)
     return fail(ctx, PRHS_ERR_STATE, "no decode step to report (or a different batch)");
   prhs_status rc = launch_build(ctx, ctx->last_set, ctx->last_seq_lens, batch, ctx->idx, ctx->idx_cap,
                                 ctx->count, st);
@@ -750,17 +828,47 @@ prhs_status prhs_get_shared_set(prhs_ctx* ctx, int32_t layer, int32_t batch, int
   if (layer < 0 || g >= ctx->num_groups) return fail(ctx, PRHS_ERR_INVALID_ARG, "layer out of range");
   cudaStream_t st = as_stream(stream);
   const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
-  if (host_s_star)
-    PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_star, ctx->sstar_desc + state_off(ctx, g, ctx->cfg.max_k),
-                                   n * ctx->cfg.max_k * sizeof(int), cudaMemcpyDeviceToHost, st));
-  if (host_n_star)
-    PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_star, ctx->n_star + state_off(ctx, g, 1), n * sizeof(int),
+  // the slot each unit used in the group's latest step (slot 0 without the cosine gate)
+  std::vector<int> slot(n, 0);
+  if (ctx->slots > 1 && ctx->gate_step[g] >= 0) {
+    PRHS_CUDA(ctx, cudaMemcpyAsync(slot.data(), ctx->g_slot + unit_off(ctx, g), n * sizeof(int),
                                    cudaMemcpyDeviceToHost, st));
-  if (host_s_hat)
-    PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_hat, ctx->shat_asc + state_off(ctx, g, ctx->shat_cap),
-                                   n * ctx->shat_cap * sizeof(int), cudaMemcpyDeviceToHost, st));
-  if (host_n_hat)
-    PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_hat, ctx->n_hat + state_off(ctx, g, 1), n * sizeof(int),
+    PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  }
+  const size_t mk = ctx->cfg.max_k, hc = ctx->shat_cap, SL = ctx->slots;
+  for (size_t u = 0; u < n; ++u) {
+    const size_t e = u * SL + (size_t)slot[u];
+    if (host_s_star)
+      PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_star + u * mk, ctx->sstar_desc + state_off(ctx, g, mk) + e * mk,
+                                     mk * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (host_n_star)
+      PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_star + u, ctx->n_star + state_off(ctx, g, 1) + e, sizeof(int),
+                                     cudaMemcpyDeviceToHost, st));
+    if (host_s_hat)
+      PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_hat + u * hc, ctx->shat_asc + state_off(ctx, g, hc) + e * hc,
+                                     hc * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (host_n_hat)
+      PRHS_CUDA(ctx, cudaMemcpyAsync(host_n_hat + u, ctx->n_hat + state_off(ctx, g, 1) + e, sizeof(int),
+                                     cudaMemcpyDeviceToHost, st));
+  }
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+prhs_status prhs_get_gate(prhs_ctx* ctx, int32_t layer, int32_t batch, int32_t* host_need,
+                          int32_t* host_ref, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  const int g = layer / ctx->last_layer_group;
+  if (layer < 0 || g >= ctx->num_groups) return fail(ctx, PRHS_ERR_INVALID_ARG, "layer out of range");
+  if (ctx->gate_step[g] < 0) return fail(ctx, PRHS_ERR_STATE, "no gated step has run for this layer group");
+  cudaStream_t st = as_stream(stream);
+  const size_t n = (size_t)batch * ctx->cfg.num_q_heads;
+  if (host_need)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_need, ctx->g_need + unit_off(ctx, g), n * sizeof(int),
+                                   cudaMemcpyDeviceToHost, st));
+  if (host_ref)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_ref, ctx->g_ref + unit_off(ctx, g), n * sizeof(int),
                                    cudaMemcpyDeviceToHost, st));
   PRHS_CUDA(ctx, cudaStreamSynchronize(st));
   return PRHS_OK;

@@ -34,11 +34,14 @@ struct SelectParams {
   int k, sinks, window, r, m;
   double psaw_c;            // sliding-window factor of this layer (0 = off)
   int max_k, shat_cap, num_q_heads;
-  int* sstar_desc;          // [B][Hq][max_k]
-  int* sstar_asc;           // [B][Hq][max_k]
-  int* shat_asc;            // [B][Hq][shat_cap]
-  int* n_star;              // [B][Hq]
-  int* n_hat;               // [B][Hq]
+  int* sstar_desc;          // [B][Hq][slots][max_k]
+  int* sstar_asc;           // [B][Hq][slots][max_k]
+  int* shat_asc;            // [B][Hq][slots][shat_cap]
+  int* n_star;              // [B][Hq][slots]
+  int* n_hat;               // [B][Hq][slots]
+  const int* need;          // [B][Hq] or nullptr: only units with need != 0 select (cosine gate)
+  const int* slot_of;       // [B][Hq] or nullptr (slot 0): where the new set goes
+  int slots;
   int* anchor_t;            // [B]: t_b at this retrieval
   int* out_idx;             // optional [B][Hq][max_k]
   int* out_count;           // optional
@@ -214,6 +217,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x;
+  if (p.need != nullptr && __ldg(p.need + unit) == 0) return;     // this head shares: no retrieval
+  const long long sunit = (long long)unit * p.slots + (p.slot_of ? __ldg(p.slot_of + unit) : 0);
   const int b = unit / p.num_q_heads;
   const int t = __ldg(p.seq_lens + b);
   int k = p.k_per_seq ? __ldg(p.k_per_seq + b) : p.k;
@@ -434,14 +439,14 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   block_sort_desc(wbuf, P);
 
   // ---- S* in descending-logit order
-  int* sd = p.sstar_desc + (long long)unit * p.max_k;
+  int* sd = p.sstar_desc + sunit * p.max_k;
   for (int e = tid; e < p.max_k; e += kSelThreads) {
     const int v = e < kk ? (int)(0xffffffffu - (uint32_t)(wbuf[e] & 0xffffffffull)) : -1;
     sd[e] = v;
     if (p.out_idx) p.out_idx[(long long)unit * p.max_k + e] = v;
   }
   if (tid == 0) {
-    p.n_star[unit] = kk;
+    p.n_star[sunit] = kk;
     if (p.out_count) p.out_count[unit] = kk;
   }
 
@@ -454,7 +459,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
     atomicOr(&bm[pos >> 5], 1u << (pos & 31u));
   }
   __syncthreads();
-  compact_bitmap(bm, words, p.sstar_asc + (long long)unit * p.max_k, p.max_k, misc + 8);
+  compact_bitmap(bm, words, p.sstar_asc + sunit * p.max_k, p.max_k, misc + 8);
   __syncthreads();   // every thread has finished reading the bitmap before it grows
   for (int e = tid; e < m_eff; e += kSelThreads) {
     const int pos = (int)(0xffffffffu - (uint32_t)(wbuf[e] & 0xffffffffull));
@@ -464,9 +469,9 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
     }
   }
   __syncthreads();
-  const int nh = compact_bitmap(bm, words, p.shat_asc + (long long)unit * p.shat_cap, p.shat_cap,
+  const int nh = compact_bitmap(bm, words, p.shat_asc + sunit * p.shat_cap, p.shat_cap,
                                 misc + 8);
-  if (tid == 0) p.n_hat[unit] = min(nh, p.shat_cap);
+  if (tid == 0) p.n_hat[sunit] = min(nh, p.shat_cap);
 }
 
 }  // namespace prhs

@@ -62,6 +62,7 @@ class Workload:
     psaw_layer_start: int = 0   # l_s of the sliding attention window (1-based); 0 = off
     psaw_phi: float = 0.7
     psaw_alpha: float = 1.0
+    sim_threshold: float | None = None   # tau of the cosine gate; None = fixed sharing schedule
 
     @property
     def capacity(self) -> int:

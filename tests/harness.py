@@ -20,6 +20,7 @@ from paper_2602_08329_b200 import workloads as W
 Y_TOL = 2e-2
 DELTA_TOL = 1e-4
 TIE_REL = 1e-3
+SIM_TOL = 1e-4          # a cosine similarity this close to tau may fall either way (fp32 vs float64)
 
 
 def np32(t: torch.Tensor) -> np.ndarray:
@@ -55,7 +56,8 @@ def make_ctx(w: W.Workload, **over):
     kw = dict(num_layers=w.layers, max_batch=w.batch, num_q_heads=w.q_heads, num_kv_heads=w.kv_heads,
               max_context=w.capacity, max_k=max(w.top_k, int(w.k_frac * w.context)),
               max_window=w.window, max_sinks=w.sinks, max_dilate_r=max(w.dilate_r, 1), max_dilate_m=-1,
-              page_size=w.page_size, min_layer_group=w.layer_group)
+              page_size=w.page_size, min_layer_group=w.layer_group,
+              max_block_sets=w.refresh if w.sim_threshold is not None else 1)
     kw.update(over)
     return P.Context(**kw)
 
@@ -66,7 +68,8 @@ def make_sched(w: W.Workload, device, flags=0, **over):
     kw = dict(top_k=w.top_k, window=w.window, sinks=w.sinks, refresh_interval=w.refresh,
               layer_group=w.layer_group, dilate_r=w.dilate_r, dilate_m=-1, top_k_per_seq=kps_dev,
               flags=flags, psaw_phi=w.psaw_phi, psaw_alpha=w.psaw_alpha,
-              psaw_layer_start=w.psaw_layer_start)
+              psaw_layer_start=w.psaw_layer_start,
+              sim_threshold=-1.0 if w.sim_threshold is None else w.sim_threshold)
     kw.update(over)
     return P.make_schedule(**kw)
 
@@ -78,7 +81,8 @@ def oracle_sched(w: W.Workload, **over) -> O.Schedule:
               top_k_per_seq=None if kps is None else kps.numpy(),
               # the C ABI carries phi and alpha as fp32: give the oracle the same values
               psaw_phi=float(np.float32(w.psaw_phi)), psaw_alpha=float(np.float32(w.psaw_alpha)),
-              psaw_layer_start=w.psaw_layer_start, num_layers=w.layers)
+              psaw_layer_start=w.psaw_layer_start, num_layers=w.layers,
+              sim_threshold=None if w.sim_threshold is None else float(np.float32(w.sim_threshold)))
     kw.update(over)
     return O.Schedule(**kw)
 
@@ -157,15 +161,42 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
             assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
             stats["select_fallback"] = stats["select_fallback"] or bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK)
             y_gpu, d_gpu = np32(out), np32(dlt)
-            retrieve = orc.is_retrieval(l, n)
+            gated = w.sim_threshold is not None
+            leader = l % w.layer_group == 0
+            qh = np32(q)
+            Ks, Vs = _HostSlices(host, ("k", l), k_l), _HostSlices(host, ("v", l), v_l)
+            # which units retrieved: the fixed schedule, or the cosine gate's decision on the device
+            over_ref = {}
+            if gated and leader:
+                need, gref = ctx.get_gate(l, B)
+                retr = {u: bool(need[u[0], u[1]]) for u in units}
+                pos = n % w.refresh
+                if pos > 0:
+                    tau = osched.sim_threshold
+                    for (b, h) in units:
+                        blk = orc.blocks[(l // w.layer_group, b, h)]
+                        want_ref, sims = O.gate_decision(qh[b, h], blk.queries, tau)
+                        got_ref = int(gref[b, h])
+                        where = f"layer {l} step {n} unit ({b},{h})"
+                        assert -1 <= got_ref < pos and (got_ref < 0) == retr[(b, h)], where
+                        if got_ref != want_ref:       # only similarities within rounding of tau may differ
+                            assert all(sims[j] <= tau + SIM_TOL for j in range(got_ref + 1, pos)), where
+                            assert got_ref < 0 or sims[got_ref] > tau - SIM_TOL, where
+                            stats["near_tie_sets"] += 1
+                        over_ref[(b, h)] = got_ref
+            elif gated:
+                retr = {u: False for u in units}
+            else:
+                retr = {u: orc.is_retrieval(l, n) for u in units}
+            retrieve = any(retr.values())
             if retrieve:
                 s_star, n_star, s_hat, n_hat = ctx.get_shared_set(l, B)
                 scores = ctx.get_scores(B) if check_scores else None
-            qh = np32(q)
-            Ks, Vs = _HostSlices(host, ("k", l), k_l), _HostSlices(host, ("v", l), v_l)
             over_s = {}
             if retrieve:
                 for (b, h) in units:
+                    if not retr[(b, h)]:
+                        continue
                     t = int(t_host[b])
                     where = f"layer {l} step {n} unit ({b},{h})"
                     a = O.dense_scores(qh[b, h], Ks[b, h // gq], t)
@@ -180,12 +211,12 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                         assert np.allclose(sg, a32, atol=1e-4, rtol=1e-5), f"{where}: logits differ"
                     over_s[(b, h)] = got          # legal: the oracle adopts it
             ref = orc.decode_step(l, n, qh, Ks, Vs, t_host.numpy(), units=units, want_delta=want_delta,
-                                  override_s_star=over_s)
+                                  override_s_star=over_s, override_ref=over_ref)
             for (b, h) in units:
                 t = int(t_host[b])
                 where = f"layer {l} step {n} unit ({b},{h})"
-                assert ref["retrieved"][(b, h)] == retrieve, where
-                if retrieve:
+                assert ref["retrieved"][(b, h)] == retr[(b, h)], where
+                if retr[(b, h)]:
                     got_hat = s_hat[b, h, : int(n_hat[b, h])].numpy().astype(np.int64)
                     assert np.array_equal(got_hat, ref["s_hat"][(b, h)]), f"{where}: dilated set differs"
                     stats["retrievals"] += 1

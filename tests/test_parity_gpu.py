@@ -285,6 +285,28 @@ def test_schedule_with_sliding_window(cuda_device, phi, alpha, ls):
     assert min(st["set_sizes"]) < max(st["set_sizes"])         # deeper layers attend over fewer rows
 
 
+@pytest.mark.parametrize("tau,sigma", [(0.8, 0.7), (0.95, 0.3), (-0.5, 1.5), (0.999, 0.05)])
+def test_schedule_with_cosine_gate(cuda_device, tau, sigma):
+    # per-head sharing decisions on the device: some heads retrieve, others share, inside one
+    # launch; followers (second layer of each group) follow their leader's decision
+    w = small(layers=4, layer_group=2, steps=9, refresh=4, q_heads=8, kv_heads=2, context=2300, seed=15,
+              sigma=sigma, sim_threshold=tau)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w))
+    assert st["checked"] == 4 * 9 * w.batch * w.q_heads
+    leaders_heads = 2 * w.batch * w.q_heads
+    assert st["retrievals"] >= 3 * leaders_heads          # steps 0, 4 and 8 always retrieve
+    if (tau, sigma) == (0.8, 0.7):
+        assert 3 * leaders_heads < st["retrievals"] < 9 * leaders_heads    # a real mix
+
+
+def test_cosine_gate_gqa_paged_with_window(cuda_device):
+    w = small(layers=2, layer_group=1, steps=6, refresh=3, batch=3, q_heads=8, kv_heads=1, context=2100,
+              min_context=500, page_size=16, top_k=0, k_frac=0.03, seed=16, sigma=0.6, sim_threshold=0.85,
+              psaw_layer_start=1, psaw_phi=0.8)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=True)
+    assert st["checked"] == 2 * 6 * w.batch * w.q_heads
+
+
 def test_schedule_paged_and_ragged(cuda_device):
     w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=5, q_heads=8, kv_heads=2,
               context=3000, min_context=300, page_size=16, top_k=0, k_frac=0.03, seed=13)
