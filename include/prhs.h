@@ -85,7 +85,9 @@ typedef struct {
   const int32_t* page_table; /* device [B][page_table_stride] or NULL */
   int32_t page_table_stride;
   const int32_t* seq_lens;   /* device [B]: t_b, current token included; 0 <= t_b <= max_seq_len */
-  int32_t max_seq_len;       /* host-side upper bound of every t_b (sizes the launch); 0 = max_context */
+  int32_t max_seq_len;       /* host-side upper bound of every t_b (sizes the launch); 0 = max_context.
+                                The cache must hold max_seq_len positions per (b, kvh): tiled copies
+                                may read rows in [t_b, max_seq_len) and ignore them */
   int32_t num_pages;         /* paged: pages in the pool (bounds check); contiguous: ignored */
 } prhs_kv_view;
 
@@ -271,6 +273,7 @@ int32_t prhs_scores_ld(const prhs_ctx* ctx);
 #define PRHS_FLAG_BAD_INDEX       1u /* an index outside [0, t_b) was skipped                */
 #define PRHS_FLAG_BAD_PAGE        2u /* a page id outside [0, num_pages) was skipped          */
 #define PRHS_FLAG_SELECT_FALLBACK 4u /* informational: selection took the multi-pass path     */
+#define PRHS_FLAG_TIMEOUT         8u /* a bounded wait on a TMA barrier ran out; results invalid */
 prhs_status prhs_check(prhs_ctx* ctx, void* stream, uint32_t* out_flags);
 
 /* Per-kernel device timing for benchmarks (no counterpart in the paper: measurement support).

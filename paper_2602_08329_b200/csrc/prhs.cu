@@ -12,6 +12,7 @@
 
 #include "attn.cuh"
 #include "common.cuh"
+#include "score_tma.cuh"
 #include "select.cuh"
 
 using namespace prhs;
@@ -68,6 +69,8 @@ struct prhs_ctx {
   // staging for the host-buffer entry point (device)
   __nv_bfloat16 *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_out = nullptr;
   int last_batch = 0, last_layer_group = 1, last_nchunks = 1;
+  // cuTensorMapEncodeTiled, resolved at run time (no link against libcuda); nullptr = no TMA path
+  void* encode_tiled = nullptr;
   SetRef last_set{};                // what the last decode step attended over (for diagnostics)
   const int* last_seq_lens = nullptr;
   long long launches = 0;
@@ -201,7 +204,36 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.group_size = c->gq;
   sp.need = need;
   sp.flags = c->flags;
-  {
+  bool tma_done = false;
+  if (c->encode_tiled && kv.page_table == nullptr) {
+    // K as a 2-D tensor [rows][128] bf16; rows past the last sequence's max length are out of
+    // bounds for the copy engine (zero fill), rows in between belong to the cache
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    const unsigned long long outer_rows = (unsigned long long)(kv.stride_outer >> 7);
+    const unsigned long long head_rows = (unsigned long long)(kv.stride_head >> 7);
+    const unsigned long long rows_total =
+        (unsigned long long)(batch - 1) * outer_rows + (unsigned long long)(c->cfg.num_kv_heads - 1) * head_rows +
+        (unsigned long long)max_t;
+    if (rows_total < (1ull << 31)) {
+      alignas(64) CUtensorMap tm;
+      const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows_total};
+      const cuuint64_t gstr[1] = {(cuuint64_t)kRowBytes};
+      const cuuint32_t box[2] = {64u, (cuuint32_t)kSTStageRows};
+      const cuuint32_t estr[2] = {1u, 1u};
+      const CUresult cr = reinterpret_cast<EncodeFn>(c->encode_tiled)(
+          &tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(kv.k), gdim, gstr, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (cr == CUDA_SUCCESS) {
+        LaunchScope ls(c, PRHS_KIND_SCORE, st);
+        score_tma_kernel<<<dim3(sp.splits, c->cfg.num_kv_heads, batch), kSTThreads, kSTSmemBytes, st>>>(tm, sp);
+        tma_done = true;
+      }
+    }
+  }
+  if (!tma_done) {
     LaunchScope ls(c, PRHS_KIND_SCORE, st);
     score_ring_kernel<<<dim3(sp.splits, c->cfg.num_kv_heads, batch), kTThreads, kSRSmemBytes, st>>>(sp);
   }
@@ -438,6 +470,17 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
+  if (e == cudaSuccess) {
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      c->encode_tiled = fn;
+    else
+      cudaGetLastError();      // no TMA path: the cp.async ring kernel serves every layout
+  }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSRSmemBytes);
   if (e == cudaSuccess)
@@ -943,7 +986,7 @@ prhs_status prhs_check(prhs_ctx* ctx, void* stream, uint32_t* out_flags) {
     PRHS_CUDA(ctx, cudaMemsetAsync(ctx->flags, 0, sizeof(uint32_t), st));
     PRHS_CUDA(ctx, cudaStreamSynchronize(st));
   }
-  if (f & (PRHS_FLAG_BAD_INDEX | PRHS_FLAG_BAD_PAGE)) {
+  if (f & (PRHS_FLAG_BAD_INDEX | PRHS_FLAG_BAD_PAGE | PRHS_FLAG_TIMEOUT)) {
     char buf[96];
     snprintf(buf, sizeof buf, "device flag word 0x%x", f);
     return fail(ctx, PRHS_ERR_DEVICE_FLAG, buf);

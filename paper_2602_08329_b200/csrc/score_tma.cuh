@@ -1,0 +1,222 @@
+// Retrieval scoring with the K stream staged by TMA (contiguous caches).
+//
+// Logits a_i = q . k_i / sqrt(d) for all i < t (Eq. 2), as in score_ring_kernel, but the K
+// tiles are brought into shared memory by the tensor memory accelerator: one elected thread
+// issues two `cp.async.bulk.tensor.2d` copies per 64-key stage (a [64 rows][64 columns] box for
+// each half of the 128 dimensions, 128-byte swizzle so that ldmatrix reads are conflict-free),
+// completion is signalled on an mbarrier, and four consumer warps (16 keys each) run the
+// m16n8k16 MMAs for all heads of the KV group.  A six-stage ring keeps up to 80 KB in flight
+// per CTA with no address arithmetic in the consumer warps.
+//
+// Every wait on an mbarrier is bounded: a wait that exceeds its budget records
+// kFlagTimeout and the CTA drains and returns, so a wrong descriptor cannot hang the GPU.
+#pragma once
+#include <cuda.h>
+
+#include "attn.cuh"
+#include "common.cuh"
+
+namespace prhs {
+
+constexpr int kSTConsumers = 4;                         // consumer warps
+constexpr int kSTThreads = (kSTConsumers + 1) * 32;     // + one producer warp
+constexpr int kSTStageRows = 64;                        // keys per stage
+constexpr int kSTHalfBytes = kSTStageRows * 128;        // one [64][64] bf16 box = 8 KB
+constexpr int kSTStageBytes = 2 * kSTHalfBytes;         // 16 KB
+constexpr int kSTStages = 6;
+constexpr int kSTSmemBytes = kSTStages * kSTStageBytes + 1024;   // + slack to align to 1 KB
+constexpr uint32_t kFlagTimeout = 8u;
+constexpr long long kWaitBudgetCycles = 4000000000ll;   // about two seconds
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait: false if the phase did not complete within the cycle budget, or if another
+// thread of the CTA has already given up (*abort != 0).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (*abort || clock64() - t0 > kWaitBudgetCycles) return false;
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+// grid (splits, Hkv, B).  tm_k: K viewed as [rows][128] bf16 (row pitch 256 B), box [64][64],
+// 128-byte swizzle; row of (b, kvh, i) = b * outer_rows + kvh * head_rows + i.
+__global__ void __launch_bounds__(kSTThreads)
+score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+  extern __shared__ unsigned char st_smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * kSTStages];     // full[0..NS), empty[NS..2NS)
+  __shared__ float sm_m[kSTConsumers][16], sm_l[kSTConsumers][16];
+  __shared__ int sh_abort;
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int gq = p.group_size;
+  const int head0 = kvh * gq;
+  if (p.need != nullptr) {
+    bool any = false;
+    for (int j = 0; j < gq; ++j) any |= __ldg(p.need + b * p.num_q_heads + head0 + j) != 0;
+    if (!any) return;
+  }
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  const int t = __ldg(p.kv.seq_lens + b);
+  int per = (t + p.splits - 1) / p.splits;
+  per = (per + kSTStageRows - 1) & ~(kSTStageRows - 1);
+  const int start = min(split * per, t);
+  const int end = min(start + per, t);
+  const int nstages = (end - start + kSTStageRows - 1) / kSTStageRows;
+  const uint32_t smem0 = ((uint32_t)__cvta_generic_to_shared(st_smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+  const int row_base = b * (int)(p.kv.stride_outer >> 7) + kvh * (int)(p.kv.stride_head >> 7) + start;
+
+  if (tid == 0) {
+    for (int s = 0; s < kSTStages; ++s) {
+      mbar_init(bar0 + 8 * s, 1);                          // full: the producer's expect_tx arrive
+      mbar_init(bar0 + 8 * (kSTStages + s), kSTConsumers); // empty: one arrive per consumer warp
+    }
+    sh_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == kSTConsumers) {
+    // ---------------- producer: one elected lane feeds the ring
+    if (lane == 0) {
+      for (int j = 0; j < nstages; ++j) {
+        const int slot = j % kSTStages;
+        if (j >= kSTStages && !mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort)) {
+          atomicOr(p.flags, kFlagTimeout);
+          sh_abort = 1;
+          break;
+        }
+        if (*(volatile int*)&sh_abort) break;
+        const uint32_t full = bar0 + 8 * slot;
+        const uint32_t dst = smem0 + slot * kSTStageBytes;
+        mbar_expect_tx(full, kSTStageBytes);
+        tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full);
+        tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full);
+      }
+    }
+  } else {
+    // ---------------- consumers: 16 keys of every stage per warp
+    const bool has0 = g < gq, has1 = g + 8 < gq;
+    uint32_t aq[8][4];
+    {
+      const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + ((long long)b * p.num_q_heads + head0 + g) * kHeadDim);
+      const uint32_t* q1 = q0 + 8 * (kHeadDim / 2);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        aq[ks][0] = has0 ? __ldg(q0 + ks * 8 + tg) : 0u;
+        aq[ks][1] = has1 ? __ldg(q1 + ks * 8 + tg) : 0u;
+        aq[ks][2] = has0 ? __ldg(q0 + ks * 8 + 4 + tg) : 0u;
+        aq[ks][3] = has1 ? __ldg(q1 + ks * 8 + 4 + tg) : 0u;
+      }
+    }
+    float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+    const int lm_mi = lane >> 3, lm_r = lane & 7;
+    for (int j = 0; j < nstages; ++j) {
+      const int slot = j % kSTStages;
+      // every lane polls; the verdict is made uniform so that the warp leaves the loop together
+      if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8 * slot, (j / kSTStages) & 1, &sh_abort))) {
+        if (lane == 0) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; }
+        break;
+      }
+      const uint32_t kt = smem0 + slot * kSTStageBytes;
+      const int pos0 = start + j * kSTStageRows + warp * 16;
+      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+      for (int pp = 0; pp < 4; ++pp) {
+        // logical 16-byte chunk 4pp + lm_mi of the 256-byte row: half = chunk / 8, c = chunk % 8
+        const int chunk = 4 * pp + lm_mi;
+        const uint32_t hb = kt + (chunk >> 3) * kSTHalfBytes + (((chunk & 7) ^ lm_r) << 4);
+        uint32_t bk0[4], bk1[4];
+        ldmatrix_x4(bk0, hb + (warp * 16 + lm_r) * 128);
+        ldmatrix_x4(bk1, hb + (warp * 16 + 8 + lm_r) * 128);
+        mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
+        mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
+        mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
+        mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
+      }
+      // the tile has been read into registers: hand the slot back to the producer
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar0 + 8 * (kSTStages + slot));
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        if (hh == 0 ? has0 : has1) {
+          float& m = hh == 0 ? m0 : m1;
+          float& l = hh == 0 ? l0 : l1;
+          float* dst = p.scores ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            const int key0 = pos0 + 8 * nt + 2 * tg;
+            const float s0 = s[nt][2 * hh] * kScale, s1 = s[nt][2 * hh + 1] * kScale;
+            if (key0 + 1 < end) {
+              if (dst) *reinterpret_cast<float2*>(dst + key0) = make_float2(s0, s1);
+              const float x0 = s0 * kLog2e, x1 = s1 * kLog2e;
+              const float mn = fmaxf(m, fmaxf(x0, x1));
+              l = l * exp2f(m - mn) + exp2f(x0 - mn) + exp2f(x1 - mn);
+              m = mn;
+            } else if (key0 < end) {
+              if (dst) dst[key0] = s0;
+              const float x0 = s0 * kLog2e;
+              const float mn = fmaxf(m, x0);
+              l = l * exp2f(m - mn) + exp2f(x0 - mn);
+              m = mn;
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+      float m2 = __shfl_xor_sync(0xffffffffu, m0, off), l2 = __shfl_xor_sync(0xffffffffu, l0, off);
+      ml_combine(m0, l0, m2, l2);
+      m2 = __shfl_xor_sync(0xffffffffu, m1, off);
+      l2 = __shfl_xor_sync(0xffffffffu, l1, off);
+      ml_combine(m1, l1, m2, l2);
+    }
+    if (tg == 0) {
+      sm_m[warp][g] = m0; sm_l[warp][g] = l0;
+      sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1;
+    }
+  }
+  __syncthreads();
+  if (tid < gq) {
+    float mm = -INFINITY, ll = 0.f;
+    for (int w = 0; w < kSTConsumers; ++w) ml_combine(mm, ll, sm_m[w][tid], sm_l[w][tid]);
+    p.part_ml[((long long)b * p.num_q_heads + head0 + tid) * p.splits + split] = make_float2(mm, ll);
+  }
+  // After an aborted wait some copies may still be in flight towards this CTA's shared
+  // memory: give each full barrier one more bounded wait before the CTA returns.
+  if (sh_abort && tid == 0) {
+    for (int s = 0; s < kSTStages; ++s) {
+      const long long t0 = clock64();
+      while (!mbar_try_wait(bar0 + 8 * s, 0) && !mbar_try_wait(bar0 + 8 * s, 1))
+        if (clock64() - t0 > kWaitBudgetCycles / 8) break;
+    }
+  }
+}
+
+}  // namespace prhs
