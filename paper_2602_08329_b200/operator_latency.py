@@ -1,7 +1,7 @@
 """Attention-operator latency of the library on the shapes of the paper's efficiency study.
 
     python -m paper_2602_08329_b200.operator_latency            # Table-3 shapes
-    python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C4 shapes
+    python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C5 shapes
 
 The paper (Sec. 5.4, Table 3) times one attention layer of LLaMA-2-7B-Chat (32 MHA heads,
 head_dim 128) in decode at batch 8 / 16 and 1k-4k cached tokens, token sparsity 1/8, block
@@ -32,19 +32,28 @@ PAPER_TABLE3_MS = {  # (batch, seqlen): (Flash, CPE-8, CPE-16) in ms on an A100 
 def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6):
     """Median device time (us) of a dense step, a retrieval step and a sharing step."""
     w = w.scaled(layers=copies, steps=max(w.refresh, 2) + 1)
-    kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
+    table = None
+    if w.page_size:
+        table, pool = W.make_page_table(w)
+        kv = []
+        for _, k, v in W.make_layer_kv(w, dev):       # page one copy at a time to bound memory
+            kv.append((W.to_paged(w, k, table, pool), W.to_paged(w, v, table, pool)))
+            del k, v
+        table = table.to(dev)
+    else:
+        kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
     q = W.make_queries(w, dev)
     B, Hq = w.batch, w.q_heads
     kps = W.top_k_per_seq(w)
     max_k = max(w.top_k, int(w.k_frac * w.context))
     ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
-                    page_size=0)
+                    page_size=w.page_size)
     sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
                             top_k_per_seq=None if kps is None else kps.to(dev))
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     t0, t1 = W.seq_lens_at(w, 0).to(dev), W.seq_lens_at(w, 1).to(dev)
-    views0 = [P.make_view(kv[l][0], kv[l][1], t0, max_seq_len=w.capacity) for l in range(copies)]
-    views1 = [P.make_view(kv[l][0], kv[l][1], t1, max_seq_len=w.capacity) for l in range(copies)]
+    views0 = [P.make_view(kv[l][0], kv[l][1], t0, page_table=table, max_seq_len=w.capacity) for l in range(copies)]
+    views1 = [P.make_view(kv[l][0], kv[l][1], t1, page_table=table, max_seq_len=w.capacity) for l in range(copies)]
     stream = torch.cuda.current_stream()
 
     def timed(fn):
@@ -92,8 +101,8 @@ def configs(dev):
     print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
           "mean set size | dense / amortised |")
     print("|---|---|---|---|---|---|---|")
-    for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K):
-        r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 100000 else 2)
+    for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
+        r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 50000 else 2)
         period = w.refresh * w.layer_group      # layer-steps per retrieval
         am = (r["refresh_us"] + (period - 1) * r["shared_us"]) / period
         print(f"| {w.name} | {r['dense_us']:.1f} | {r['refresh_us']:.1f} | {r['shared_us']:.1f} | {am:.1f} | "
@@ -102,7 +111,7 @@ def configs(dev):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C4 shapes instead")
+    ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C5 shapes instead")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
