@@ -74,10 +74,29 @@ def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6):
     dense = timed(lambda l: ctx.dense_decode_attn(q[l, 0], views0[l], B, out))
     refresh = timed(lambda l: ctx.decode_step(l, 0, sched, q[l, 0], views0[l], B, out))
     shared = timed(lambda l: ctx.decode_step(l, 1, sched, q[l, 1], views1[l], B, out))
-    _, cnt = ctx.get_index_set(B)
+    idx, cnt = ctx.get_index_set(B)
+    # Per-kernel times of a retrieval step: event pairs recorded inside the library.
+    ctx.profile_begin()
+    for _ in range(2):
+        for l in range(copies):
+            ctx.decode_step(l, 0, sched, q[l, 0], views0[l], B, out)
+    kern = {name: ms * 1e3 / n for name, (ms, n) in ctx.profile_end().items() if n}
     ctx.close()
+    # Bytes a sharing step must move: every listed row once per query head (logical), and once
+    # per KV head for the union over the heads of a group (unique).
+    G = Hq // w.kv_heads
+    cap = idx.shape[-1]
+    valid = torch.arange(cap, device=idx.device)[None, None, :] < cnt[:, :, None]
+    logical = int(cnt.sum()) * 512
+    mark = torch.zeros(B * w.kv_heads, w.capacity + 1, dtype=torch.bool, device=idx.device)
+    unit = (torch.arange(B, device=idx.device)[:, None] * w.kv_heads
+            + torch.arange(Hq, device=idx.device)[None, :] // G)[:, :, None].expand_as(idx)
+    mark[unit[valid].long(), idx[valid].long()] = True
+    unique = int(mark.sum()) * 512
+    key_bytes = int(t0.sum()) * w.kv_heads * 256
     return {"dense_us": dense, "refresh_us": refresh, "shared_us": shared,
-            "set_size": float(cnt.float().mean())}
+            "set_size": float(cnt.float().mean()), "kernels": kern, "logical_bytes": logical,
+            "unique_bytes": unique, "key_bytes": key_bytes}
 
 
 def table3(dev):
@@ -99,14 +118,17 @@ def table3(dev):
 
 def configs(dev):
     print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
-          "mean set size | dense / amortised |")
-    print("|---|---|---|---|---|---|---|")
+          "mean set size | dense / amortised | sharing step GB/s logical / unique | retrieval step kernels us |")
+    print("|---|---|---|---|---|---|---|---|---|")
     for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
         r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 50000 else 2)
         period = w.refresh * w.layer_group      # layer-steps per retrieval
         am = (r["refresh_us"] + (period - 1) * r["shared_us"]) / period
+        gbs = [r[k] / (r["shared_us"] * 1e3) for k in ("logical_bytes", "unique_bytes")]
+        kern = ", ".join(f"{k} {v:.1f}" for k, v in r["kernels"].items())
         print(f"| {w.name} | {r['dense_us']:.1f} | {r['refresh_us']:.1f} | {r['shared_us']:.1f} | {am:.1f} | "
-              f"{r['set_size']:.0f} | {r['dense_us'] / am:.2f}x |")
+              f"{r['set_size']:.0f} | {r['dense_us'] / am:.2f}x | {gbs[0]:.0f} / {gbs[1]:.0f} | {kern} "
+              f"(K stream {r['key_bytes'] / 1e6:.0f} MB) |")
 
 
 def main():

@@ -443,3 +443,23 @@ def test_host_side_errors(cuda_device):
     ctx.decode_step(0, 0, good, q, view, w.batch, out)                                   # still usable
     assert ctx.check() == 0
     ctx.close()
+
+
+@pytest.mark.gpu
+def test_radius_sweep_cells_small():
+    """The sweep script's cell on a small shape: the s = 1 row is the per-step oracle selector
+    (beta 0, coverage 1, whatever r), and sharing can only lose coverage."""
+    from paper_2602_08329_b200 import radius_sweep as RS
+    dev = torch.device("cuda:0")
+    w = W.C1_TINY.scaled(steps=8, halo=0.7, q_scale=3.0, sigma=0.3, heavy_hitters=32)
+    k, v = W.make_kv(w, dev)
+    q = W.make_queries(w, dev)
+    c1 = RS.run_cell(w, dev, k, v, q, 1, 2)
+    assert c1["beta_max"] == 0.0 and c1["cov_min"] == 1.0
+    assert c1["size"] <= w.sinks + w.top_k + w.window
+    c4 = RS.run_cell(w, dev, k, v, q, 4, 1)
+    assert c4["cov_mean"] <= 1.0 and c4["size"] > c1["size"]
+    assert abs(c4["delta1_mean"] - c1["delta_mean"]) < 1e-5      # delta* does not depend on the cell
+    c40 = RS.run_cell(w, dev, k, v, q, 4, 0)
+    assert c40["beta_mean"] >= -1e-5        # without dilation a shared set never beats the step's own top-k
+    assert c40["cov_mean"] <= c4["cov_mean"] + 1e-9
