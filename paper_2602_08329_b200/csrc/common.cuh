@@ -123,6 +123,11 @@ __device__ __forceinline__ uint32_t float_to_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Inverse of float_to_key.
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 // Combine two online-softmax states kept in the log2 domain: (m, l) <- (m, l) (+) (m2, l2).
 __device__ __forceinline__ void ml_combine(float& m, float& l, float m2, float l2) {
   float mn = fmaxf(m, m2);

@@ -42,6 +42,7 @@ struct prhs_ctx {
   prhs_config cfg{};
   int device = 0, sm_count = 148;
   int gq = 1, num_groups = 1, max_m = 0, shat_cap = 0, idx_cap = 0, ld = 0, sort_cap = 2;
+  int cand_cap = 0, two_bitmaps = 0;
   int max_chunks = 1, attn_ctas_per_sm = 2;
   size_t sel_smem = 0;
   // workspaces (device)
@@ -340,9 +341,15 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.out_lse_full = out_lse_full;
   p.flags = c->flags;
   p.sort_cap = c->sort_cap;
+  p.cand_cap = c->cand_cap;
+  p.two_bitmaps = c->two_bitmaps;
   {
+    // One CTA per unit.  With few units per SM the CTA is wide (the unit's latency chain is what
+    // counts); with many, narrower CTAs let four chains overlap on an SM instead of two.
+    const int units = batch * c->cfg.num_q_heads;
+    const int threads = units > 3 * c->sm_count ? kSelMaxThreads / 2 : kSelMaxThreads;
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
-    select_kernel<<<batch * c->cfg.num_q_heads, kSelThreads, c->sel_smem, st>>>(p);
+    select_kernel<<<units, threads, c->sel_smem, st>>>(p);
   }
   PRHS_CUDA(c, cudaGetLastError());
   if (!need) c->anchor_step[g] = step;
@@ -459,10 +466,21 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     delete c;
     return fail(nullptr, PRHS_ERR_CUDA, msg);
   }
-  // selection kernel shared memory: histogram + scalars + sort buffer + max(candidates, bitmap)
-  const int fixed = (kHistBins + kSelMiscWords) * 4 + c->sort_cap * 8;
-  const int bitmap_bytes = ((cfg->max_context + 31) / 32) * 4;
-  c->sel_smem = (size_t)fixed + (size_t)std::max(kCandCap * 8, bitmap_bytes);
+  // selection kernel shared memory: histogram + scalars + the candidate list, which later holds
+  // the sorted entries (at most sort_cap) followed by one or two position bitmaps
+  {
+    const size_t fixed = (size_t)(kHistWords + kSelMiscWords) * 4;
+    const size_t bitmap_bytes = (size_t)((cfg->max_context + 31) / 32) * 4;
+    auto need = [&](int cand_cap, int nbm) {
+      return fixed + std::max((size_t)cand_cap * 8, (size_t)c->sort_cap * 8 + nbm * bitmap_bytes);
+    };
+    c->cand_cap = std::max(4096, 2 * c->sort_cap);
+    c->two_bitmaps = 1;
+    if (need(c->cand_cap, 2) > (size_t)kMaxSmemBytes) c->two_bitmaps = 0;
+    while (need(c->cand_cap, 1 + c->two_bitmaps) > (size_t)kMaxSmemBytes && c->cand_cap > c->sort_cap)
+      c->cand_cap >>= 1;
+    c->sel_smem = need(c->cand_cap, 1 + c->two_bitmaps);
+  }
   if (c->sel_smem > (size_t)kMaxSmemBytes) {
     delete c;
     return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context / max_k too large for the selection kernel");

@@ -55,11 +55,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
     if (*abort || clock64() - t0 > kWaitBudgetCycles) return false;
   return true;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+// The key stream is read once and is far larger than L2: its lines are marked evict-first, and
+// the logits (a few tens of MB that the selection kernel reads next) evict-last, so that the
+// stream does not push the logits out to DRAM before they are used.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar), "l"(policy)
       : "memory");
+}
+__device__ __forceinline__ void st_f32x2_hint(float* p, float a, float b, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;" ::"l"(p), "f"(a), "f"(b), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void st_f32_hint(float* p, float a, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(a), "l"(policy) : "memory");
 }
 
 // grid (splits, Hkv, B).  tm_k: K viewed as [rows][128] bf16 (row pitch 256 B), box [64][64],
@@ -104,6 +125,7 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
   if (warp == kSTConsumers) {
     // ---------------- producer: one elected lane feeds the ring
     if (lane == 0) {
+      const uint64_t pol_k = l2_policy_evict_first();
       for (int j = 0; j < nstages; ++j) {
         const int slot = j % kSTStages;
         if (j >= kSTStages && !mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort)) {
@@ -115,8 +137,8 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
         const uint32_t full = bar0 + 8 * slot;
         const uint32_t dst = smem0 + slot * kSTStageBytes;
         mbar_expect_tx(full, kSTStageBytes);
-        tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full);
-        tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full);
+        tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full, pol_k);
+        tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full, pol_k);
       }
     }
   } else {
@@ -135,6 +157,7 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
       }
     }
     float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+    const uint64_t pol_s = l2_policy_evict_last();
     const int lm_mi = lane >> 3, lm_r = lane & 7;
     for (int j = 0; j < nstages; ++j) {
       const int slot = j % kSTStages;
@@ -173,13 +196,13 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
             const int key0 = pos0 + 8 * nt + 2 * tg;
             const float s0 = s[nt][2 * hh] * kScale, s1 = s[nt][2 * hh + 1] * kScale;
             if (key0 + 1 < end) {
-              if (dst) *reinterpret_cast<float2*>(dst + key0) = make_float2(s0, s1);
+              if (dst) st_f32x2_hint(dst + key0, s0, s1, pol_s);
               const float x0 = s0 * kLog2e, x1 = s1 * kLog2e;
               const float mn = fmaxf(m, fmaxf(x0, x1));
               l = l * exp2f(m - mn) + exp2f(x0 - mn) + exp2f(x1 - mn);
               m = mn;
             } else if (key0 < end) {
-              if (dst) dst[key0] = s0;
+              if (dst) st_f32_hint(dst + key0, s0, pol_s);
               const float x0 = s0 * kLog2e;
               const float mn = fmaxf(m, x0);
               l = l * exp2f(m - mn) + exp2f(x0 - mn);

@@ -1,31 +1,31 @@
 // Retrieval pass, part 2: exact top-k over the middle range (Sec. 4.1 "Selection
 // Criteria"), descending-logit order with ties broken by lower position, then the
-// neighbour dilation of Eq. 10.  One CTA per (sequence, query head).
+// neighbour dilation of Eq. 10.  One CTA per (sequence, query head), 256 or 512 threads.
 //
-// Fast path: a 1-in-16 sample of the unit's logits is histogrammed on the top 11 bits of the
-// order-preserving key; from it a conservative bin d_lo is chosen so that, with a wide
-// margin, at least k logits lie in bins >= d_lo.  ONE pass over all logits then collects those
-// into a short list in shared memory (about 1.5-2 k entries), and everything else -- the exact
-// bin of the k-th key, the remaining 21 key bits, ties -- is resolved on that list.  Small
-// problems (at most 8192 candidates) skip the sample and list every candidate.  If the list
-// comes out too short or too long (sampling bad luck, or degenerate inputs such as all-equal
-// logits), a generic 4 x 8-bit radix select over the logits in global memory takes over; it
-// orders ties by position explicitly.
+// Fast path: a 1-in-16 sample of the unit's logits (one aligned 16-byte group out of every 64
+// logits) is histogrammed on the top 11 bits of the order-preserving key; from it a
+// conservative bin d_lo is chosen so that, with a wide margin, at least k logits lie in bins
+// >= d_lo.  ONE pass over all logits (16-byte loads) then collects those into a short list in
+// shared memory (about 1.5-2 k entries), and everything else -- the exact bin of the k-th key,
+// the remaining 21 key bits, ties, the sort -- is resolved on that list, in place.  Small
+// problems (no more candidates than the list holds) skip the sample and list every candidate.
+// If the list comes out too short or too long (sampling bad luck, or degenerate inputs such as
+// all-equal logits), a generic 4 x 8-bit radix select over the logits in global memory takes
+// over; it orders ties by position explicitly.  Logits crowd into a few histogram bins (a
+// bin is a quarter of a binade), so every histogram update first merges the lanes of a warp
+// that hit the same bin (`match.any`) and issues one shared-memory atomic per distinct bin.
 #pragma once
 #include "common.cuh"
 
 namespace prhs {
 
-constexpr int kSelThreads = 512;
-constexpr int kHistBits = 11;
-constexpr int kHistBins = 1 << kHistBits;          // 2048
-constexpr int kHistShift = 32 - kHistBits;         // key >> 21
-constexpr int kSelMiscWords = 64;
-constexpr int kCandCap = 8192;                      // candidate list entries (8 bytes each)
+constexpr int kSelMaxThreads = 512;
+constexpr int kHistWords = 1024;                   // four 256-bin histograms
+constexpr int kSelMiscWords = 128;
 constexpr int kSampleStride = 16;
 
 struct SelectParams {
-  const float* scores;      // [B][Hq][ld]
+  const float* scores;      // [B][Hq][ld], 16-byte aligned, ld a multiple of 4
   int ld;
   const float2* part_ml;    // [B][Hq][nchunks] (m, l) in the log2 domain; chunks past t are unset
   int nchunks, chunk_rows;
@@ -48,7 +48,9 @@ struct SelectParams {
   float* lse_full;          // [B][Hq] workspace
   float* out_lse_full;      // optional
   uint32_t* flags;
-  int sort_cap;             // power of two >= max_k
+  int sort_cap;             // power of two >= max_k: most entries the sort takes
+  int cand_cap;             // candidate list entries (8 bytes each), >= sort_cap
+  int two_bitmaps;          // room for two position bitmaps behind the sorted entries
 };
 
 // Exclusive block scan of one int per thread; returns the exclusive prefix, *total gets the sum.
@@ -80,6 +82,51 @@ __device__ __forceinline__ int block_exclusive_scan(int v, uint32_t* ws /*>= 34 
   return res;
 }
 
+// The same for two ints per thread at once (one set of barriers).  ws >= 68 words.
+__device__ __forceinline__ void block_exclusive_scan2(int va, int vb, uint32_t* ws, int* ea, int* eb,
+                                                      int* ta, int* tb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int ia = va, ib = vb;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int xa = __shfl_up_sync(0xffffffffu, ia, off);
+    const int xb = __shfl_up_sync(0xffffffffu, ib, off);
+    if (lane >= off) { ia += xa; ib += xb; }
+  }
+  if (lane == 31) { ws[warp] = (uint32_t)ia; ws[34 + warp] = (uint32_t)ib; }
+  __syncthreads();
+  if (warp == 0) {
+    const bool in = lane < (int)(blockDim.x >> 5);
+    const int wa = in ? (int)ws[lane] : 0, wb = in ? (int)ws[34 + lane] : 0;
+    int sa = wa, sb = wb;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int xa = __shfl_up_sync(0xffffffffu, sa, off);
+      const int xb = __shfl_up_sync(0xffffffffu, sb, off);
+      if (lane >= off) { sa += xa; sb += xb; }
+    }
+    ws[lane] = (uint32_t)(sa - wa);
+    ws[34 + lane] = (uint32_t)(sb - wb);
+    if (lane == 31) { ws[32] = (uint32_t)sa; ws[66] = (uint32_t)sb; }
+  }
+  __syncthreads();
+  *ea = ia - va + (int)ws[warp];
+  *eb = ib - vb + (int)ws[34 + warp];
+  *ta = (int)ws[32];
+  *tb = (int)ws[66];
+  __syncthreads();
+}
+
+__device__ __forceinline__ int emit_bits(uint32_t x, int base, int* out, int o, int cap) {
+  while (x) {
+    const int bit = __ffs(x) - 1;
+    if (o < cap) out[o] = base + bit;
+    ++o;
+    x &= x - 1;
+  }
+  return o;
+}
+
 // Ascending list of the set bits of bm[0..words): out[0..min(total,cap)); returns total.
 __device__ __forceinline__ int compact_bitmap(const uint32_t* bm, int words, int* out, int cap,
                                               uint32_t* ws) {
@@ -90,16 +137,34 @@ __device__ __forceinline__ int compact_bitmap(const uint32_t* bm, int words, int
   for (int w = w0; w < w1; ++w) cnt += __popc(bm[w]);
   int total;
   int o = block_exclusive_scan(cnt, ws, &total);
-  for (int w = w0; w < w1; ++w) {
-    uint32_t x = bm[w];
-    while (x) {
-      const int bit = __ffs(x) - 1;
-      if (o < cap) out[o] = w * 32 + bit;
-      ++o;
-      x &= x - 1;
-    }
-  }
+  for (int w = w0; w < w1; ++w) o = emit_bits(bm[w], w * 32, out, o, cap);
   return total;
+}
+
+// Two bitmaps of the same length listed in one sweep (one scan, one set of barriers).
+__device__ __forceinline__ void compact_two(const uint32_t* bma, const uint32_t* bmb, int words, int* outa,
+                                            int capa, int* outb, int capb, uint32_t* ws, int* ta, int* tb) {
+  const int per = (words + (int)blockDim.x - 1) / (int)blockDim.x;
+  const int w0 = min((int)threadIdx.x * per, words);
+  const int w1 = min(w0 + per, words);
+  int ca = 0, cb = 0;
+  for (int w = w0; w < w1; ++w) {
+    ca += __popc(bma[w]);
+    cb += __popc(bmb[w]);
+  }
+  int oa, ob;
+  block_exclusive_scan2(ca, cb, ws, &oa, &ob, ta, tb);
+  for (int w = w0; w < w1; ++w) {
+    oa = emit_bits(bma[w], w * 32, outa, oa, capa);
+    ob = emit_bits(bmb[w], w * 32, outb, ob, capb);
+  }
+}
+
+// hist[bin] += 1 for the lanes with `valid`, one atomic per distinct bin of the warp.  Every lane
+// of the warp must call it.
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t bin, bool valid) {
+  const uint32_t peers = __match_any_sync(0xffffffffu, valid ? bin : 0xffffffffu);
+  if (valid && (int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
 }
 
 // Append `v` to list[] for the lanes with f set: one shared-memory atomic per warp.
@@ -147,6 +212,70 @@ __device__ __forceinline__ void find_bin_from_top(const uint32_t* hist, int nb, 
       c += hc;
     }
   }
+}
+
+// The warp's sample of logits (NX per lane: sample x * nt + slot of S, one logit out of every
+// sstride) and the largest value, at the resolution of the top 13 key bits, that at least rw of
+// them reach.  Bisection on the key bits; the count is a compare per sample and one warp
+// reduction per bit.
+constexpr int kThrBits = 13;
+template <int NX>
+__device__ __forceinline__ uint32_t sample_quantile(const float* g, int S, int sstride, int nt, int slot, int rw) {
+  uint32_t u[NX];
+#pragma unroll
+  for (int x = 0; x < NX; ++x) {
+    const int sidx = x * nt + slot;
+    u[x] = sidx < S ? float_to_key(__ldcg(g + (long long)sidx * sstride + ((sidx * 5) & 15))) : 0u;
+  }
+  uint32_t prefix = 0u;
+#pragma unroll 1
+  for (int bit = 31; bit > 31 - kThrBits; --bit) {
+    const uint32_t trial = prefix | (1u << bit);
+    int cnt = 0;
+#pragma unroll
+    for (int x = 0; x < NX; ++x) cnt += u[x] >= trial ? 1 : 0;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (cnt >= rw) prefix = trial;
+  }
+  return prefix;
+}
+
+// Warp-wide: the digit (of 256 bins, h 16-byte aligned) that holds the rem-th largest entry counted
+// from the top bin; every lane receives the bin, how many of that bin are still needed, and the
+// bin's count.
+__device__ __forceinline__ void find_bin_warp256(const uint32_t* h, int rem, int* bin, int* rem_out, int* eq_out) {
+  const int lane = threadIdx.x & 31;
+  const uint4 lo4 = *reinterpret_cast<const uint4*>(h + lane * 8);
+  const uint4 hi4 = *reinterpret_cast<const uint4*>(h + lane * 8 + 4);
+  const int c[8] = {(int)lo4.x, (int)lo4.y, (int)lo4.z, (int)lo4.w, (int)hi4.x, (int)hi4.y, (int)hi4.z, (int)hi4.w};
+  int s = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) s += c[j];
+  int incl = s;     // sum over lanes >= lane
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int x = __shfl_down_sync(0xffffffffu, incl, off);
+    if (lane + off < 32) incl += x;
+  }
+  const int above = incl - s;
+  const bool hit = above < rem && rem <= incl;
+  int b = 0, r = 0, e = 0, cc = above;
+  bool done = false;
+#pragma unroll
+  for (int j = 7; j >= 0; --j) {
+    if (!done && cc + c[j] >= rem) {
+      b = lane * 8 + j;
+      r = rem - cc;
+      e = c[j];
+      done = true;
+    }
+    cc += c[j];
+  }
+  const uint32_t bal = __ballot_sync(0xffffffffu, hit);
+  const int src = bal ? __ffs(bal) - 1 : 0;
+  *bin = __shfl_sync(0xffffffffu, b, src);
+  *rem_out = __shfl_sync(0xffffffffu, r, src);
+  *eq_out = __shfl_sync(0xffffffffu, e, src);
 }
 
 // ---- block-wide bitonic sort, descending, of P (a power of two >= 64) 64-bit entries in
@@ -207,15 +336,15 @@ __device__ __forceinline__ void block_sort_desc(unsigned long long* buf, int P) 
   }
 }
 
-__global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) {
+__global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);                     // kHistBins
-  uint32_t* misc = hist + kHistBins;                                          // kSelMiscWords
-  unsigned long long* wbuf = reinterpret_cast<unsigned long long*>(misc + kSelMiscWords);  // sort_cap
-  unsigned long long* cand = wbuf + p.sort_cap;                               // kCandCap
-  uint32_t* bm = reinterpret_cast<uint32_t*>(cand);                           // bitmap aliases cand
+  uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);                     // kHistWords
+  uint32_t* misc = hist + kHistWords;                                         // kSelMiscWords
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(misc + kSelMiscWords);  // cand_cap
+  uint32_t* bm = reinterpret_cast<uint32_t*>(cand + p.sort_cap);              // bitmaps behind the sorted entries
+  uint32_t* ws = misc + 8;                                                    // scan scratch (68 words)
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x;
   const int unit = blockIdx.x;
   if (p.need != nullptr && __ldg(p.need + unit) == 0) return;     // this head shares: no retrieval
   const long long sunit = (long long)unit * p.slots + (p.slot_of ? __ldg(p.slot_of + unit) : 0);
@@ -228,6 +357,11 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   const int kk = min(k, n);
   const int m_eff = min(p.m < 0 ? k / 3 : p.m, kk);
   const float* g = p.scores + (long long)unit * p.ld + lo;
+  // 16-byte groups: g[a0 + 4 i .. a0 + 4 i + 3], i < nb4; the few logits before and after are
+  // handled one by one
+  const int a0 = min(n, (4 - (int)(((long long)unit * p.ld + lo) & 3)) & 3);
+  const int nb4 = (n - a0) >> 2;
+  const float4* g4 = reinterpret_cast<const float4*>(g + a0);
 
   // full-softmax log-sum-exp from the scoring pass' per-chunk partials
   if (warp == 1) {
@@ -251,55 +385,78 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   }
   if (tid == 0) {
     if ((unit % p.num_q_heads) == 0) p.anchor_t[b] = t;
-    misc[4] = 0u;   // winners appended
-    misc[5] = 0u;   // candidates appended
+    misc[4] = 0u;   // winners kept
+    misc[5] = 0u;   // candidates listed
   }
   __syncthreads();
 
-  int total = 0;          // entries in wbuf to sort; the first kk after sorting are S*
+  int total = 0;          // entries in cand to sort; the first kk after sorting are S*
   bool fast_ok = false;
   if (kk > 0) {
     // ---------------- fast path
-    // 1. conservative bin d_lo from a sample (or 0: list everything)
-    uint32_t d_lo = 0u;
-    if (n > kCandCap) {
-      for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0u;
+    // the histograms of the four 8-bit passes of step 3 (the barrier after step 2 covers this)
+    for (int i = tid; i < kHistWords; i += nt) hist[i] = 0u;
+    // 1. conservative threshold from a sample (or -inf: list everything).  Every warp takes a
+    //    stratified 1-in-16 sample spread over the whole range (at most 16 logits per thread)
+    //    and finds, by bisection on the top 13 key bits, the value that
+    //    1.75 k/16 + 16 sampled logits of the CTA would reach if all warps saw the same
+    //    distribution; the lower median of the warps' values is the threshold.
+    float thr = -INFINITY;
+    if (n > p.cand_cap) {
+      const int nw = nt >> 5;
+      const int sstride = max(kSampleStride, (n + 16 * nt - 1) / (16 * nt));
+      const int S = n / sstride;
+      const int nx = (S + nt - 1) / nt;            // <= 16
+      const int slot = lane * nw + warp;
+      const int want = (int)((7ll * kk * S) / (4ll * n)) + 16;
+      const int rw = (want + nw - 1) / nw;
+      uint32_t prefix;
+      if (nx <= 4) prefix = sample_quantile<4>(g, S, sstride, nt, slot, rw);
+      else prefix = sample_quantile<16>(g, S, sstride, nt, slot, rw);
+      if (lane == 0) misc[80 + warp] = prefix;
       __syncthreads();
-      const int ns = n / kSampleStride;
-      for (int j0 = 0; j0 < ns; j0 += 8 * kSelThreads) {     // 8 independent loads in flight
-        uint32_t u8[8];
-#pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          const int j = j0 + x * kSelThreads + tid;
-          u8[x] = j < ns ? float_to_key(__ldcg(g + j * kSampleStride + (j & (kSampleStride - 1)))) : 0u;
-        }
-#pragma unroll
-        for (int x = 0; x < 8; ++x)
-          if (j0 + x * kSelThreads + tid < ns) atomicAdd(&hist[u8[x] >> kHistShift], 1u);
+      const uint32_t mine = lane < nw ? misc[80 + lane] : 0xffffffffu;
+      int rank = 0;
+      for (int j = 0; j < nw; ++j) {
+        const uint32_t o = __shfl_sync(0xffffffffu, mine, j);
+        rank += (o < mine || (o == mine && j < lane)) ? 1 : 0;
       }
-      __syncthreads();
-      // want at least 1.5 k/16 + 16 sampled logits at or above d_lo (several sigma of margin)
-      const int want = min(ns, (3 * kk) / (2 * kSampleStride) + 16);
-      if (warp == 0) find_bin_from_top(hist, kHistBins, want, misc);
-      __syncthreads();
-      d_lo = misc[0];
-      __syncthreads();
+      const uint32_t pick = __ballot_sync(0xffffffffu, lane < nw && rank == (nw - 1) / 2);
+      thr = key_to_float(__shfl_sync(0xffffffffu, mine, __ffs(pick) - 1));
+      if (!(thr == thr)) thr = -INFINITY;
     }
-    // 2. one pass over the logits: 16 independent loads in flight per thread, then one warp
-    //    scan and one shared-memory atomic per warp and batch to place the listed entries
-    const int nrounds = (n + kSelThreads - 1) / kSelThreads;
-    for (int rd0 = 0; rd0 < nrounds; rd0 += 16) {
-      uint32_t u16[16];
+    // 2. one pass over the logits: four 16-byte loads in flight per thread, a float compare per
+    //    logit, then one warp scan and one shared-memory atomic per warp and batch to place the
+    //    positions of the listed logits (their keys are fetched afterwards)
+    if (warp == 0) {     // the logits before the first and after the last 16-byte group
+      const int tail0 = a0 + 4 * nb4;
+      int i = -1;
+      if (lane < a0) i = lane;
+      else if (lane >= 4 && tail0 + (lane - 4) < n) i = tail0 + (lane - 4);
+      float v = -INFINITY;
+      if (i >= 0) v = __ldcg(g + i);
+      warp_append(i >= 0 && v >= thr, (unsigned long long)(uint32_t)(lo + i), cand, &misc[5],
+                  (uint32_t)p.cand_cap);
+    }
+    for (int i0 = 0; i0 < nb4; i0 += 4 * nt) {
+      float4 v[4];
 #pragma unroll
-      for (int x = 0; x < 16; ++x) {
-        const int i = (rd0 + x) * kSelThreads + tid;
-        u16[x] = i < n ? float_to_key(__ldcg(g + i)) : 0u;
+      for (int x = 0; x < 4; ++x) {
+        const int i4 = i0 + x * nt + tid;
+        v[x] = i4 < nb4 ? __ldcg(g4 + i4) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
       }
       uint32_t cmask = 0u;
 #pragma unroll
-      for (int x = 0; x < 16; ++x) {
-        const int i = (rd0 + x) * kSelThreads + tid;
-        cmask |= (uint32_t)(i < n && (u16[x] >> kHistShift) >= d_lo) << x;
+      for (int x = 0; x < 4; ++x) {
+        cmask |= (uint32_t)(v[x].x >= thr) << (4 * x);
+        cmask |= (uint32_t)(v[x].y >= thr) << (4 * x + 1);
+        cmask |= (uint32_t)(v[x].z >= thr) << (4 * x + 2);
+        cmask |= (uint32_t)(v[x].w >= thr) << (4 * x + 3);
+      }
+      if (i0 + 4 * nt > nb4) {          // last batch: drop the groups past the end
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+          if (i0 + x * nt + tid >= nb4) cmask &= ~(0xfu << (4 * x));
       }
       const uint32_t mine = (uint32_t)__popc(cmask);
       uint32_t incl = mine;
@@ -311,58 +468,68 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
       uint32_t bc = 0u;
       if (lane == 31 && incl) bc = atomicAdd(&misc[5], incl);
       uint32_t oc = __shfl_sync(0xffffffffu, bc, 31) + incl - mine;
-#pragma unroll
-      for (int x = 0; x < 16; ++x) {
-        if ((cmask >> x) & 1u) {
-          if (oc < (uint32_t)kCandCap) cand[oc] = make_entry(u16[x], lo + (rd0 + x) * kSelThreads + tid);
-          ++oc;
-        }
+      const int pos0 = lo + a0 + 4 * (i0 + tid);
+      while (cmask) {
+        const int x = __ffs(cmask) - 1;
+        cmask &= cmask - 1u;
+        if (oc < (uint32_t)p.cand_cap)
+          cand[oc] = (unsigned long long)(uint32_t)(pos0 + 4 * (x >> 2) * nt + (x & 3));
+        ++oc;
       }
     }
     __syncthreads();
     const int ncand = (int)misc[5];
-    fast_ok = ncand >= kk && ncand <= kCandCap;
+    fast_ok = ncand >= kk && ncand <= p.cand_cap;
     if (fast_ok) {
-      // 3. exact histogram of the list -> bin d1 of the kk-th largest key
-      for (int i = tid; i < kHistBins; i += kSelThreads) hist[i] = 0u;
+      // 3. exact radix select on the list: four 8-bit passes, one barrier each; every warp finds
+      //    the digit for itself.  The first pass also fetches the keys of the listed positions.
+      const float* srow = p.scores + (long long)unit * p.ld;
+      for (int i0 = 0; i0 < ncand; i0 += nt) {
+        const int i = i0 + tid;
+        uint32_t key = 0u;
+        if (i < ncand) {
+          const int pos = (int)(uint32_t)cand[i];
+          key = float_to_key(__ldcg(srow + pos));
+          cand[i] = make_entry(key, pos);
+        }
+        hist_add(hist, key >> 24, i < ncand);
+      }
       __syncthreads();
-      for (int i = tid; i < ncand; i += kSelThreads)
-        atomicAdd(&hist[(uint32_t)(cand[i] >> 32) >> kHistShift], 1u);
-      __syncthreads();
-      if (warp == 0) find_bin_from_top(hist, kHistBins, kk, misc);
-      __syncthreads();
-      uint32_t prefix = misc[0] << kHistShift;
-      int rem = (int)misc[1], eq = (int)misc[2];
-      __syncthreads();
-      // 4. the remaining 21 key bits within that bin: 3 passes of 7 bits
-      if (rem < eq) {
-        for (int pass = 0; pass < 3; ++pass) {
-          const int shift = kHistShift - 7 * (pass + 1);
-          const uint32_t mask = 0xffffffffu << (shift + 7);
-          if (tid < 128) hist[tid] = 0u;
-          __syncthreads();
-          for (int i = tid; i < ncand; i += kSelThreads) {
-            const uint32_t u = (uint32_t)(cand[i] >> 32);
-            if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 127u], 1u);
+      uint32_t T = 0u;
+      int rem = kk, eq = 0;
+      for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t* h = hist + 256 * pass;
+        if (pass > 0) {
+          const uint32_t mask = 0xffffffffu << (shift + 8);
+          for (int i0 = 0; i0 < ncand; i0 += nt) {
+            const int i = i0 + tid;
+            const uint32_t key = i < ncand ? (uint32_t)(cand[i] >> 32) : 0u;
+            hist_add(hist + 256 * pass, (key >> shift) & 255u, i < ncand && (key & mask) == T);
           }
           __syncthreads();
-          if (warp == 0) find_bin_from_top(hist, 128, rem, misc);
-          __syncthreads();
-          prefix |= misc[0] << shift;
-          rem = (int)misc[1];
-          eq = (int)misc[2];
-          __syncthreads();
         }
-      }   // else every key of bin d1 is needed: the threshold is the start of the bin
-      const uint32_t T = prefix;            // keys >= T: the winners plus the surplus ties at T
-      // 5. winners and ties into the sort buffer; sorting orders ties by position and the
-      //    surplus falls behind the first kk entries
-      const int crounds = (ncand + kSelThreads - 1) / kSelThreads;
-      for (int rd = 0; rd < crounds; ++rd) {
-        const int i = rd * kSelThreads + tid;
-        unsigned long long e = 0ull;
-        if (i < ncand) e = cand[i];
-        warp_append(i < ncand && (uint32_t)(e >> 32) >= T, e, wbuf, &misc[4], (uint32_t)p.sort_cap);
+        int bin;
+        find_bin_warp256(h, rem, &bin, &rem, &eq);
+        T |= (uint32_t)bin << shift;
+        if (rem == eq) break;      // every key that starts like T is needed: the low bits stay zero
+      }
+      // 4. winners and ties (keys >= T) to the front of the list, in place: a batch of entries
+      //    is read by all threads before any of them is overwritten, and later batches lie
+      //    behind everything written.  Sorting orders ties by position; the surplus ties fall
+      //    behind the first kk entries.
+      for (int c0 = 0; c0 < ncand; c0 += 8 * nt) {
+        unsigned long long e[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          const int i = c0 + x * nt + tid;
+          e[x] = i < ncand ? cand[i] : 0ull;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+          if (c0 + x * nt < ncand)
+            warp_append(e[x] != 0ull && (uint32_t)(e[x] >> 32) >= T, e[x], cand, &misc[4], (uint32_t)p.sort_cap);
       }
       __syncthreads();
       total = (int)misc[4];
@@ -383,9 +550,10 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
         const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
-        for (int i = tid; i < n; i += kSelThreads) {
-          const uint32_t u = float_to_key(__ldcg(g + i));
-          if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
+        for (int i0 = 0; i0 < n; i0 += nt) {
+          const int i = i0 + tid;
+          const uint32_t u = i < n ? float_to_key(__ldcg(g + i)) : 0u;
+          hist_add(hist, (u >> shift) & 255u, i < n && (u & mask) == prefix);
         }
         __syncthreads();
         if (warp == 0) find_bin_from_top(hist, 256, rem, misc);
@@ -397,31 +565,30 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
       const uint32_t T = prefix;
       const int need = rem, gt_total = kk - need;
       const bool all_ties = (eq == need);
-      const int nrounds2 = (n + kSelThreads - 1) / kSelThreads;
-      for (int rd = 0; rd < nrounds2; ++rd) {
-        const int i = rd * kSelThreads + tid;
+      for (int i0 = 0; i0 < n; i0 += nt) {
+        const int i = i0 + tid;
         uint32_t u = 0u;
         if (i < n) u = float_to_key(__ldcg(g + i));
-        warp_append(i < n && (u > T || (all_ties && u == T)), make_entry(u, lo + i), wbuf, &misc[4],
+        warp_append(i < n && (u > T || (all_ties && u == T)), make_entry(u, lo + i), cand, &misc[4],
                     (uint32_t)p.sort_cap);
       }
       if (!all_ties) {
         // ties at T, lowest positions first
         int base = 0;
-        for (int c0 = 0; c0 < n && base < need; c0 += kSelThreads) {
+        for (int c0 = 0; c0 < n && base < need; c0 += nt) {
           const int i = c0 + tid;
           const bool f = (i < n) && float_to_key(__ldcg(g + i)) == T;
           const uint32_t bal = __ballot_sync(0xffffffffu, f);
           if (lane == 0) misc[8 + warp] = __popc(bal);
           __syncthreads();
           int before = 0, tot = 0;
-          for (int w = 0; w < kSelThreads / 32; ++w) {
+          for (int w = 0; w < (nt >> 5); ++w) {
             const int c = (int)misc[8 + w];
             if (w < warp) before += c;
             tot += c;
           }
           const int rank = base + before + __popc(bal & ((1u << lane) - 1u));
-          if (f && rank < need) wbuf[gt_total + rank] = make_entry(T, lo + i);
+          if (f && rank < need) cand[gt_total + rank] = make_entry(T, lo + i);
           base += tot;
           __syncthreads();
         }
@@ -434,14 +601,17 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
   // ---- sort: descending key, ascending position among equal keys
   int P = 64;
   while (P < total) P <<= 1;
-  for (int i = total + tid; i < P; i += kSelThreads) wbuf[i] = 0ull;
+  for (int i = total + tid; i < P; i += nt) cand[i] = 0ull;
+  const int words = (t + 31) >> 5;      // the bitmaps live behind the sort_cap entries
+  const int bm_words = p.two_bitmaps ? 2 * words : words;
+  for (int w = tid; w < bm_words; w += nt) bm[w] = 0u;
   __syncthreads();
-  block_sort_desc(wbuf, P);
+  block_sort_desc(cand, P);
 
   // ---- S* in descending-logit order
   int* sd = p.sstar_desc + sunit * p.max_k;
-  for (int e = tid; e < p.max_k; e += kSelThreads) {
-    const int v = e < kk ? (int)(0xffffffffu - (uint32_t)(wbuf[e] & 0xffffffffull)) : -1;
+  for (int e = tid; e < p.max_k; e += nt) {
+    const int v = e < kk ? (int)(0xffffffffu - (uint32_t)(cand[e] & 0xffffffffull)) : -1;
     sd[e] = v;
     if (p.out_idx) p.out_idx[(long long)unit * p.max_k + e] = v;
   }
@@ -450,27 +620,41 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(SelectParams p) 
     if (p.out_count) p.out_count[unit] = kk;
   }
 
-  // ---- ascending S*, then the dilated S^ (Eq. 10), through a position bitmap
-  const int words = (t + 31) >> 5;
-  for (int w = tid; w < words; w += kSelThreads) bm[w] = 0u;
-  __syncthreads();
-  for (int e = tid; e < kk; e += kSelThreads) {
-    const uint32_t pos = 0xffffffffu - (uint32_t)(wbuf[e] & 0xffffffffull);
+  // ---- ascending S*, and the dilated S^ (Eq. 10), through position bitmaps
+  if (p.two_bitmaps) {
+    uint32_t* bh = bm + words;
+    for (int e = tid; e < kk; e += nt) {
+      const int pos = (int)(0xffffffffu - (uint32_t)(cand[e] & 0xffffffffull));
+      atomicOr(&bm[pos >> 5], 1u << (pos & 31));
+      const int rr = e < m_eff ? p.r : 0;
+      for (int j = -rr; j <= rr; ++j) {
+        const int x = pos + j;
+        if (x >= 0 && x < t) atomicOr(&bh[x >> 5], 1u << (x & 31));
+      }
+    }
+    __syncthreads();
+    int ns, nh;
+    compact_two(bm, bh, words, p.sstar_asc + sunit * p.max_k, p.max_k, p.shat_asc + sunit * p.shat_cap,
+                p.shat_cap, ws, &ns, &nh);
+    if (tid == 0) p.n_hat[sunit] = min(nh, p.shat_cap);
+    return;
+  }
+  for (int e = tid; e < kk; e += nt) {
+    const uint32_t pos = 0xffffffffu - (uint32_t)(cand[e] & 0xffffffffull);
     atomicOr(&bm[pos >> 5], 1u << (pos & 31u));
   }
   __syncthreads();
-  compact_bitmap(bm, words, p.sstar_asc + sunit * p.max_k, p.max_k, misc + 8);
+  compact_bitmap(bm, words, p.sstar_asc + sunit * p.max_k, p.max_k, ws);
   __syncthreads();   // every thread has finished reading the bitmap before it grows
-  for (int e = tid; e < m_eff; e += kSelThreads) {
-    const int pos = (int)(0xffffffffu - (uint32_t)(wbuf[e] & 0xffffffffull));
+  for (int e = tid; e < m_eff; e += nt) {
+    const int pos = (int)(0xffffffffu - (uint32_t)(cand[e] & 0xffffffffull));
     for (int j = -p.r; j <= p.r; ++j) {
       const int x = pos + j;
       if (x >= 0 && x < t) atomicOr(&bm[x >> 5], 1u << (x & 31));
     }
   }
   __syncthreads();
-  const int nh = compact_bitmap(bm, words, p.shat_asc + sunit * p.shat_cap, p.shat_cap,
-                                misc + 8);
+  const int nh = compact_bitmap(bm, words, p.shat_asc + sunit * p.shat_cap, p.shat_cap, ws);
   if (tid == 0) p.n_hat[sunit] = min(nh, p.shat_cap);
 }
 
