@@ -344,10 +344,10 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.cand_cap = c->cand_cap;
   p.two_bitmaps = c->two_bitmaps;
   {
-    // One CTA per unit.  With few units per SM the CTA is wide (the unit's latency chain is what
-    // counts); with many, narrower CTAs let four chains overlap on an SM instead of two.
+    // One CTA of 512 threads per unit (two per SM).  256 threads measured slower on every
+    // configuration but one (the kernel is a chain of short phases; wide CTAs shorten it).
     const int units = batch * c->cfg.num_q_heads;
-    const int threads = units > 3 * c->sm_count ? kSelMaxThreads / 2 : kSelMaxThreads;
+    const int threads = kSelMaxThreads;
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
     select_kernel<<<units, threads, c->sel_smem, st>>>(p);
   }
@@ -466,14 +466,12 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     delete c;
     return fail(nullptr, PRHS_ERR_CUDA, msg);
   }
-  // selection kernel shared memory: histogram + scalars + the candidate list, which later holds
-  // the sorted entries (at most sort_cap) followed by one or two position bitmaps
+  // selection kernel shared memory: histograms + scalars + the candidate list (which later holds
+  // the sorted entries and the merge sort's second buffer) + one or two position bitmaps
   {
     const size_t fixed = (size_t)(kHistWords + kSelMiscWords) * 4;
     const size_t bitmap_bytes = (size_t)((cfg->max_context + 31) / 32) * 4;
-    auto need = [&](int cand_cap, int nbm) {
-      return fixed + std::max((size_t)cand_cap * 8, (size_t)c->sort_cap * 8 + nbm * bitmap_bytes);
-    };
+    auto need = [&](int cand_cap, int nbm) { return fixed + (size_t)cand_cap * 8 + nbm * bitmap_bytes; };
     c->cand_cap = std::max(4096, 2 * c->sort_cap);
     c->two_bitmaps = 1;
     if (need(c->cand_cap, 2) > (size_t)kMaxSmemBytes) c->two_bitmaps = 0;

@@ -1,19 +1,22 @@
 // Retrieval pass, part 2: exact top-k over the middle range (Sec. 4.1 "Selection
 // Criteria"), descending-logit order with ties broken by lower position, then the
-// neighbour dilation of Eq. 10.  One CTA per (sequence, query head), 256 or 512 threads.
+// neighbour dilation of Eq. 10.  One CTA per (sequence, query head); any multiple of 32 threads
+// up to 512 works, 512 is what the library launches.
 //
-// Fast path: a 1-in-16 sample of the unit's logits (one aligned 16-byte group out of every 64
-// logits) is histogrammed on the top 11 bits of the order-preserving key; from it a
-// conservative bin d_lo is chosen so that, with a wide margin, at least k logits lie in bins
-// >= d_lo.  ONE pass over all logits (16-byte loads) then collects those into a short list in
-// shared memory (about 1.5-2 k entries), and everything else -- the exact bin of the k-th key,
-// the remaining 21 key bits, ties, the sort -- is resolved on that list, in place.  Small
-// problems (no more candidates than the list holds) skip the sample and list every candidate.
-// If the list comes out too short or too long (sampling bad luck, or degenerate inputs such as
-// all-equal logits), a generic 4 x 8-bit radix select over the logits in global memory takes
-// over; it orders ties by position explicitly.  Logits crowd into a few histogram bins (a
-// bin is a quarter of a binade), so every histogram update first merges the lanes of a warp
-// that hit the same bin (`match.any`) and issues one shared-memory atomic per distinct bin.
+// Fast path: every warp takes a stratified 1-in-16 sample of the unit's logits and finds by
+// bisection on the top 13 key bits (a compare per sample and one warp reduction per bit) the
+// value that a conservative share of them reach; the lower median over the warps is the
+// threshold, chosen so that about 2 k logits pass it and, with a wide margin, no fewer than k.
+// ONE pass over all logits (16-byte loads, one float compare each) lists the positions of those
+// in shared memory, and everything else -- their keys, an exact 4 x 8-bit radix select of the
+// k-th key, ties, the sort -- is resolved on that list, in place.  Small problems (no more
+// candidates than the list holds) skip the sample and list every candidate.  If the list comes
+// out too short or too long (sampling bad luck, or degenerate inputs such as all-equal logits),
+// a generic 4 x 8-bit radix select over the logits in global memory takes over; it orders ties
+// by position explicitly.  Logits crowd into a few histogram bins, so every histogram update
+// first merges the lanes of a warp that hit the same bin (`match.any`) and issues one
+// shared-memory atomic per distinct bin.  The winners are sorted by a merge sort (64-entry runs
+// in registers, then one binary-search merge level per barrier).
 #pragma once
 #include "common.cuh"
 
@@ -336,12 +339,51 @@ __device__ __forceinline__ void block_sort_desc(unsigned long long* buf, int P) 
   }
 }
 
+// ---- block-wide merge sort, descending, of P (a power of two >= 64) DISTINCT 64-bit entries.
+// Warps sort 64-entry runs in registers; then runs are merged pairwise, log2(P / 64) times: every
+// entry finds by binary search how many entries of the sibling run precede it, which with its
+// own index in its run is its place in the merged run.  One barrier per level (a bitonic
+// network needs one per stride).  Reads buf, ping-pongs with alt, leaves the result in buf.
+__device__ __forceinline__ void block_merge_sort_desc(unsigned long long* buf, unsigned long long* alt, int P) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nwarps = blockDim.x >> 5;
+  int levels = 0;
+  while ((64 << levels) < P) ++levels;
+  unsigned long long* src = (levels & 1) ? alt : buf;     // an even number of moves ends in buf
+  unsigned long long* dst = (levels & 1) ? buf : alt;
+  for (int blk = warp; blk < (P >> 6); blk += nwarps) {
+    const int pos_a = blk * 64 + lane;
+    unsigned long long a = buf[pos_a], b = buf[pos_a + 32];
+    for (int size = 2; size <= 64; size <<= 1) warp_sort_steps(a, b, lane, size, size >> 1);   // every run descending
+    src[pos_a] = a;
+    src[pos_a + 32] = b;
+  }
+  __syncthreads();
+  for (int lg = 6; (1 << lg) < P; ++lg) {
+    const int L = 1 << lg;
+#pragma unroll 2
+    for (int i = tid; i < P; i += blockDim.x) {
+      const unsigned long long e = src[i];
+      const int run = i >> lg, within = i & (L - 1);
+      const unsigned long long* sib = src + (run ^ 1) * L;
+      int cnt = 0;                                   // sibling entries greater than e
+      for (int step = L >> 1; step > 0; step >>= 1)
+        if (sib[cnt + step - 1] > e) cnt += step;
+      if (sib[cnt] > e) ++cnt;
+      // equal entries do not occur; between the two runs of a pair the left one would go first
+      dst[(run & ~1) * L + within + cnt] = e;
+    }
+    __syncthreads();
+    unsigned long long* t = src; src = dst; dst = t;
+  }
+}
+
 __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);                     // kHistWords
   uint32_t* misc = hist + kHistWords;                                         // kSelMiscWords
   unsigned long long* cand = reinterpret_cast<unsigned long long*>(misc + kSelMiscWords);  // cand_cap
-  uint32_t* bm = reinterpret_cast<uint32_t*>(cand + p.sort_cap);              // bitmaps behind the sorted entries
+  uint32_t* bm = reinterpret_cast<uint32_t*>(cand + p.cand_cap);              // position bitmaps behind the list
   uint32_t* ws = misc + 8;                                                    // scan scratch (68 words)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x;
@@ -601,12 +643,13 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
   // ---- sort: descending key, ascending position among equal keys
   int P = 64;
   while (P < total) P <<= 1;
-  for (int i = total + tid; i < P; i += nt) cand[i] = 0ull;
-  const int words = (t + 31) >> 5;      // the bitmaps live behind the sort_cap entries
+  for (int i = total + tid; i < P; i += nt) cand[i] = (unsigned long long)(P - i);   // distinct, below every entry
+  const int words = (t + 31) >> 5;
   const int bm_words = p.two_bitmaps ? 2 * words : words;
   for (int w = tid; w < bm_words; w += nt) bm[w] = 0u;
   __syncthreads();
-  block_sort_desc(cand, P);
+  if (p.sort_cap + P <= p.cand_cap) block_merge_sort_desc(cand, cand + p.sort_cap, P);
+  else block_sort_desc(cand, P);
 
   // ---- S* in descending-logit order
   int* sd = p.sstar_desc + sunit * p.max_k;
