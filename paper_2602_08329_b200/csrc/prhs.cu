@@ -206,22 +206,25 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.need = need;
   sp.flags = c->flags;
   bool tma_done = false;
-  if (c->encode_tiled && kv.page_table == nullptr) {
-    // K as a 2-D tensor [rows][128] bf16; rows past the last sequence's max length are out of
-    // bounds for the copy engine (zero fill), rows in between belong to the cache
+  if (c->encode_tiled) {
+    // K as a 2-D tensor [rows][128] bf16.  Contiguous cache: rows past the last sequence's max
+    // length are out of bounds for the copy engine (zero fill), rows in between belong to the
+    // cache; a copy brings 64 rows.  Paged cache: the rows of the page pool; a copy brings the
+    // 16 rows of one page.
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    const bool paged = kv.page_table != nullptr;
     const unsigned long long outer_rows = (unsigned long long)(kv.stride_outer >> 7);
     const unsigned long long head_rows = (unsigned long long)(kv.stride_head >> 7);
     const unsigned long long rows_total =
-        (unsigned long long)(batch - 1) * outer_rows + (unsigned long long)(c->cfg.num_kv_heads - 1) * head_rows +
-        (unsigned long long)max_t;
+        (unsigned long long)((paged ? kv.num_pages : batch) - 1) * outer_rows +
+        (unsigned long long)(c->cfg.num_kv_heads - 1) * head_rows + (unsigned long long)(paged ? 16 : max_t);
     if (rows_total < (1ull << 31)) {
       alignas(64) CUtensorMap tm;
       const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows_total};
       const cuuint64_t gstr[1] = {(cuuint64_t)kRowBytes};
-      const cuuint32_t box[2] = {64u, (cuuint32_t)kSTStageRows};
+      const cuuint32_t box[2] = {64u, paged ? 16u : (cuuint32_t)kSTStageRows};
       const cuuint32_t estr[2] = {1u, 1u};
       const CUresult cr = reinterpret_cast<EncodeFn>(c->encode_tiled)(
           &tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(kv.k), gdim, gstr, box, estr,
@@ -229,7 +232,9 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (cr == CUDA_SUCCESS) {
         LaunchScope ls(c, PRHS_KIND_SCORE, st);
-        score_tma_kernel<<<dim3(sp.splits, c->cfg.num_kv_heads, batch), kSTThreads, kSTSmemBytes, st>>>(tm, sp);
+        const dim3 grid(sp.splits, c->cfg.num_kv_heads, batch);
+        if (paged) score_tma_kernel<true><<<grid, kSTThreads, kSTSmemBytes, st>>>(tm, sp);
+        else score_tma_kernel<false><<<grid, kSTThreads, kSTSmemBytes, st>>>(tm, sp);
         tma_done = true;
       }
     }
@@ -487,7 +492,9 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(score_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
+    e = cudaFuncSetAttribute(score_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
   if (e == cudaSuccess) {
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;

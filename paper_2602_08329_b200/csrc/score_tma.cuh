@@ -1,4 +1,4 @@
-// Retrieval scoring with the K stream staged by TMA (contiguous caches).
+// Retrieval scoring with the K stream staged by TMA (contiguous and paged caches).
 //
 // Logits a_i = q . k_i / sqrt(d) for all i < t (Eq. 2), as in score_ring_kernel, but the K
 // tiles are brought into shared memory by the tensor memory accelerator: one elected thread
@@ -6,7 +6,11 @@
 // each half of the 128 dimensions, 128-byte swizzle so that ldmatrix reads are conflict-free),
 // completion is signalled on an mbarrier, and four consumer warps (16 keys each) run the
 // m16n8k16 MMAs for all heads of the KV group.  A six-stage ring keeps up to 80 KB in flight
-// per CTA with no address arithmetic in the consumer warps.
+// per CTA with no address arithmetic in the consumer warps.  With a paged cache the tensor is
+// the page pool, a stage is four pages of 16 keys, and the producer issues one pair of
+// [16 rows][64 columns] boxes per page after looking its id up in the page table (ids of the
+// next stage are fetched while the current one is issued); pages past the end of the
+// sequence are not fetched and an id outside the pool is skipped and flagged.
 //
 // Every wait on an mbarrier is bounded: a wait that exceeds its budget records
 // kFlagTimeout and the CTA drains and returns, so a wrong descriptor cannot hang the GPU.
@@ -83,8 +87,10 @@ __device__ __forceinline__ void st_f32_hint(float* p, float a, uint64_t policy) 
   asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(a), "l"(policy) : "memory");
 }
 
-// grid (splits, Hkv, B).  tm_k: K viewed as [rows][128] bf16 (row pitch 256 B), box [64][64],
-// 128-byte swizzle; row of (b, kvh, i) = b * outer_rows + kvh * head_rows + i.
+// grid (splits, Hkv, B).  tm_k: K viewed as [rows][128] bf16 (row pitch 256 B), 128-byte swizzle.
+// Contiguous: box [64][64], row of (b, kvh, i) = b * outer_rows + kvh * head_rows + i.
+// Paged: box [16][64], row of (page, kvh, i mod 16) = page * outer_rows + kvh * head_rows + i mod 16.
+template <bool kPaged>
 __global__ void __launch_bounds__(kSTThreads)
 score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
   extern __shared__ unsigned char st_smem_raw[];
@@ -109,7 +115,8 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
   const int nstages = (end - start + kSTStageRows - 1) / kSTStageRows;
   const uint32_t smem0 = ((uint32_t)__cvta_generic_to_shared(st_smem_raw) + 1023u) & ~1023u;
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
-  const int row_base = b * (int)(p.kv.stride_outer >> 7) + kvh * (int)(p.kv.stride_head >> 7) + start;
+  const int outer_rows = (int)(p.kv.stride_outer >> 7), head_rows = (int)(p.kv.stride_head >> 7);
+  const int row_base = kPaged ? kvh * head_rows : b * outer_rows + kvh * head_rows + start;
 
   if (tid == 0) {
     for (int s = 0; s < kSTStages; ++s) {
@@ -126,8 +133,21 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     // ---------------- producer: one elected lane feeds the ring
     if (lane == 0) {
       const uint64_t pol_k = l2_policy_evict_first();
+      const int* ptab = kPaged ? p.kv.page_table + (long long)b * p.kv.page_table_stride + (start >> kPageShift) : nullptr;
+      int pg_next[4] = {0, 0, 0, 0};
+      if (kPaged) {
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+          if (start + 16 * x < end) pg_next[x] = __ldg(ptab + x);
+      }
       for (int j = 0; j < nstages; ++j) {
         const int slot = j % kSTStages;
+        int pg[4] = {pg_next[0], pg_next[1], pg_next[2], pg_next[3]};
+        if (kPaged && j + 1 < nstages) {      // page ids of the next stage, in flight during the wait below
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+            if (start + (j + 1) * kSTStageRows + 16 * x < end) pg_next[x] = __ldg(ptab + 4 * (j + 1) + x);
+        }
         if (j >= kSTStages && !mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort)) {
           atomicOr(p.flags, kFlagTimeout);
           sh_abort = 1;
@@ -136,9 +156,30 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
         if (*(volatile int*)&sh_abort) break;
         const uint32_t full = bar0 + 8 * slot;
         const uint32_t dst = smem0 + slot * kSTStageBytes;
-        mbar_expect_tx(full, kSTStageBytes);
-        tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full, pol_k);
-        tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full, pol_k);
+        if (!kPaged) {
+          mbar_expect_tx(full, kSTStageBytes);
+          tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full, pol_k);
+          tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full, pol_k);
+        } else {
+          uint32_t okmask = 0u;
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            if (start + j * kSTStageRows + 16 * x < end) {
+              if ((unsigned)pg[x] < (unsigned)p.kv.num_pages) okmask |= 1u << x;
+              else atomicOr(p.flags, kFlagBadPage);
+            }
+          }
+          // the barrier needs its arrive even when no page of the stage is fetched
+          mbar_expect_tx(full, (uint32_t)__popc(okmask) * 4096u);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            if ((okmask >> x) & 1u) {
+              const int row = pg[x] * outer_rows + row_base;
+              tma_load_2d(dst + x * 2048, &tm_k, 0, row, full, pol_k);
+              tma_load_2d(dst + kSTHalfBytes + x * 2048, &tm_k, 64, row, full, pol_k);
+            }
+          }
+        }
       }
     }
   } else {
