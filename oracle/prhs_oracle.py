@@ -119,6 +119,19 @@ def topk_middle(a: np.ndarray, t: int, sinks: int, window: int, k: int, psaw_lo:
     return cand[order[: min(k, hi - lo)]]
 
 
+def group_logits(per_head: list) -> np.ndarray:
+    """Group-shared ranking logits of a KV head: the element-wise maximum over its query heads.
+
+    NOT in the paper (its index sets are per head, Sec. 4.1): a labelled variant for
+    grouped-query attention in which the heads that share a KV head also share ONE index set,
+    so that a gathered K/V row serves the whole group.  A position is ranked by the largest
+    float32 logit any head of the group gives it; top-k, dilation and the set are then built
+    exactly as for a single head.  Every winner is in the own top-k of at least one head
+    (the head that attains its maximum), which is what the tests pin.
+    """
+    return np.maximum.reduce([rank_logits(a) for a in per_head])
+
+
 # ------------------------------------------------------------- Eq. (10): neighbour dilation
 def dilate(s_star: np.ndarray, m: int, r: int, t_anchor: int) -> np.ndarray:
     """S^ = S* ∪ ⋃_{i<m} { p_i + j : -r <= j <= r }, clipped to [0, t_anchor)  (Eq. 10).
@@ -221,6 +234,7 @@ class Schedule:
     psaw_alpha: float = 1.0
     psaw_layer_start: int = 0      # l_s, 1-based; 0 = no sliding window
     num_layers: int = 1            # N of Eq. 11
+    group_sets: bool = False       # labelled variant, NOT in the paper: one set per KV head (see group_logits)
 
     def k_for(self, b: int) -> int:
         return int(self.top_k_per_seq[b]) if self.top_k_per_seq is not None else self.top_k
@@ -335,12 +349,46 @@ class PrhsOracle:
         leader = layer % self.s.layer_group == 0
         out = {"y": {}, "lse": {}, "delta": {}, "set": {}, "s_star": {}, "lse_full": {},
                "scores32": {}, "retrieved": {}, "ref": {}, "s_hat": {}}
+        if self.s.group_sets and self.s.sim_threshold is not None:
+            raise ValueError("the cosine gate is per head: not defined with group-shared sets")
+        group_plan: dict = {}           # (b, kv) -> plan of the group (group_sets only)
         for (b, h) in units:
             t = int(seq_lens[b])
             kv = h // self.gq
-            blk, set_id, own, ref = self._plan(layer, step, b, h, q[b, h], override_ref)
             a = None
-            if own:
+            if self.s.group_sets:
+                # the group's first head carries the block state; one plan and one retrieval per group
+                h0 = kv * self.gq
+                first = (b, kv) not in group_plan
+                if first:
+                    blk, set_id, own, ref = self._plan(layer, step, b, h0, q[b, h0], override_ref)
+                    if own:
+                        heads = [dense_scores(q[b, h0 + j], K[b, kv], t) for j in range(self.gq)]
+                        ag = group_logits(heads)
+                        if override_s_star is not None and (b, h0) in override_s_star:
+                            s_star = np.asarray(override_s_star[(b, h0)], dtype=np.int64)
+                        else:
+                            s_star = topk_middle(ag, t, self.s.sinks, self.s.window, self.s.k_for(b),
+                                                 self.s.psaw_for(layer, t))
+                        blk.sets.append((s_star, dilate(s_star, self.s.m_for(b), self.s.dilate_r, t)))
+                        group_plan[(b, kv)] = (blk, set_id, own, ref, ag)
+                    else:
+                        group_plan[(b, kv)] = (blk, set_id, own, ref, None)
+                    if leader:
+                        blk.queries.append(np.array(q[b, h0], dtype=np.float64))
+                        blk.set_of_pos.append(set_id)
+                        self.last[(layer // self.s.layer_group, b, h0)] = (step, set_id, own)
+                blk, set_id, own, ref, ag = group_plan[(b, kv)]
+                if own:
+                    out["s_star"][(b, h)] = blk.sets[set_id][0]
+                    out["s_hat"][(b, h)] = blk.sets[set_id][1]
+                    out["scores32"][(b, h)] = ag
+                    self.retrievals += 1
+                if leader:
+                    out["ref"][(b, h)] = ref
+            else:
+                blk, set_id, own, ref = self._plan(layer, step, b, h, q[b, h], override_ref)
+            if own and not self.s.group_sets:
                 a = dense_scores(q[b, h], K[b, kv], t)
                 if override_s_star is not None and (b, h) in override_s_star:
                     s_star = np.asarray(override_s_star[(b, h)], dtype=np.int64)
@@ -352,7 +400,7 @@ class PrhsOracle:
                 out["s_hat"][(b, h)] = blk.sets[-1][1]
                 out["scores32"][(b, h)] = rank_logits(a)
                 self.retrievals += 1
-            if leader:
+            if leader and not self.s.group_sets:
                 g = layer // self.s.layer_group
                 blk.queries.append(np.array(q[b, h], dtype=np.float64))
                 blk.set_of_pos.append(set_id)

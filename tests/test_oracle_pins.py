@@ -574,3 +574,62 @@ def test_schedule_sampled_units_match_full_run():
         b = part.decode_step(0, n, q[0, n], K[0], V[0], t, units=[(1, 3)])
         assert list(b["y"]) == [(1, 3)]
         assert np.array_equal(a["y"][(1, 3)], b["y"][(1, 3)])
+
+
+# ------------------------------------------------ labelled variant: one set per KV head (not in the paper)
+def test_group_sets_properties():
+    """Group-shared sets (ranking by the maximum logit over the heads of a KV group).
+
+    What fixes the rule without retyping it: with one head per KV head it IS the per-head
+    method; heads with identical queries reproduce the per-head set; every winner lies in the
+    own top-k of at least one head of the group (the head attaining its maximum has fewer than
+    k positions above it); and no head retains more mass over the group's undilated set than
+    over its own top-k of the same size (Sec. 3.2: top-k maximises the retained mass).
+    """
+    q, K, V = _stack(31, layers=2, Hq=8, Hkv=2)
+    kw = dict(top_k=16, window=8, sinks=2, refresh_interval=2, layer_group=2, dilate_r=0)
+    grp = O.PrhsOracle(O.Schedule(group_sets=True, **kw), 8, 2)
+    own = O.PrhsOracle(O.Schedule(**kw), 8, 2)
+    for n in range(3):
+        t = np.array([200 + n + 1, 170 + n + 1])
+        for layer in range(2):
+            a = grp.decode_step(layer, n, q[layer, n], K[layer], V[layer], t)
+            b = own.decode_step(layer, n, q[layer, n], K[layer], V[layer], t)
+            for (bb, h), C in a["set"].items():
+                h0 = (h // 4) * 4
+                assert np.array_equal(C, a["set"][(bb, h0)])                     # one set per group
+                y, _ = O.attn_over_set(q[layer, n, bb, h], K[layer, bb, h // 4], V[layer, bb, h // 4], C)
+                assert np.allclose(a["y"][(bb, h)], y)                          # own q, shared rows
+                if layer == 0 and n % 2 == 0:
+                    union = set()
+                    for j in range(4):
+                        union |= set(b["s_star"][(bb, h0 + j)].tolist())
+                    assert set(a["s_star"][(bb, h)].tolist()) <= union
+                    assert a["delta"][(bb, h)] >= b["delta"][(bb, h)] - 1e-12
+    assert grp.retrieval_ratio() == own.retrieval_ratio() == pytest.approx(1 / 3)
+    # one head per KV head: the variant is the method itself
+    q1, K1, V1 = _stack(32, layers=1, Hq=2, Hkv=2)
+    g1 = O.PrhsOracle(O.Schedule(top_k=12, window=8, sinks=2, refresh_interval=2, group_sets=True), 2, 2)
+    p1 = O.PrhsOracle(O.Schedule(top_k=12, window=8, sinks=2, refresh_interval=2), 2, 2)
+    for n in range(3):
+        t = np.array([150 + n, 190 + n])
+        x, y = g1.decode_step(0, n, q1[0, n], K1[0], V1[0], t), p1.decode_step(0, n, q1[0, n], K1[0], V1[0], t)
+        for u in x["set"]:
+            assert np.array_equal(x["set"][u], y["set"][u]) and np.array_equal(x["y"][u], y["y"][u])
+    # identical queries inside a group: the group's set is every head's own set
+    qs = q[0, 0].copy()
+    qs[:, 1:4] = qs[:, 0:1]
+    qs[:, 5:8] = qs[:, 4:5]
+    t = np.array([201, 171])
+    x = O.PrhsOracle(O.Schedule(group_sets=True, **kw), 8, 2).decode_step(0, 0, qs, K[0], V[0], t)
+    y = O.PrhsOracle(O.Schedule(**kw), 8, 2).decode_step(0, 0, qs, K[0], V[0], t)
+    for u in x["set"]:
+        assert np.array_equal(x["s_star"][u], y["s_star"][u])
+    # sampled units give the same result as a full run
+    part = O.PrhsOracle(O.Schedule(group_sets=True, **kw), 8, 2).decode_step(0, 0, q[0, 0], K[0], V[0], t,
+                                                                              units=[(1, 6)])
+    full = O.PrhsOracle(O.Schedule(group_sets=True, **kw), 8, 2).decode_step(0, 0, q[0, 0], K[0], V[0], t)
+    assert np.array_equal(part["set"][(1, 6)], full["set"][(1, 6)])
+    with pytest.raises(ValueError):
+        O.PrhsOracle(O.Schedule(group_sets=True, sim_threshold=0.8, **kw), 8, 2).decode_step(
+            0, 0, q[0, 0], K[0], V[0], t)
