@@ -95,6 +95,14 @@ typedef struct {
 #define PRHS_DILATE_ANCHOR 1u /* the retrieving (layer, step) also attends over the dilated set */
 #define PRHS_WANT_DELTA    2u /* prhs_decode_step fills out_delta (runs a dense log-sum-exp pass
                                  on every non-retrieving call: diagnostic, not the timed path)  */
+#define PRHS_GROUP_SETS    4u /* labelled variant, NOT in the paper (its sets are per head, Sec. 4.1):
+                                 the query heads that share a KV head share ONE index set.  A position
+                                 is ranked by the largest fp32 logit any head of the group gives it;
+                                 top-k, dilation and the set follow as for a single head; a gathered
+                                 K/V row then serves the whole group.  Outputs keep their [B][Hq]
+                                 shapes (the heads of a group receive the same set).  Not combinable
+                                 with the cosine gate (PRHS_ERR_UNSUPPORTED).  No effect when
+                                 num_q_heads == num_kv_heads. */
 
 /* The knobs of CIS (Sec. 4.1; defaults Sec. 5.1) plus the cross-layer group size. */
 typedef struct {

@@ -20,6 +20,7 @@ STATUS_NAMES = {0: "PRHS_OK", 1: "PRHS_ERR_INVALID_ARG", 2: "PRHS_ERR_UNSUPPORTE
                 7: "PRHS_ERR_DEVICE_FLAG"}
 PRHS_DILATE_ANCHOR = 1
 PRHS_WANT_DELTA = 2
+PRHS_GROUP_SETS = 4
 PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TIMEOUT = 1, 2, 4, 8
 
 # every symbol include/prhs.h declares

@@ -471,6 +471,158 @@ __device__ __forceinline__ void mma_bf16_full(float (&d)[4], uint32_t a0, uint32
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// One 16-row stage of grouped attention: S = Q K^T for the heads on tile rows g and g + 8,
+// online softmax per row with a lazy reference exponent, O += P V.  v0..v3 say which of this
+// lane's four keys (rows 2tg, 2tg+1, 8+2tg, 9+2tg of the stage) are real.
+__device__ __forceinline__ void group_stage(uint32_t kt, uint32_t vt, const uint32_t (&aq)[8][4], bool v0, bool v1,
+                                            bool v2, bool v3, float (&o)[16][4], float& m0, float& l0, float& m1,
+                                            float& l1) {
+  const int lane = threadIdx.x & 31;
+  const int lm_mi = lane >> 3, lm_r = lane & 7;
+  const int vrow = (lm_mi & 1) * 8 + lm_r;
+  const float sc = kScale * kLog2e;
+  float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+  for (int pp = 0; pp < 4; ++pp) {
+    uint32_t bk0[4], bk1[4];
+    ldmatrix_x4(bk0, kt + lm_r * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+    ldmatrix_x4(bk1, kt + (8 + lm_r) * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
+    mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
+    mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
+    mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
+    mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
+  }
+  float x[2][4];   // [row half][key]
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {
+    x[hh][0] = v0 ? s[0][2 * hh] * sc : -INFINITY;
+    x[hh][1] = v1 ? s[0][2 * hh + 1] * sc : -INFINITY;
+    x[hh][2] = v2 ? s[1][2 * hh] * sc : -INFINITY;
+    x[hh][3] = v3 ? s[1][2 * hh + 1] * sc : -INFINITY;
+  }
+  // ---- online softmax per row (lazy reference exponent, as in the gathered kernel)
+  float mx0 = fmaxf(fmaxf(x[0][0], x[0][1]), fmaxf(x[0][2], x[0][3]));
+  float mx1 = fmaxf(fmaxf(x[1][0], x[1][1]), fmaxf(x[1][2], x[1][3]));
+  if (__any_sync(0xffffffffu, mx0 > m0 + 8.f || mx1 > m1 + 8.f)) {
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);
+    const float c0 = (n0 == -INFINITY) ? 1.f : exp2f(m0 - n0);
+    const float c1 = (n1 == -INFINITY) ? 1.f : exp2f(m1 - n1);
+    m0 = n0; m1 = n1;
+    l0 *= c0; l1 *= c1;
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c1; o[nt][3] *= c1; }
+  }
+  float pw[2][4];
+#pragma unroll
+  for (int k4 = 0; k4 < 4; ++k4) {
+    pw[0][k4] = (m0 == -INFINITY) ? 0.f : exp2f(x[0][k4] - m0);
+    pw[1][k4] = (m1 == -INFINITY) ? 0.f : exp2f(x[1][k4] - m1);
+  }
+  l0 += (pw[0][0] + pw[0][1]) + (pw[0][2] + pw[0][3]);
+  l1 += (pw[1][0] + pw[1][1]) + (pw[1][2] + pw[1][3]);
+  const uint32_t a0 = pack_bf16x2(pw[0][0], pw[0][1]), a1 = pack_bf16x2(pw[1][0], pw[1][1]);
+  const uint32_t a2 = pack_bf16x2(pw[0][2], pw[0][3]), a3 = pack_bf16x2(pw[1][2], pw[1][3]);
+  // ---- O += P V
+#pragma unroll
+  for (int np = 0; np < 8; ++np) {
+    uint32_t bv[4];
+    ldmatrix_x4_trans(bv, vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
+    mma_bf16_full(o[2 * np], a0, a1, a2, a3, bv[0], bv[1]);
+    mma_bf16_full(o[2 * np + 1], a0, a1, a2, a3, bv[2], bv[3]);
+  }
+}
+
+// Epilogue of the grouped kernels: combine the warps of the CTA per head, then either write
+// the result (one split) or the split's partials; the last CTA of the (b, kvh) to arrive merges
+// the splits of the group's heads (ticket on the group's first head, no waiting).  The ring
+// is free by now and holds [warp][head][128] floats.
+__device__ __forceinline__ void group_epilogue(const AttnParams& p, unsigned char* g_smem, int b, int head0, int gq,
+                                               int split, float (&o)[16][4], float m0, float l0, float m1,
+                                               float l1) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  __syncthreads();
+  float* sm_o = reinterpret_cast<float*>(g_smem);                       // 4 x 16 x 128 floats = 32 KB
+  float* sm_m = sm_o + kTWarps * 16 * kHeadDim;                         // [warp][16]
+  float* sm_l = sm_m + kTWarps * 16;
+  __shared__ bool is_last;
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt) {
+    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
+    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g + 8) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][2], o[nt][3]);
+  }
+  if (tg == 0) {
+    sm_m[warp * 16 + g] = m0; sm_l[warp * 16 + g] = l0;
+    sm_m[warp * 16 + g + 8] = m1; sm_l[warp * 16 + g + 8] = l1;
+  }
+  __syncthreads();
+  auto finish = [&](int unit, float acc, float M, float L) {
+    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+    if (tid == 0) {
+      const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+      if (p.out_lse) p.out_lse[unit] = lse;
+      if (p.out_delta) p.out_delta[unit] = L > 0.f ? -expm1f(lse - p.lse_full[unit]) : 1.f;
+    }
+  };
+  for (int j = 0; j < gq; ++j) {
+    const int unit = b * p.num_q_heads + head0 + j;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w * 16 + j]);
+    float acc = 0.f, L = 0.f;
+    if (M != -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < kTWarps; ++w) {
+        const float scw = exp2f(sm_m[w * 16 + j] - M);
+        acc = fmaf(sm_o[(w * 16 + j) * kHeadDim + tid], scw, acc);
+        L = fmaf(sm_l[w * 16 + j], scw, L);
+      }
+    }
+    if (p.splits == 1) {
+      finish(unit, acc, M, L);
+    } else {
+      float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
+      part[tid] = acc;
+      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
+    }
+  }
+  if (p.splits == 1) return;
+  __threadfence();
+  __syncthreads();
+  const int tunit = b * p.num_q_heads + head0;      // ticket slot: the group's first head
+  if (tid == 0) {
+    const unsigned int ticket = atomicAdd(p.tickets + tunit, 1u);
+    is_last = (ticket == (unsigned int)p.splits - 1u);
+    if (is_last) p.tickets[tunit] = 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int j = 0; j < gq; ++j) {
+    const int unit = tunit + j;
+    const float* base = p.partials + (long long)unit * p.splits * kPartStride;
+    float M = -INFINITY;
+    for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
+    float acc = 0.f, L = 0.f;
+    if (M != -INFINITY) {
+      for (int sp = 0; sp < p.splits; ++sp) {
+        const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
+        acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
+        L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
+      }
+    }
+    finish(unit, acc, M, L);
+  }
+}
+
 __global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p) {
   extern __shared__ __align__(128) unsigned char g_smem[];
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
@@ -542,148 +694,18 @@ __global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p)
 #pragma unroll
   for (int j = 0; j < kTStages - 1; ++j) issue(j);
 
-  const float sc = kScale * kLog2e;
-  const int lm_mi = lane >> 3, lm_r = lane & 7;
-  const int vrow = (lm_mi & 1) * 8 + lm_r;
   for (int i = 0; i < nstages; ++i) {
     cp_async_wait<kTStages - 2>();
     __syncwarp();
     issue(i + kTStages - 1);
     const uint32_t kt = ring + (uint32_t)(i % kTStages) * kTStageBytes;
-    const uint32_t vt = kt + kTTileBytes;
     const int pos0 = start + i * kTStageRows;
-    // ---- S = Q K^T for the whole group
-    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-    for (int pp = 0; pp < 4; ++pp) {
-      uint32_t bk0[4], bk1[4];
-      ldmatrix_x4(bk0, kt + lm_r * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
-      ldmatrix_x4(bk1, kt + (8 + lm_r) * kRowBytes + (((4 * pp + lm_mi) ^ (lm_r & 7)) << 4));
-      mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
-      mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
-      mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
-      mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
-    }
     // keys of this lane: pos0 + 2tg, +1 (n-tile 0) and pos0 + 8 + 2tg, +1 (n-tile 1)
-    const bool v0 = pos0 + 2 * tg < end, v1 = pos0 + 2 * tg + 1 < end;
-    const bool v2 = pos0 + 8 + 2 * tg < end, v3 = pos0 + 9 + 2 * tg < end;
-    float x[2][4];   // [row half][key]
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      x[hh][0] = v0 ? s[0][2 * hh] * sc : -INFINITY;
-      x[hh][1] = v1 ? s[0][2 * hh + 1] * sc : -INFINITY;
-      x[hh][2] = v2 ? s[1][2 * hh] * sc : -INFINITY;
-      x[hh][3] = v3 ? s[1][2 * hh + 1] * sc : -INFINITY;
-    }
-    // ---- online softmax per row (lazy reference exponent, as in the gathered kernel)
-    float mx0 = fmaxf(fmaxf(x[0][0], x[0][1]), fmaxf(x[0][2], x[0][3]));
-    float mx1 = fmaxf(fmaxf(x[1][0], x[1][1]), fmaxf(x[1][2], x[1][3]));
-    if (__any_sync(0xffffffffu, mx0 > m0 + 8.f || mx1 > m1 + 8.f)) {
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);
-      const float c0 = (n0 == -INFINITY) ? 1.f : exp2f(m0 - n0);
-      const float c1 = (n1 == -INFINITY) ? 1.f : exp2f(m1 - n1);
-      m0 = n0; m1 = n1;
-      l0 *= c0; l1 *= c1;
-#pragma unroll
-      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c1; o[nt][3] *= c1; }
-    }
-    float pw[2][4];
-#pragma unroll
-    for (int k4 = 0; k4 < 4; ++k4) {
-      pw[0][k4] = (m0 == -INFINITY) ? 0.f : exp2f(x[0][k4] - m0);
-      pw[1][k4] = (m1 == -INFINITY) ? 0.f : exp2f(x[1][k4] - m1);
-    }
-    l0 += (pw[0][0] + pw[0][1]) + (pw[0][2] + pw[0][3]);
-    l1 += (pw[1][0] + pw[1][1]) + (pw[1][2] + pw[1][3]);
-    const uint32_t a0 = pack_bf16x2(pw[0][0], pw[0][1]), a1 = pack_bf16x2(pw[1][0], pw[1][1]);
-    const uint32_t a2 = pack_bf16x2(pw[0][2], pw[0][3]), a3 = pack_bf16x2(pw[1][2], pw[1][3]);
-    // ---- O += P V
-#pragma unroll
-    for (int np = 0; np < 8; ++np) {
-      uint32_t bv[4];
-      ldmatrix_x4_trans(bv, vt + vrow * kRowBytes + (((2 * np + (lm_mi >> 1)) ^ (vrow & 7)) << 4));
-      mma_bf16_full(o[2 * np], a0, a1, a2, a3, bv[0], bv[1]);
-      mma_bf16_full(o[2 * np + 1], a0, a1, a2, a3, bv[2], bv[3]);
-    }
+    group_stage(kt, kt + kTTileBytes, aq, pos0 + 2 * tg < end, pos0 + 2 * tg + 1 < end, pos0 + 8 + 2 * tg < end,
+                pos0 + 9 + 2 * tg < end, o, m0, l0, m1, l1);
   }
   cp_async_wait<0>();
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-
-  // ---- combine the warps of this CTA; the ring is free now and holds [warp][head][128] floats
-  __syncthreads();
-  float* sm_o = reinterpret_cast<float*>(g_smem);                       // 4 x 16 x 128 floats = 32 KB
-  float* sm_m = sm_o + kTWarps * 16 * kHeadDim;                         // [warp][16]
-  float* sm_l = sm_m + kTWarps * 16;
-  __shared__ bool is_last;
-#pragma unroll
-  for (int nt = 0; nt < 16; ++nt) {
-    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
-    *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g + 8) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][2], o[nt][3]);
-  }
-  if (tg == 0) {
-    sm_m[warp * 16 + g] = m0; sm_l[warp * 16 + g] = l0;
-    sm_m[warp * 16 + g + 8] = m1; sm_l[warp * 16 + g + 8] = l1;
-  }
-  __syncthreads();
-  for (int j = 0; j < gq; ++j) {
-    const int unit = b * p.num_q_heads + head0 + j;
-    float M = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w * 16 + j]);
-    float acc = 0.f, L = 0.f;
-    if (M != -INFINITY) {
-#pragma unroll
-      for (int w = 0; w < kTWarps; ++w) {
-        const float scw = exp2f(sm_m[w * 16 + j] - M);
-        acc = fmaf(sm_o[(w * 16 + j) * kHeadDim + tid], scw, acc);
-        L = fmaf(sm_l[w * 16 + j], scw, L);
-      }
-    }
-    if (p.splits == 1) {
-      p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-      if (tid == 0 && p.out_lse) p.out_lse[unit] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-    } else {
-      float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
-      part[tid] = acc;
-      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
-    }
-  }
-  if (p.splits == 1) return;
-  // ---- the last CTA of this (b, kvh) merges the split partials of the group's heads
-  __threadfence();
-  __syncthreads();
-  const int tunit = b * p.num_q_heads + head0;      // ticket slot: the group's first head
-  if (tid == 0) {
-    const unsigned int ticket = atomicAdd(p.tickets + tunit, 1u);
-    is_last = (ticket == (unsigned int)p.splits - 1u);
-    if (is_last) p.tickets[tunit] = 0u;
-  }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  for (int j = 0; j < gq; ++j) {
-    const int unit = tunit + j;
-    const float* base = p.partials + (long long)unit * p.splits * kPartStride;
-    float M = -INFINITY;
-    for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
-    float acc = 0.f, L = 0.f;
-    if (M != -INFINITY) {
-      for (int sp = 0; sp < p.splits; ++sp) {
-        const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
-        acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
-        L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
-      }
-    }
-    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-    if (tid == 0 && p.out_lse) p.out_lse[unit] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-  }
+  group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1);
 }
 
 // ------------------------------------------------------- retrieval scoring, ring variant
@@ -703,8 +725,35 @@ struct ScoreParams {
   float2* part_ml;        // [B][Hq][splits]
   int splits, num_q_heads, group_size;
   const int* need;        // [B][Hq] or nullptr: score only KV heads with a query head that retrieves
+  int group_max;          // 1: write max over the group's heads to the row of its first head only
   uint32_t* flags;
 };
+
+// Group-shared ranking logits: the maximum over the heads on the tile rows (g and g + 8 of every
+// lane quad) of the four logits a lane holds, stored by the lanes of row 0 into the row of the
+// group's first head.  s[nt][2 hh + c]: n-tile nt, row half hh, column c.
+__device__ __forceinline__ void store_group_max(const float (&s)[2][4], bool has0, bool has1, float* dst,
+                                                int pos0, int end) {
+  const int lane = threadIdx.x & 31;
+  const int g = lane >> 2, tg = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    float v[2];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      float x = fmaxf(has0 ? s[nt][c] : -INFINITY, has1 ? s[nt][2 + c] : -INFINITY);
+      x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
+      x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 8));
+      x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 16));
+      v[c] = x * kScale;
+    }
+    const int key0 = pos0 + 8 * nt + 2 * tg;
+    if (g == 0) {
+      if (key0 + 1 < end) *reinterpret_cast<float2*>(dst + key0) = make_float2(v[0], v[1]);
+      else if (key0 < end) dst[key0] = v[0];
+    }
+  }
+}
 
 __global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
   extern __shared__ __align__(128) unsigned char g_smem[];
@@ -797,12 +846,14 @@ __global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
       mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
     }
     // lane (g, tg): head g -> s[nt][0..1], head g + 8 -> s[nt][2..3]; keys pos0 + 8 nt + 2 tg, +1
+    if (p.scores && p.group_max)
+      store_group_max(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       if (hh == 0 ? has0 : has1) {
         float& m = hh == 0 ? m0 : m1;
         float& l = hh == 0 ? l0 : l1;
-        float* dst = p.scores ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
+        float* dst = (p.scores && !p.group_max) ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
           const int key0 = pos0 + 8 * nt + 2 * tg;

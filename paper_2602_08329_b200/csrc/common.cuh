@@ -55,12 +55,14 @@ struct SetRef {
   const int* slot_of;     // [U] slot each unit uses this step, or nullptr = slot 0
   const int* own_of;      // [U] != 0 where the unit retrieved this step, or nullptr = own_all
   int star_stride, hat_stride, slots, own_all;
+  int share_gq;           // > 1: the heads of a KV group share the set stored for the group's first head
   int sinks, window;
   double psaw_c;          // sliding-window factor of this layer (0 = off)
 };
 
 // The unit's middle set M (ascending, unique) and its length.
 __device__ __forceinline__ const int* middle_of(const SetRef& r, int unit, int* n, int* stride) {
+  if (r.share_gq > 1) unit -= unit % r.share_gq;      // units are b * Hq + h and Hq is a multiple of the group
   const int slot = r.slot_of ? __ldg(r.slot_of + unit) : 0;
   const bool own = r.own_of ? (__ldg(r.own_of + unit) != 0) : (r.own_all != 0);
   const long long e = (long long)unit * r.slots + slot;

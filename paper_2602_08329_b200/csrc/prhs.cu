@@ -12,6 +12,7 @@
 
 #include "attn.cuh"
 #include "common.cuh"
+#include "attn_group.cuh"
 #include "score_tma.cuh"
 #include "select.cuh"
 
@@ -42,7 +43,7 @@ struct prhs_ctx {
   prhs_config cfg{};
   int device = 0, sm_count = 148;
   int gq = 1, num_groups = 1, max_m = 0, shat_cap = 0, idx_cap = 0, ld = 0, sort_cap = 2;
-  int cand_cap = 0, two_bitmaps = 0;
+  int cand_cap = 0, two_bitmaps = 0, last_share_gq = 1;
   int max_chunks = 1, attn_ctas_per_sm = 2;
   size_t sel_smem = 0;
   // workspaces (device)
@@ -150,6 +151,8 @@ prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
   if (s->top_k > ctx->cfg.max_k || s->window > ctx->cfg.max_window || s->sinks > ctx->cfg.max_sinks ||
       s->dilate_r > ctx->cfg.max_dilate_r || (s->dilate_m >= 0 && s->dilate_m > ctx->max_m))
     return fail(ctx, PRHS_ERR_CAPACITY, "schedule: budget exceeds the configured maximum");
+  if ((s->flags & PRHS_GROUP_SETS) && s->sim_threshold > -1.f)
+    return fail(ctx, PRHS_ERR_UNSUPPORTED, "schedule: the cosine gate is per head, group-shared sets are per KV head");
   return PRHS_OK;
 }
 
@@ -204,6 +207,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.num_q_heads = c->cfg.num_q_heads;
   sp.group_size = c->gq;
   sp.need = need;
+  sp.group_max = (sched && (sched->flags & PRHS_GROUP_SETS) && c->gq > 1) ? 1 : 0;
   sp.flags = c->flags;
   bool tma_done = false;
   if (c->encode_tiled) {
@@ -277,6 +281,12 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
     dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
     LaunchScope ls(c, PRHS_KIND_ATTN_DENSE, st);
     dense_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
+  } else if (!idx && fs.share_gq > 1) {
+    // group-shared sets: one CTA column per KV head, a gathered row serves the whole group
+    p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
+    dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
+    LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
+    gather_group_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   } else {
     dim3 grid(p.splits, c->cfg.num_q_heads, batch);
     LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
@@ -348,10 +358,11 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   p.sort_cap = c->sort_cap;
   p.cand_cap = c->cand_cap;
   p.two_bitmaps = c->two_bitmaps;
+  p.unit_mul = ((s->flags & PRHS_GROUP_SETS) && c->gq > 1) ? c->gq : 1;
   {
     // One CTA of 512 threads per unit (two per SM).  256 threads measured slower on every
     // configuration but one (the kernel is a chain of short phases; wide CTAs shorten it).
-    const int units = batch * c->cfg.num_q_heads;
+    const int units = batch * c->cfg.num_q_heads / p.unit_mul;
     const int threads = kSelMaxThreads;
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
     select_kernel<<<units, threads, c->sel_smem, st>>>(p);
@@ -359,6 +370,7 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
   PRHS_CUDA(c, cudaGetLastError());
   if (!need) c->anchor_step[g] = step;
   c->last_layer_group = s->layer_group;
+  c->last_share_gq = p.unit_mul;
   return PRHS_OK;
 }
 
@@ -392,6 +404,7 @@ prhs_status pick_middle(prhs_ctx* c, int layer, int step, const prhs_schedule* s
   fs->star_stride = c->cfg.max_k;
   fs->hat_stride = c->shat_cap;
   fs->slots = c->slots;
+  fs->share_gq = ((s->flags & PRHS_GROUP_SETS) && c->gq > 1) ? c->gq : 1;
   fs->sinks = s->sinks;
   fs->window = s->window;
   fs->psaw_c = psaw_factor(c, s, layer);
@@ -491,6 +504,8 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_group_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
   if (e == cudaSuccess)
@@ -902,8 +917,9 @@ prhs_status prhs_get_shared_set(prhs_ctx* ctx, int32_t layer, int32_t batch, int
     PRHS_CUDA(ctx, cudaStreamSynchronize(st));
   }
   const size_t mk = ctx->cfg.max_k, hc = ctx->shat_cap, SL = ctx->slots;
+  const size_t share = (size_t)std::max(ctx->last_share_gq, 1);   // group-shared sets live with the group's first head
   for (size_t u = 0; u < n; ++u) {
-    const size_t e = u * SL + (size_t)slot[u];
+    const size_t e = (u - u % share) * SL + (size_t)slot[u];
     if (host_s_star)
       PRHS_CUDA(ctx, cudaMemcpyAsync(host_s_star + u * mk, ctx->sstar_desc + state_off(ctx, g, mk) + e * mk,
                                      mk * sizeof(int), cudaMemcpyDeviceToHost, st));

@@ -226,12 +226,14 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
       // the tile has been read into registers: hand the slot back to the producer
       __syncwarp();
       if (lane == 0) mbar_arrive(bar0 + 8 * (kSTStages + slot));
+      if (p.scores && p.group_max)
+        store_group_max(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         if (hh == 0 ? has0 : has1) {
           float& m = hh == 0 ? m0 : m1;
           float& l = hh == 0 ? l0 : l1;
-          float* dst = p.scores ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
+          float* dst = (p.scores && !p.group_max) ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt) {
             const int key0 = pos0 + 8 * nt + 2 * tg;

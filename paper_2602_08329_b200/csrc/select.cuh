@@ -53,7 +53,8 @@ struct SelectParams {
   uint32_t* flags;
   int sort_cap;             // power of two >= max_k: most entries the sort takes
   int cand_cap;             // candidate list entries (8 bytes each), >= sort_cap
-  int two_bitmaps;          // room for two position bitmaps behind the sorted entries
+  int two_bitmaps;          // room for two position bitmaps
+  int unit_mul;             // 1, or the group size when one CTA selects for a whole KV group (its first head's rows)
 };
 
 // Exclusive block scan of one int per thread; returns the exclusive prefix, *total gets the sum.
@@ -387,7 +388,7 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
   uint32_t* ws = misc + 8;                                                    // scan scratch (68 words)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x;
-  const int unit = blockIdx.x;
+  const int unit = blockIdx.x * p.unit_mul;
   if (p.need != nullptr && __ldg(p.need + unit) == 0) return;     // this head shares: no retrieval
   const long long sunit = (long long)unit * p.slots + (p.slot_of ? __ldg(p.slot_of + unit) : 0);
   const int b = unit / p.num_q_heads;
@@ -405,12 +406,12 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
   const int nb4 = (n - a0) >> 2;
   const float4* g4 = reinterpret_cast<const float4*>(g + a0);
 
-  // full-softmax log-sum-exp from the scoring pass' per-chunk partials
-  if (warp == 1) {
+  // full-softmax log-sum-exp from the scoring pass' per-chunk partials (of every head of the group)
+  for (int j = warp; j < p.unit_mul; j += (nt >> 5)) {
     float mm = -INFINITY, ll = 0.f;
     const int nch = p.chunk_rows > 0 ? min(p.nchunks, (t + p.chunk_rows - 1) / p.chunk_rows) : p.nchunks;
     for (int c = lane; c < nch; c += 32) {
-      const float2 x = p.part_ml[(long long)unit * p.nchunks + c];
+      const float2 x = p.part_ml[(long long)(unit + j) * p.nchunks + c];
       ml_combine(mm, ll, x.x, x.y);
     }
 #pragma unroll
@@ -421,8 +422,8 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
     }
     if (lane == 0) {
       const float lse = (ll > 0.f) ? (mm + log2f(ll)) * kLn2 : -INFINITY;
-      p.lse_full[unit] = lse;
-      if (p.out_lse_full) p.out_lse_full[unit] = lse;
+      p.lse_full[unit + j] = lse;
+      if (p.out_lse_full) p.out_lse_full[unit + j] = lse;
     }
   }
   if (tid == 0) {
@@ -656,11 +657,13 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
   for (int e = tid; e < p.max_k; e += nt) {
     const int v = e < kk ? (int)(0xffffffffu - (uint32_t)(cand[e] & 0xffffffffull)) : -1;
     sd[e] = v;
-    if (p.out_idx) p.out_idx[(long long)unit * p.max_k + e] = v;
+    if (p.out_idx)
+      for (int j = 0; j < p.unit_mul; ++j) p.out_idx[(long long)(unit + j) * p.max_k + e] = v;
   }
   if (tid == 0) {
     p.n_star[sunit] = kk;
-    if (p.out_count) p.out_count[unit] = kk;
+    if (p.out_count)
+      for (int j = 0; j < p.unit_mul; ++j) p.out_count[unit + j] = kk;
   }
 
   // ---- ascending S*, and the dilated S^ (Eq. 10), through position bitmaps

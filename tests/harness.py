@@ -112,21 +112,23 @@ class _HostSlices:
 
 
 def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, want_delta=True,
-                        paged=False, check_scores=True):
+                        paged=False, check_scores=True, group_sets=False):
     """Drive prhs_decode_step over the workload's schedule and compare sampled (b, h) units.
 
     The oracle follows the same schedule.  Where the GPU retrieved, its S* is first checked
     for legality against the oracle's own top-k (near-ties at the k-th logit only) and then
     handed to the oracle as an override, so that every later comparison in the block
     (dilation, shared sets, attention, delta) is exact.
+    `group_sets` runs the labelled variant with one set per KV head (ranking by the group's
+    maximum logit) on both sides.
     Returns a dict of summary statistics.
     """
     layers = list(range(w.layers)) if layers is None else layers
     steps = w.steps if steps is None else steps
     ctx = make_ctx(w)
-    flags = P.PRHS_WANT_DELTA if want_delta else 0
+    flags = (P.PRHS_WANT_DELTA if want_delta else 0) | (P.PRHS_GROUP_SETS if group_sets else 0)
     sched = make_sched(w, device, flags=flags)
-    osched = oracle_sched(w)
+    osched = oracle_sched(w, group_sets=group_sets)
     orc = O.PrhsOracle(osched, w.q_heads, w.kv_heads)
     q_all = W.make_queries(w, device)
     kv = {l: (k, v) for l, k, v in W.make_layer_kv(w, device, layers=layers)}
@@ -199,7 +201,11 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                         continue
                     t = int(t_host[b])
                     where = f"layer {l} step {n} unit ({b},{h})"
-                    a = O.dense_scores(qh[b, h], Ks[b, h // gq], t)
+                    hs = h - h % gq if group_sets else h        # whose rows hold the set and the logits
+                    if group_sets:
+                        a = O.group_logits([O.dense_scores(qh[b, hs + j], Ks[b, h // gq], t) for j in range(gq)])
+                    else:
+                        a = O.dense_scores(qh[b, h], Ks[b, h // gq], t)
                     a32 = O.rank_logits(a)
                     want = O.topk_middle(a, t, w.sinks, w.window, osched.k_for(b), osched.psaw_for(l, t))
                     got = s_star[b, h, : int(n_star[b, h])].numpy().astype(np.int64)
@@ -207,9 +213,9 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                     check_topk_legal(a32, got, want, where)
                     stats["near_tie_sets"] += int(before > 0)
                     if check_scores:
-                        sg = scores[b, h, :t].numpy()
+                        sg = scores[b, hs, :t].numpy()
                         assert np.allclose(sg, a32, atol=1e-4, rtol=1e-5), f"{where}: logits differ"
-                    over_s[(b, h)] = got          # legal: the oracle adopts it
+                    over_s[(b, hs)] = got         # legal: the oracle adopts it
             ref = orc.decode_step(l, n, qh, Ks, Vs, t_host.numpy(), units=units, want_delta=want_delta,
                                   override_s_star=over_s, override_ref=over_ref)
             for (b, h) in units:

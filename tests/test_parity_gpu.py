@@ -463,3 +463,41 @@ def test_radius_sweep_cells_small():
     c40 = RS.run_cell(w, dev, k, v, q, 4, 0)
     assert c40["beta_mean"] >= -1e-5        # without dilation a shared set never beats the step's own top-k
     assert c40["cov_mean"] <= c4["cov_mean"] + 1e-9
+
+
+# ------------------------------------------------ labelled variant: one index set per KV head
+@pytest.mark.gpu
+@pytest.mark.parametrize("hq,hkv,paged", [(8, 2, False), (16, 1, False), (12, 4, True), (4, 4, False)])
+def test_group_sets_schedule(cuda_device, hq, hkv, paged):
+    # group-shared sets (ranking by the group's maximum logit), cross-layer groups and a
+    # sliding window on the top layers; the (4, 4) case has one head per KV head, where the
+    # variant is the method itself
+    w = small(layers=4, layer_group=2, steps=5, refresh=2, q_heads=hq, kv_heads=hkv, context=2400, seed=41,
+              psaw_layer_start=3, page_size=16 if paged else 0)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=True)
+    assert st["checked"] == 4 * 5 * w.batch * w.q_heads
+    assert not st["select_fallback"]
+
+
+@pytest.mark.gpu
+def test_group_sets_rejects_cosine_gate(cuda_device):
+    w = small(q_heads=8, kv_heads=2, sim_threshold=0.8)
+    ctx = H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device, flags=P.PRHS_GROUP_SETS)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device), max_seq_len=w.capacity)
+    with pytest.raises(P.PrhsError) as e:
+        ctx.decode_step(0, 0, sched, q[0, 0].contiguous(), view, w.batch, out)
+    assert e.value.status == 2       # PRHS_ERR_UNSUPPORTED
+    ctx.close()
+
+
+@pytest.mark.gpu
+def test_group_sets_c3_slice_sampled(cuda_device):
+    # the Mistral-shaped stack at full per-layer size with group-shared sets
+    w = W.C3_MISTRAL.scaled(layers=8, steps=5, batch=4)
+    units = [(0, 0), (0, 3), (2, 21), (3, 31)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3, 4], group_sets=True)
+    assert st["checked"] == 4 * 5 * len(units)
