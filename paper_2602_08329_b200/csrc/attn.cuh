@@ -732,12 +732,13 @@ struct ScoreParams {
 // Group-shared ranking logits: the maximum over the heads on the tile rows (g and g + 8 of every
 // lane quad) of the four logits a lane holds, stored by the lanes of row 0 into the row of the
 // group's first head.  s[nt][2 hh + c]: n-tile nt, row half hh, column c.
-__device__ __forceinline__ void store_group_max(const float (&s)[2][4], bool has0, bool has1, float* dst,
+template <int NT>
+__device__ __forceinline__ void store_group_max(const float (&s)[NT][4], bool has0, bool has1, float* dst,
                                                 int pos0, int end) {
   const int lane = threadIdx.x & 31;
   const int g = lane >> 2, tg = lane & 3;
 #pragma unroll
-  for (int nt = 0; nt < 2; ++nt) {
+  for (int nt = 0; nt < NT; ++nt) {
     float v[2];
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
@@ -847,7 +848,7 @@ __global__ void __launch_bounds__(kTThreads) score_ring_kernel(ScoreParams p) {
     }
     // lane (g, tg): head g -> s[nt][0..1], head g + 8 -> s[nt][2..3]; keys pos0 + 8 nt + 2 tg, +1
     if (p.scores && p.group_max)
-      store_group_max(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
+      store_group_max<2>(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       if (hh == 0 ? has0 : has1) {

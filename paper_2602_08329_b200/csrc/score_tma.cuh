@@ -22,7 +22,8 @@
 
 namespace prhs {
 
-constexpr int kSTConsumers = 4;                         // consumer warps
+constexpr int kSTConsumers = 8;                         // consumer warps
+constexpr int kSTNT = 64 / (8 * kSTConsumers);          // 8-key MMA n-tiles per warp and stage
 constexpr int kSTThreads = (kSTConsumers + 1) * 32;     // + one producer warp
 constexpr int kSTStageRows = 64;                        // keys per stage
 constexpr int kSTHalfBytes = kSTStageRows * 128;        // one [64][64] bf16 box = 8 KB
@@ -183,7 +184,7 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
       }
     }
   } else {
-    // ---------------- consumers: 16 keys of every stage per warp
+    // ---------------- consumers: 8 kSTNT keys of every stage per warp
     const bool has0 = g < gq, has1 = g + 8 < gq;
     uint32_t aq[8][4];
     {
@@ -208,26 +209,30 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
         break;
       }
       const uint32_t kt = smem0 + slot * kSTStageBytes;
-      const int pos0 = start + j * kSTStageRows + warp * 16;
-      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      const int pos0 = start + j * kSTStageRows + warp * (8 * kSTNT);
+      float s[kSTNT][4];
+#pragma unroll
+      for (int nt = 0; nt < kSTNT; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
 #pragma unroll
       for (int pp = 0; pp < 4; ++pp) {
         // logical 16-byte chunk 4pp + lm_mi of the 256-byte row: half = chunk / 8, c = chunk % 8
         const int chunk = 4 * pp + lm_mi;
         const uint32_t hb = kt + (chunk >> 3) * kSTHalfBytes + (((chunk & 7) ^ lm_r) << 4);
-        uint32_t bk0[4], bk1[4];
-        ldmatrix_x4(bk0, hb + (warp * 16 + lm_r) * 128);
-        ldmatrix_x4(bk1, hb + (warp * 16 + 8 + lm_r) * 128);
-        mma_bf16_full(s[0], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk0[0], bk0[1]);
-        mma_bf16_full(s[1], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk1[0], bk1[1]);
-        mma_bf16_full(s[0], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk0[2], bk0[3]);
-        mma_bf16_full(s[1], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk1[2], bk1[3]);
+        uint32_t bk[kSTNT][4];
+#pragma unroll
+        for (int nt = 0; nt < kSTNT; ++nt) ldmatrix_x4(bk[nt], hb + (warp * (8 * kSTNT) + 8 * nt + lm_r) * 128);
+#pragma unroll
+        for (int nt = 0; nt < kSTNT; ++nt)
+          mma_bf16_full(s[nt], aq[2 * pp][0], aq[2 * pp][1], aq[2 * pp][2], aq[2 * pp][3], bk[nt][0], bk[nt][1]);
+#pragma unroll
+        for (int nt = 0; nt < kSTNT; ++nt)
+          mma_bf16_full(s[nt], aq[2 * pp + 1][0], aq[2 * pp + 1][1], aq[2 * pp + 1][2], aq[2 * pp + 1][3], bk[nt][2], bk[nt][3]);
       }
       // the tile has been read into registers: hand the slot back to the producer
       __syncwarp();
       if (lane == 0) mbar_arrive(bar0 + 8 * (kSTStages + slot));
       if (p.scores && p.group_max)
-        store_group_max(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
+        store_group_max<kSTNT>(s, has0, has1, p.scores + ((long long)b * p.num_q_heads + head0) * p.ld, pos0, end);
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         if (hh == 0 ? has0 : has1) {
@@ -235,7 +240,7 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
           float& l = hh == 0 ? l0 : l1;
           float* dst = (p.scores && !p.group_max) ? p.scores + ((long long)b * p.num_q_heads + head0 + g + 8 * hh) * p.ld : nullptr;
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt) {
+          for (int nt = 0; nt < kSTNT; ++nt) {
             const int key0 = pos0 + 8 * nt + 2 * tg;
             const float s0 = s[nt][2 * hh] * kScale, s1 = s[nt][2 * hh + 1] * kScale;
             if (key0 + 1 < end) {

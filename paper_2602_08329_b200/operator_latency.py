@@ -2,6 +2,7 @@
 
     python -m paper_2602_08329_b200.operator_latency            # Table-3 shapes
     python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C5 shapes
+    python -m paper_2602_08329_b200.operator_latency --configs --group-sets   # one set per KV head (variant)
 
 The paper (Sec. 5.4, Table 3) times one attention layer of LLaMA-2-7B-Chat (32 MHA heads,
 head_dim 128) in decode at batch 8 / 16 and 1k-4k cached tokens, token sparsity 1/8, block
@@ -29,7 +30,7 @@ PAPER_TABLE3_MS = {  # (batch, seqlen): (Flash, CPE-8, CPE-16) in ms on an A100 
 }
 
 
-def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6):
+def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6, group_sets: bool = False):
     """Median device time (us) of a dense step, a retrieval step and a sharing step."""
     w = w.scaled(layers=copies, steps=max(w.refresh, 2) + 1)
     table = None
@@ -49,7 +50,8 @@ def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6):
     ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
                     page_size=w.page_size)
     sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
-                            top_k_per_seq=None if kps is None else kps.to(dev))
+                            top_k_per_seq=None if kps is None else kps.to(dev),
+                            flags=P.PRHS_GROUP_SETS if group_sets else 0)
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     t0, t1 = W.seq_lens_at(w, 0).to(dev), W.seq_lens_at(w, 1).to(dev)
     views0 = [P.make_view(kv[l][0], kv[l][1], t0, page_table=table, max_seq_len=w.capacity) for l in range(copies)]
@@ -116,12 +118,12 @@ def table3(dev):
                   f"{am[8]:.1f} | {am[16]:.1f} | {r['dense_us'] / am[16]:.2f}x | {pf} / {p8} / {p16} |")
 
 
-def configs(dev):
+def configs(dev, group_sets=False):
     print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
           "mean set size | dense / amortised | sharing step GB/s logical / unique | retrieval step kernels us |")
     print("|---|---|---|---|---|---|---|---|---|")
     for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
-        r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 50000 else 2)
+        r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 50000 else 2, group_sets=group_sets)
         period = w.refresh * w.layer_group      # layer-steps per retrieval
         am = (r["refresh_us"] + (period - 1) * r["shared_us"]) / period
         gbs = [r[k] / (r["shared_us"] * 1e3) for k in ("logical_bytes", "unique_bytes")]
@@ -134,12 +136,17 @@ def configs(dev):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C5 shapes instead")
+    ap.add_argument("--group-sets", action="store_true",
+                    help="with --configs: the labelled variant with one index set per KV head (not in the paper)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
-    (configs if args.configs else table3)(dev)
+    if args.configs:
+        configs(dev, args.group_sets)
+    else:
+        table3(dev)
 
 
 if __name__ == "__main__":
