@@ -227,7 +227,11 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
 /* The same step for a caller whose per-step tensors live in HOST memory (contiguous cache
  * only).  Copies q, the new token's key and value rows and seq_lens host->device, writes
  * the rows into the cache at position t_b - 1, runs prhs_decode_step, copies the output
- * device->host and synchronises the stream before returning.
+ * device->host and synchronises the stream before returning.  When all five host buffers are
+ * pinned memory that the device can address (cudaHostAlloc / cudaHostRegister under unified
+ * addressing; q, k, v 16-byte aligned) the transfers are made by the kernels themselves: one
+ * launch reads q, the rows and the lengths from host memory, and the attention kernel stores
+ * the output into host_out.  Pageable buffers take cudaMemcpyAsync.  Results are identical.
  *   host_q [batch][Hq][128], host_new_k / host_new_v [batch][Hkv][128], host_out
  *   [batch][Hq][128]: bf16 host memory;  host_seq_lens [batch] int32 host memory.
  *   kv->k / kv->v are written (the view's const is cast away); kv->seq_lens must point to

@@ -974,6 +974,40 @@ __global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunk
   }
   lse_full[i] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
 }
+// One launch that takes a decode step's inputs straight from PINNED, device-mapped host memory:
+// the queries into the staging buffer, the new K and V rows into the cache at position t_b - 1,
+// the lengths into the device array.  Replaces four host-to-device copies and the append
+// kernel: the transfers are 16-byte loads over the host link, all in flight at once.
+// grid (batch, kIngestSplit), 256 threads.
+constexpr int kIngestSplit = 4;
+__global__ void __launch_bounds__(256)
+ingest_kernel(const uint4* __restrict__ host_q, const uint4* __restrict__ host_k, const uint4* __restrict__ host_v,
+              const int* __restrict__ host_lens, uint4* q_dev, __nv_bfloat16* k, __nv_bfloat16* v,
+              long long stride_outer, long long stride_head, int* lens_dev, int hq, int hkv) {
+  __shared__ int sh_t;
+  const int b = blockIdx.x;
+  if (threadIdx.x == 0) {
+    sh_t = host_lens[b];
+    if (blockIdx.y == 0) lens_dev[b] = sh_t;
+  }
+  __syncthreads();
+  const int t = sh_t;
+  const int nq = hq * 16, nk = hkv * 16;             // 16-byte items of this sequence
+  const int total = nq + 2 * nk;
+  for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < total; i += kIngestSplit * blockDim.x) {
+    if (i < nq) {
+      q_dev[(long long)b * nq + i] = host_q[(long long)b * nq + i];
+    } else if (t > 0) {
+      const int j = (i - nq) % nk, is_v = (i - nq) / nk;
+      const int kvh = j >> 4, c = j & 15;
+      const uint4 x = (is_v ? host_v : host_k)[(long long)b * nk + j];
+      __nv_bfloat16* dst = (is_v ? v : k) + (long long)b * stride_outer + (long long)kvh * stride_head +
+                           (long long)(t - 1) * kHeadDim + c * 8;
+      *reinterpret_cast<uint4*>(dst) = x;
+    }
+  }
+}
+
 
 // Write the new token's K and V rows at position t_b - 1 (contiguous cache).
 // grid (Hkv, B), 32 threads: lanes 0-15 copy the K row, lanes 16-31 the V row.

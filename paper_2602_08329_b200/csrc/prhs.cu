@@ -835,6 +835,41 @@ prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, co
   cudaStream_t st = as_stream(stream);
   const size_t qb = (size_t)batch * ctx->cfg.num_q_heads * kRowBytes;
   const size_t kb = (size_t)batch * ctx->cfg.num_kv_heads * kRowBytes;
+  // Pinned host buffers that the device can address (what cudaHostAlloc / cudaHostRegister give
+  // under unified addressing) are read and written by the kernels themselves: one ingest launch
+  // instead of four copies and an append, and the attention kernel stores the result where the
+  // caller wants it.  Anything else (pageable memory) goes through cudaMemcpyAsync.
+  auto mapped = [](const void* p) -> void* {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+  };
+  void* dq = mapped(host_q);
+  void* dk = dq ? mapped(host_new_k) : nullptr;
+  void* dv = dk ? mapped(host_new_v) : nullptr;
+  void* dl = dv ? mapped(host_seq_lens) : nullptr;
+  void* dout = dl ? mapped(host_out) : nullptr;
+  const bool aligned = (((uintptr_t)dq | (uintptr_t)dk | (uintptr_t)dv) & 15u) == 0 && ((uintptr_t)dl & 3u) == 0 &&
+                       ((uintptr_t)dout & 1u) == 0;
+  if (dout && aligned) {
+    {
+      LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+      ingest_kernel<<<dim3(batch, kIngestSplit), 256, 0, st>>>(
+          static_cast<const uint4*>(dq), static_cast<const uint4*>(dk), static_cast<const uint4*>(dv),
+          static_cast<const int*>(dl), reinterpret_cast<uint4*>(ctx->st_q),
+          static_cast<__nv_bfloat16*>(const_cast<void*>(kv->k)), static_cast<__nv_bfloat16*>(const_cast<void*>(kv->v)),
+          kv->stride_outer, kv->stride_head, const_cast<int32_t*>(kv->seq_lens), ctx->cfg.num_q_heads,
+          ctx->cfg.num_kv_heads);
+    }
+    PRHS_CUDA(ctx, cudaGetLastError());
+    prhs_status rc = prhs_decode_step(ctx, layer, step, sched, ctx->st_q, kv, batch, dout, nullptr, stream);
+    if (rc != PRHS_OK) return rc;
+    PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+    return PRHS_OK;
+  }
   PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_q, host_q, qb, cudaMemcpyHostToDevice, st));
   PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_k, host_new_k, kb, cudaMemcpyHostToDevice, st));
   PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_v, host_new_v, kb, cudaMemcpyHostToDevice, st));

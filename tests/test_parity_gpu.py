@@ -386,7 +386,10 @@ def test_c5_serving_mix_sampled(cuda_device):
 
 
 # ------------------------------------------------------------------- host-buffer entry point
-def test_decode_step_host_buffers(cuda_device):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_host_buffers(cuda_device, pinned):
+    # pinned buffers are read and written by the kernels directly, pageable ones are copied
+    pin = (lambda x: x.pin_memory()) if pinned else (lambda x: x)
     w = small(steps=3, refresh=2, context=1200)
     k, v = W.make_kv(w, cuda_device)
     q = W.make_queries(w, cuda_device)
@@ -405,9 +408,10 @@ def test_decode_step_host_buffers(cuda_device):
         new_k, new_v = k[bi, :, pos].cpu().contiguous(), v[bi, :, pos].cpu().contiguous()
         k2[bi, :, pos] = 0
         v2[bi, :, pos] = 0
-        host_out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16).pin_memory()
-        ctx_b.decode_step_host(0, n, sched, q[0, n].cpu().contiguous().pin_memory(), new_k.pin_memory(),
-                               new_v.pin_memory(), t_host, P.make_view(k2, v2, t_dev), w.batch, host_out)
+        host_out = pin(torch.zeros(w.batch, w.q_heads, 128, dtype=torch.bfloat16))
+        ctx_b.decode_step_host(0, n, sched, pin(q[0, n].cpu().contiguous()), pin(new_k), pin(new_v),
+                               pin(t_host.contiguous()), P.make_view(k2, v2, t_dev), w.batch, host_out)
+        assert torch.equal(t_dev.cpu(), t_host)
         assert torch.equal(host_out, out_a.cpu())
     assert torch.equal(k2, k) and torch.equal(v2, v)
     ctx_a.close(); ctx_b.close()
