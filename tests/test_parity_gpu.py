@@ -505,3 +505,51 @@ def test_group_sets_c3_slice_sampled(cuda_device):
     units = [(0, 0), (0, 3), (2, 21), (3, 31)]
     st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3, 4], group_sets=True)
     assert st["checked"] == 4 * 5 * len(units)
+
+
+# ------------------------------------------- selection kernel: the rarely taken configurations
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", ["large_k_bitonic", "one_bitmap", "k_above_candidates", "list_everything"])
+def test_selection_shared_memory_layouts(cuda_device, case):
+    """The selection kernel sizes its shared memory from the context's maxima and switches
+    layout with them: a budget so large that the list cannot hold a second sort buffer (the
+    in-place bitonic sort takes over), a context so long that only one position bitmap fits
+    (two sweeps), k above the middle range (everything is a winner), and a range short enough
+    to list every candidate without sampling."""
+    if case == "large_k_bitonic":
+        w, over = small(context=30000, top_k=5000, batch=1, q_heads=2, kv_heads=2, seed=61), {}
+    elif case == "one_bitmap":
+        w, over = small(context=20000, top_k=300, batch=1, q_heads=2, kv_heads=1, seed=62), dict(max_context=1_000_000)
+    elif case == "k_above_candidates":
+        w, over = small(context=900, top_k=2000, batch=2, seed=63), {}
+    else:
+        w, over = small(context=3000, top_k=64, batch=2, seed=64), {}
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = W.seq_lens_at(w, 0)
+    ctx = H.make_ctx(w, **over)
+    sched = H.make_sched(w, cuda_device)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    ctx.score_topk(0, 0, q, view, sched, w.batch)
+    assert ctx.check() == 0                         # in particular: no fallback to the generic path
+    s_star, n_star, s_hat, n_hat = ctx.get_shared_set(0, w.batch)
+    qh = H.np32(q)
+    gq = w.q_heads // w.kv_heads
+    for b, h in all_units(w):
+        t = int(t_host[b])
+        a = O.dense_scores(qh[b, h], H.np32(k[b, h // gq]), t)
+        want = O.topk_middle(a, t, w.sinks, w.window, w.top_k)
+        got = s_star[b, h, : int(n_star[b, h])].numpy().astype(np.int64)
+        H.check_topk_legal(O.rank_logits(a), got, want, f"{case} unit ({b},{h})")
+        hat = s_hat[b, h, : int(n_hat[b, h])].numpy().astype(np.int64)
+        assert np.array_equal(hat, O.dilate(got, w.top_k // 3, 1, t))
+    # and a whole step over that set
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    ctx.decode_step(0, 0, sched, q, view, w.batch, out)
+    idx, cnt = ctx.get_index_set(w.batch)
+    assert ctx.check() == 0
+    for b, h in all_units(w)[:2]:
+        C = idx[b, h, : int(cnt[b, h])].numpy().astype(np.int64)
+        y, _ = O.attn_over_set(qh[b, h], H.np32(k[b, h // gq]), H.np32(v[b, h // gq]), C)
+        assert np.max(np.abs(H.np32(out)[b, h] - O.bf16_round(y))) <= H.Y_TOL
+    ctx.close()
