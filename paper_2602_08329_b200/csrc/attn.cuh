@@ -726,6 +726,7 @@ struct ScoreParams {
   int splits, num_q_heads, group_size;
   const int* need;        // [B][Hq] or nullptr: score only KV heads with a query head that retrieves
   int group_max;          // 1: write max over the group's heads to the row of its first head only
+  int chunk_rows;         // > 0: split j covers rows [j * chunk_rows, (j + 1) * chunk_rows) of every sequence
   uint32_t* flags;
 };
 

@@ -208,6 +208,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.group_size = c->gq;
   sp.need = need;
   sp.group_max = (sched && (sched->flags & PRHS_GROUP_SETS) && c->gq > 1) ? 1 : 0;
+  sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + kSTStageRows - 1) & ~(kSTStageRows - 1);
   sp.flags = c->flags;
   bool tma_done = false;
   if (c->encode_tiled) {

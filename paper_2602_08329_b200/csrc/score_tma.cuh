@@ -7,9 +7,9 @@
 // completion is signalled on an mbarrier, and four consumer warps (16 keys each) run the
 // m16n8k16 MMAs for all heads of the KV group.  A six-stage ring keeps up to 80 KB in flight
 // per CTA with no address arithmetic in the consumer warps.  With a paged cache the tensor is
-// the page pool, a stage is four pages of 16 keys, and the producer issues one pair of
-// [16 rows][64 columns] boxes per page after looking its id up in the page table (ids of the
-// next stage are fetched while the current one is issued); pages past the end of the
+// the page pool, a stage is four pages of 16 keys, and eight lanes of the producer warp each
+// look a page id up and issue one [16 rows][64 columns] box (ids of the next stage are fetched
+// while the current one is issued); pages past the end of the
 // sequence are not fetched and an id outside the pool is skipped and flagged.
 //
 // Every wait on an mbarrier is bounded: a wait that exceeds its budget records
@@ -109,8 +109,18 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;
   const int t = __ldg(p.kv.seq_lens + b);
-  int per = (t + p.splits - 1) / p.splits;
-  per = (per + kSTStageRows - 1) & ~(kSTStageRows - 1);
+  // Equal-sized chunks of rows (a multiple of the stage) for every sequence: a short sequence of
+  // a ragged batch fills fewer CTAs instead of many short ones; the others leave at once.
+  int per = p.chunk_rows;
+  if (per <= 0) {
+    per = (t + p.splits - 1) / p.splits;
+    per = (per + kSTStageRows - 1) & ~(kSTStageRows - 1);
+  }
+  if (split * per >= t && split > 0) {
+    if ((int)threadIdx.x < gq)
+      p.part_ml[((long long)b * p.num_q_heads + head0 + threadIdx.x) * p.splits + split] = make_float2(-INFINITY, 0.f);
+    return;
+  }
   const int start = min(split * per, t);
   const int end = min(start + per, t);
   const int nstages = (end - start + kSTStageRows - 1) / kSTStageRows;
@@ -131,55 +141,57 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
   __syncthreads();
 
   if (warp == kSTConsumers) {
-    // ---------------- producer: one elected lane feeds the ring
-    if (lane == 0) {
-      const uint64_t pol_k = l2_policy_evict_first();
-      const int* ptab = kPaged ? p.kv.page_table + (long long)b * p.kv.page_table_stride + (start >> kPageShift) : nullptr;
-      int pg_next[4] = {0, 0, 0, 0};
-      if (kPaged) {
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-          if (start + 16 * x < end) pg_next[x] = __ldg(ptab + x);
-      }
-      for (int j = 0; j < nstages; ++j) {
-        const int slot = j % kSTStages;
-        int pg[4] = {pg_next[0], pg_next[1], pg_next[2], pg_next[3]};
-        if (kPaged && j + 1 < nstages) {      // page ids of the next stage, in flight during the wait below
-#pragma unroll
-          for (int x = 0; x < 4; ++x)
-            if (start + (j + 1) * kSTStageRows + 16 * x < end) pg_next[x] = __ldg(ptab + 4 * (j + 1) + x);
-        }
-        if (j >= kSTStages && !mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort)) {
-          atomicOr(p.flags, kFlagTimeout);
-          sh_abort = 1;
-          break;
-        }
-        if (*(volatile int*)&sh_abort) break;
-        const uint32_t full = bar0 + 8 * slot;
-        const uint32_t dst = smem0 + slot * kSTStageBytes;
-        if (!kPaged) {
+    // ---------------- producer: one elected lane feeds the ring (contiguous cache); with a paged
+    // cache lanes 0-7 each look up one of the stage's four pages and fetch one half of it
+    const uint64_t pol_k = l2_policy_evict_first();
+    if (!kPaged) {
+      if (lane == 0) {
+        for (int j = 0; j < nstages; ++j) {
+          const int slot = j % kSTStages;
+          if (j >= kSTStages && !mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort)) {
+            atomicOr(p.flags, kFlagTimeout);
+            sh_abort = 1;
+            break;
+          }
+          if (*(volatile int*)&sh_abort) break;
+          const uint32_t full = bar0 + 8 * slot;
+          const uint32_t dst = smem0 + slot * kSTStageBytes;
           mbar_expect_tx(full, kSTStageBytes);
           tma_load_2d(dst, &tm_k, 0, row_base + j * kSTStageRows, full, pol_k);
           tma_load_2d(dst + kSTHalfBytes, &tm_k, 64, row_base + j * kSTStageRows, full, pol_k);
-        } else {
-          uint32_t okmask = 0u;
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            if (start + j * kSTStageRows + 16 * x < end) {
-              if ((unsigned)pg[x] < (unsigned)p.kv.num_pages) okmask |= 1u << x;
-              else atomicOr(p.flags, kFlagBadPage);
-            }
-          }
-          // the barrier needs its arrive even when no page of the stage is fetched
-          mbar_expect_tx(full, (uint32_t)__popc(okmask) * 4096u);
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            if ((okmask >> x) & 1u) {
-              const int row = pg[x] * outer_rows + row_base;
-              tma_load_2d(dst + x * 2048, &tm_k, 0, row, full, pol_k);
-              tma_load_2d(dst + kSTHalfBytes + x * 2048, &tm_k, 64, row, full, pol_k);
-            }
-          }
+        }
+      }
+    } else {
+      const int x = (lane >> 1) & 3, half = lane & 1;   // lanes 0-7: page x of the stage, 64-column half
+      const int* ptab = p.kv.page_table + (long long)b * p.kv.page_table_stride + (start >> kPageShift) + x;
+      bool have_next = lane < 8 && start + 16 * x < end;
+      int pg_next = have_next ? __ldg(ptab) : 0;
+      for (int j = 0; j < nstages; ++j) {
+        const int slot = j % kSTStages;
+        const int pg = pg_next;
+        const bool have = have_next;                // false: past the end, or lane >= 8
+        // page id of the next stage, in flight during the wait below
+        have_next = lane < 8 && j + 1 < nstages && start + (j + 1) * kSTStageRows + 16 * x < end;
+        pg_next = have_next ? __ldg(ptab + 4 * (j + 1)) : 0;
+        bool ok = true;
+        if (lane == 0 && j >= kSTStages)
+          ok = mbar_wait(bar0 + 8 * (kSTStages + slot), ((j / kSTStages) - 1) & 1, &sh_abort);
+        if (lane == 0 && !ok) {
+          atomicOr(p.flags, kFlagTimeout);
+          sh_abort = 1;
+        }
+        __syncwarp();
+        if (*(volatile int*)&sh_abort) break;       // warp-uniform: read after the barrier above
+        const bool fetch = have && (unsigned)pg < (unsigned)p.kv.num_pages;
+        if (have && !fetch) atomicOr(p.flags, kFlagBadPage);
+        const uint32_t okmask = __ballot_sync(0xffffffffu, fetch);
+        const uint32_t full = bar0 + 8 * slot;
+        // the barrier needs its arrive even when no page of the stage is fetched
+        if (lane == 0) mbar_expect_tx(full, (uint32_t)__popc(okmask) * 2048u);
+        __syncwarp();
+        if (fetch) {
+          const uint32_t dst = smem0 + slot * kSTStageBytes + half * kSTHalfBytes + x * 2048;
+          tma_load_2d(dst, &tm_k, 64 * half, pg * outer_rows + row_base, full, pol_k);
         }
       }
     }
