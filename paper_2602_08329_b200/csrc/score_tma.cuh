@@ -4,13 +4,13 @@
 // tiles are brought into shared memory by the tensor memory accelerator: one elected thread
 // issues two `cp.async.bulk.tensor.2d` copies per 64-key stage (a [64 rows][64 columns] box for
 // each half of the 128 dimensions, 128-byte swizzle so that ldmatrix reads are conflict-free),
-// completion is signalled on an mbarrier, and four consumer warps (16 keys each) run the
+// completion is signalled on an mbarrier, and eight consumer warps (8 keys each) run the
 // m16n8k16 MMAs for all heads of the KV group.  A six-stage ring keeps up to 80 KB in flight
 // per CTA with no address arithmetic in the consumer warps.  With a paged cache the tensor is
 // the page pool, a stage is four pages of 16 keys, and eight lanes of the producer warp each
 // look a page id up and issue one [16 rows][64 columns] box (ids of the next stage are fetched
-// while the current one is issued); pages past the end of the
-// sequence are not fetched and an id outside the pool is skipped and flagged.
+// while the current one is issued); pages past the end of the sequence are not fetched and an
+// id outside the pool is skipped and flagged.
 //
 // Every wait on an mbarrier is bounded: a wait that exceeds its budget records
 // kFlagTimeout and the CTA drains and returns, so a wrong descriptor cannot hang the GPU.
