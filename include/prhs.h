@@ -309,6 +309,13 @@ const char* prhs_kernel_kind_name(int32_t kind);
 /* Number of kernels this context has launched since creation (host-side counter). */
 int64_t prhs_launch_count(const prhs_ctx* ctx);
 
+/* Self-test of the failure path of the TMA kernels (no counterpart in the paper): launches one
+ * thread that waits, with the given budget in SM cycles (1 .. 2e8, about 0.1 s), on a barrier
+ * that nothing completes.  The wait must give up: *host_gave_up = 1, PRHS_FLAG_TIMEOUT is set in
+ * the device flag word (the next prhs_check reports and clears it) and the context stays
+ * usable.  Synchronises the stream. */
+prhs_status prhs_selftest_wait(prhs_ctx* ctx, int64_t budget_cycles, int32_t* host_gave_up, void* stream);
+
 /* Message of the last error on this context (or of the last failed prhs_create when ctx is
  * NULL).  The pointer stays valid until the next call on the context. */
 const char* prhs_last_error(const prhs_ctx* ctx);

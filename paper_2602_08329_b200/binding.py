@@ -28,7 +28,7 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_sparse_decode_attn", "prhs_dense_decode_attn", "prhs_decode_step",
            "prhs_decode_step_host", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
-           "prhs_launch_count", "prhs_last_error", "prhs_version", "prhs_profile_begin",
+           "prhs_launch_count", "prhs_selftest_wait", "prhs_last_error", "prhs_version", "prhs_profile_begin",
            "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate"]
 NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
@@ -97,6 +97,7 @@ def load() -> C.CDLL:
         "prhs_profile_end": (st, [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]),
         "prhs_kernel_kind_name": (C.c_char_p, [i32]),
         "prhs_launch_count": (C.c_int64, [vp]),
+        "prhs_selftest_wait": (st, [vp, C.c_int64, C.POINTER(C.c_int32), vp]),
         "prhs_last_error": (C.c_char_p, [vp]),
         "prhs_version": (C.c_char_p, []),
     }
@@ -262,6 +263,11 @@ class Context:
         self._ck(self.lib.prhs_profile_end(self.h, _stream(stream), ms, n))
         return {self.lib.prhs_kernel_kind_name(i).decode(): (float(ms[i]), int(n[i]))
                 for i in range(KERNEL_KINDS)}
+
+    def selftest_wait(self, budget_cycles=1_000_000, stream=None) -> int:
+        gave_up = C.c_int32(-1)
+        self._ck(self.lib.prhs_selftest_wait(self.h, budget_cycles, C.byref(gave_up), _stream(stream)))
+        return gave_up.value
 
     def check(self, stream=None) -> int:
         flags = C.c_uint32(0)

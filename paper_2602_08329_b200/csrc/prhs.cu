@@ -441,6 +441,24 @@ const char* prhs_last_error(const prhs_ctx* ctx) { return ctx ? ctx->err.c_str()
 
 int64_t prhs_launch_count(const prhs_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+prhs_status prhs_selftest_wait(prhs_ctx* ctx, int64_t budget_cycles, int32_t* host_gave_up, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (budget_cycles < 1 || budget_cycles > 200000000ll)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "selftest: budget must be in [1, 2e8] cycles");
+  cudaStream_t st = as_stream(stream);
+  int* d = reinterpret_cast<int*>(ctx->count);      // any device int owned by the context
+  {
+    LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+    wait_selftest_kernel<<<1, 32, 0, st>>>((long long)budget_cycles, ctx->flags, d);
+  }
+  PRHS_CUDA(ctx, cudaGetLastError());
+  int h = -1;
+  PRHS_CUDA(ctx, cudaMemcpyAsync(&h, d, sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  if (host_gave_up) *host_gave_up = h;
+  return PRHS_OK;
+}
+
 int32_t prhs_index_capacity(const prhs_ctx* ctx) { return ctx ? ctx->idx_cap : 0; }
 
 int32_t prhs_scores_ld(const prhs_ctx* ctx) { return ctx ? ctx->ld : 0; }

@@ -53,11 +53,12 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: false if the phase did not complete within the cycle budget, or if another
 // thread of the CTA has already given up (*abort != 0).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort,
+                                          long long budget = kWaitBudgetCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity))
-    if (*abort || clock64() - t0 > kWaitBudgetCycles) return false;
+    if (*abort || clock64() - t0 > budget) return false;
   return true;
 }
 // The key stream is read once and is far larger than L2: its lines are marked evict-first, and
@@ -299,6 +300,23 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
       while (!mbar_try_wait(bar0 + 8 * s, 0) && !mbar_try_wait(bar0 + 8 * s, 1))
         if (clock64() - t0 > kWaitBudgetCycles / 8) break;
     }
+  }
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier phase that nothing completes,
+// with a short budget; the wait must come back false, and the kernel records kFlagTimeout the
+// way the scoring kernel does.  Harmless by construction: the loop ends with the budget.
+__global__ void wait_selftest_kernel(long long budget, uint32_t* flags, int* gave_up) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+    mbar_init(b, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(b, 0, &abort_flag, budget);
+    if (!ok) atomicOr(flags, kFlagTimeout);
+    *gave_up = ok ? 0 : 1;
   }
 }
 

@@ -553,3 +553,34 @@ def test_selection_shared_memory_layouts(cuda_device, case):
         y, _ = O.attn_over_set(qh[b, h], H.np32(k[b, h // gq]), H.np32(v[b, h // gq]), C)
         assert np.max(np.abs(H.np32(out)[b, h] - O.bf16_round(y))) <= H.Y_TOL
     ctx.close()
+
+
+# ------------------------------------------------------------------ failure path, without a fault
+@pytest.mark.gpu
+def test_bounded_wait_gives_up_and_context_survives(cuda_device):
+    """A wait on a barrier that nothing completes runs out of its budget, the kernel reports
+    it through the flag word, and the same context then decodes as if nothing had happened."""
+    w = small(steps=2, context=1800)
+    ctx = H.make_ctx(w)
+    assert ctx.selftest_wait(500_000) == 1
+    with pytest.raises(P.PrhsError) as e:
+        ctx.check()
+    assert e.value.status == 7                                # PRHS_ERR_DEVICE_FLAG
+    assert ctx.check() == 0                                   # reported once, then cleared
+    with pytest.raises(P.PrhsError):
+        ctx.selftest_wait(10**12)                             # budgets are capped
+    # the same context decodes, bit for bit like a fresh one
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    sched = H.make_sched(w, cuda_device)
+    view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device), max_seq_len=w.capacity)
+    outs = []
+    for c in (ctx, H.make_ctx(w)):
+        out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+        c.decode_step(0, 0, sched, q, view, w.batch, out)
+        assert c.check() == 0
+        outs.append(out.cpu())
+        c.close()
+    assert torch.equal(outs[0], outs[1])
+    st = H.run_schedule_parity(w, cuda_device, all_units(w))
+    assert st["checked"] == 2 * w.batch * w.q_heads
