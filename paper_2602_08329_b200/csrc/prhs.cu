@@ -193,7 +193,8 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
   return best;
 }
 
-// `sched` != nullptr: a retrieval pass (logits are written and the selection histogram filled).
+// `sched` != nullptr: a retrieval pass (the fp32 logits are written for the selection kernel);
+// nullptr: only the per-split log-sum-exp partials (the delta diagnostic).
 prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
                          const prhs_schedule* sched, const int* need, cudaStream_t st, int* nchunks_out) {
   const int write_scores = sched != nullptr;
@@ -520,7 +521,9 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     delete c;
     return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context / max_k too large for the selection kernel");
   }
-  e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem);
+  // the opt-in limit is a property of the kernel, not of this context: always the maximum, so that
+  // contexts of different sizes can live side by side
+  e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess)

@@ -584,3 +584,24 @@ def test_bounded_wait_gives_up_and_context_survives(cuda_device):
     assert torch.equal(outs[0], outs[1])
     st = H.run_schedule_parity(w, cuda_device, all_units(w))
     assert st["checked"] == 2 * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
+def test_contexts_of_different_sizes_side_by_side(cuda_device):
+    """A large context, then a small one, then the large one is used: kernel attributes set at
+    creation must not depend on which context was created last."""
+    big = small(context=30000, top_k=5000, batch=1, q_heads=2, kv_heads=2, seed=71)
+    little = small(context=1500, seed=72)
+    ctx_big, ctx_little = H.make_ctx(big), H.make_ctx(little)
+    for w, ctx in ((big, ctx_big), (little, ctx_little), (big, ctx_big)):
+        k, v = W.make_kv(w, cuda_device)
+        q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+        view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device), max_seq_len=w.capacity)
+        out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+        ctx.decode_step(0, 0, H.make_sched(w, cuda_device), q, view, w.batch, out)
+        assert ctx.check() == 0
+        idx, cnt = ctx.get_index_set(w.batch)
+        C = idx[0, 0, : int(cnt[0, 0])].numpy().astype(np.int64)
+        y, _ = O.attn_over_set(H.np32(q)[0, 0], H.np32(k[0, 0]), H.np32(v[0, 0]), C)
+        assert np.max(np.abs(H.np32(out)[0, 0] - O.bf16_round(y))) <= H.Y_TOL
+    ctx_big.close(); ctx_little.close()
