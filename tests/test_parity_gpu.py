@@ -605,3 +605,39 @@ def test_contexts_of_different_sizes_side_by_side(cuda_device):
         y, _ = O.attn_over_set(H.np32(q)[0, 0], H.np32(k[0, 0]), H.np32(v[0, 0]), C)
         assert np.max(np.abs(H.np32(out)[0, 0] - O.bf16_round(y))) <= H.Y_TOL
     ctx_big.close(); ctx_little.close()
+
+
+@pytest.mark.gpu
+def test_non_finite_keys_stay_contained(cuda_device):
+    """NaN / Inf inputs are outside the method's definition; the library must still return, keep
+    every index in range, and leave the heads of other KV heads exactly as they are."""
+    w = small(context=6000, batch=2, q_heads=4, kv_heads=2, steps=2, seed=81)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)
+    k_bad = k.clone()
+    k_bad[0, 0, 100] = float("nan")
+    k_bad[0, 0, 2000:2010] = float("inf")
+    k_bad[0, 0, 3000] = float("-inf")
+    outs = []
+    for keys in (k, k_bad):
+        ctx = H.make_ctx(w)
+        sched = H.make_sched(w, cuda_device)
+        res = []
+        for n in range(w.steps):
+            view = P.make_view(keys, v, W.seq_lens_at(w, n).to(cuda_device), max_seq_len=w.capacity)
+            out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+            ctx.decode_step(0, n, sched, q[0, n].contiguous(), view, w.batch, out)
+            idx, cnt = ctx.get_index_set(w.batch)
+            assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+            t = W.seq_lens_at(w, n)
+            for b in range(w.batch):
+                for h in range(w.q_heads):
+                    c = idx[b, h, : int(cnt[b, h])]
+                    assert int(cnt[b, h]) <= ctx.index_capacity and bool((c >= 0).all()) and bool((c < int(t[b])).all())
+            res.append(out.cpu())
+        outs.append(res)
+        ctx.close()
+    gq = w.q_heads // w.kv_heads
+    for a, b_ in zip(*outs):
+        assert torch.equal(a[1], b_[1])                 # the other sequence
+        assert torch.equal(a[0, gq:], b_[0, gq:])       # the other KV head of the same sequence
