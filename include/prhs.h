@@ -242,6 +242,17 @@ prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step,
                                   const int32_t* host_seq_lens, const prhs_kv_view* kv,
                                   int32_t batch, void* host_out, void* stream);
 
+/* The same without the final synchronisation: everything is enqueued on `stream` and the call
+ * returns.  host_q, host_new_k, host_new_v and host_seq_lens must stay unchanged, and host_out
+ * is not valid, until the stream has reached the end of this call's work (the caller's own
+ * cudaStreamSynchronize or event).  host_seq_lens is also read on the host, for validation,
+ * during the call.  Lets a caller enqueue the next layer or step while this one runs. */
+prhs_status prhs_decode_step_host_async(prhs_ctx* ctx, int32_t layer, int32_t step,
+                                  const prhs_schedule* sched, const void* host_q,
+                                  const void* host_new_k, const void* host_new_v,
+                                  const int32_t* host_seq_lens, const prhs_kv_view* kv,
+                                  int32_t batch, void* host_out, void* stream);
+
 /* Dropped mass (Sec. 2.3): delta = 1 - sum_{i in C} A_i with A the full softmax over
  * i < t_b.  Runs a dense log-sum-exp pass and a sparse pass.  out_delta device fp32
  * [batch][Hq]. */

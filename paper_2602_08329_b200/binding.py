@@ -26,7 +26,7 @@ PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TI
 # every symbol include/prhs.h declares
 EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_set",
            "prhs_sparse_decode_attn", "prhs_dense_decode_attn", "prhs_decode_step",
-           "prhs_decode_step_host", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
+           "prhs_decode_step_host", "prhs_decode_step_host_async", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
            "prhs_launch_count", "prhs_selftest_wait", "prhs_last_error", "prhs_version", "prhs_profile_begin",
            "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate"]
@@ -85,6 +85,8 @@ def load() -> C.CDLL:
         "prhs_sparse_decode_attn_noalloc": (st, [vp, C.POINTER(KvView), vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "prhs_decode_step": (st, [vp, i32, i32, C.POINTER(Schedule), vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_decode_step_host": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32, vp, vp]),
+        "prhs_decode_step_host_async": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32,
+                                              vp, vp]),
         "prhs_delta": (st, [vp, vp, C.POINTER(KvView), vp, vp, i32, i32, vp, vp]),
         "prhs_index_capacity": (i32, [vp]),
         "prhs_get_index_set": (st, [vp, i32, vp, vp, vp]),
@@ -214,11 +216,10 @@ class Context:
                                            batch, _ptr(out), _ptr(out_delta), _stream(stream)))
 
     def decode_step_host(self, layer, step, sched, host_q, host_new_k, host_new_v, host_seq_lens,
-                         view, batch, host_out, stream=None):
-        self._ck(self.lib.prhs_decode_step_host(self.h, layer, step, C.byref(sched), _ptr(host_q),
-                                                _ptr(host_new_k), _ptr(host_new_v),
-                                                _ptr(host_seq_lens), C.byref(view), batch,
-                                                _ptr(host_out), _stream(stream)))
+                         view, batch, host_out, stream=None, sync=True):
+        fn = self.lib.prhs_decode_step_host if sync else self.lib.prhs_decode_step_host_async
+        self._ck(fn(self.h, layer, step, C.byref(sched), _ptr(host_q), _ptr(host_new_k), _ptr(host_new_v),
+                    _ptr(host_seq_lens), C.byref(view), batch, _ptr(host_out), _stream(stream)))
 
     def delta(self, q, view, idx, count, batch, out_delta, stream=None):
         self._ck(self.lib.prhs_delta(self.h, _ptr(q), C.byref(view), _ptr(idx), _ptr(count),

@@ -842,10 +842,11 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
                      want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr, st);
 }
 
-prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+namespace {
+prhs_status decode_step_host_impl(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
                                   const void* host_q, const void* host_new_k, const void* host_new_v,
                                   const int32_t* host_seq_lens, const prhs_kv_view* kv, int32_t batch,
-                                  void* host_out, void* stream) {
+                                  void* host_out, void* stream, bool sync) {
   if (!ctx) return PRHS_ERR_INVALID_ARG;
   if (!host_q || !host_new_k || !host_new_v || !host_seq_lens || !host_out || !kv)
     return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
@@ -889,7 +890,7 @@ prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, co
     PRHS_CUDA(ctx, cudaGetLastError());
     prhs_status rc = prhs_decode_step(ctx, layer, step, sched, ctx->st_q, kv, batch, dout, nullptr, stream);
     if (rc != PRHS_OK) return rc;
-    PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+    if (sync) PRHS_CUDA(ctx, cudaStreamSynchronize(st));
     return PRHS_OK;
   }
   PRHS_CUDA(ctx, cudaMemcpyAsync(ctx->st_q, host_q, qb, cudaMemcpyHostToDevice, st));
@@ -908,8 +909,25 @@ prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, co
   prhs_status rc = prhs_decode_step(ctx, layer, step, sched, ctx->st_q, kv, batch, ctx->st_out, nullptr, stream);
   if (rc != PRHS_OK) return rc;
   PRHS_CUDA(ctx, cudaMemcpyAsync(host_out, ctx->st_out, qb, cudaMemcpyDeviceToHost, st));
-  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  if (sync) PRHS_CUDA(ctx, cudaStreamSynchronize(st));
   return PRHS_OK;
+}
+}  // namespace
+
+prhs_status prhs_decode_step_host(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                                  const void* host_q, const void* host_new_k, const void* host_new_v,
+                                  const int32_t* host_seq_lens, const prhs_kv_view* kv, int32_t batch,
+                                  void* host_out, void* stream) {
+  return decode_step_host_impl(ctx, layer, step, sched, host_q, host_new_k, host_new_v, host_seq_lens, kv, batch,
+                               host_out, stream, true);
+}
+
+prhs_status prhs_decode_step_host_async(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
+                                        const void* host_q, const void* host_new_k, const void* host_new_v,
+                                        const int32_t* host_seq_lens, const prhs_kv_view* kv, int32_t batch,
+                                        void* host_out, void* stream) {
+  return decode_step_host_impl(ctx, layer, step, sched, host_q, host_new_k, host_new_v, host_seq_lens, kv, batch,
+                               host_out, stream, false);
 }
 
 prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, const int32_t* idx,

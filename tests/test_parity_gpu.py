@@ -395,6 +395,7 @@ def test_decode_step_host_buffers(cuda_device, pinned):
     q = W.make_queries(w, cuda_device)
     k2, v2 = k.clone(), v.clone()
     ctx_a, ctx_b = H.make_ctx(w), H.make_ctx(w)
+    ctx_cs = [H.make_ctx(w)]
     sched = H.make_sched(w, cuda_device)
     out_a = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
     t_dev = torch.zeros(w.batch, dtype=torch.int32, device=cuda_device)
@@ -412,9 +413,18 @@ def test_decode_step_host_buffers(cuda_device, pinned):
         ctx_b.decode_step_host(0, n, sched, pin(q[0, n].cpu().contiguous()), pin(new_k), pin(new_v),
                                pin(t_host.contiguous()), P.make_view(k2, v2, t_dev), w.batch, host_out)
         assert torch.equal(t_dev.cpu(), t_host)
+        if pinned:      # the variant that does not synchronise: valid once the stream has caught up
+            k3, v3, t3 = k2.clone(), v2.clone(), torch.zeros_like(t_dev)
+            k3[bi, :, pos] = 0
+            out_async = pin(torch.zeros(w.batch, w.q_heads, 128, dtype=torch.bfloat16))
+            held = (pin(q[0, n].cpu().contiguous()), pin(new_k), pin(new_v), pin(t_host.contiguous()))
+            ctx_cs[0].decode_step_host(0, n, sched, *held, P.make_view(k3, v3, t3), w.batch, out_async,
+                                       sync=False)
+            torch.cuda.synchronize()        # the host buffers are held until here
+            assert torch.equal(out_async, host_out) and torch.equal(k3, k)
         assert torch.equal(host_out, out_a.cpu())
     assert torch.equal(k2, k) and torch.equal(v2, v)
-    ctx_a.close(); ctx_b.close()
+    ctx_a.close(); ctx_b.close(); ctx_cs[0].close()
 
 
 # ------------------------------------------------------------------------- host validation
