@@ -118,11 +118,15 @@ def table3(dev):
                   f"{am[8]:.1f} | {am[16]:.1f} | {r['dense_us'] / am[16]:.2f}x | {pf} / {p8} / {p16} |")
 
 
-def configs(dev, group_sets=False):
+def configs(dev, group_sets=False, only=None, batch=0):
     print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
           "mean set size | dense / amortised | sharing step GB/s logical / unique | retrieval step kernels us |")
     print("|---|---|---|---|---|---|---|---|---|")
     for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
+        if only and w.name != only:
+            continue
+        if batch:
+            w = w.scaled(batch=batch)
         r = time_workload(w.scaled(layer_group=1), dev, copies=4 if w.context < 50000 else 2, group_sets=group_sets)
         period = w.refresh * w.layer_group      # layer-steps per retrieval
         am = (r["refresh_us"] + (period - 1) * r["shared_us"]) / period
@@ -136,6 +140,8 @@ def configs(dev, group_sets=False):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C5 shapes instead")
+    ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
+    ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
     ap.add_argument("--group-sets", action="store_true",
                     help="with --configs: the labelled variant with one index set per KV head (not in the paper)")
     args = ap.parse_args()
@@ -144,7 +150,7 @@ def main():
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     if args.configs:
-        configs(dev, args.group_sets)
+        configs(dev, args.group_sets, args.only, args.batch)
     else:
         table3(dev)
 
