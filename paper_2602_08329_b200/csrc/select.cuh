@@ -218,18 +218,34 @@ __device__ __forceinline__ void find_bin_from_top(const uint32_t* hist, int nb, 
   }
 }
 
-// The warp's sample of logits (NX per lane: sample x * nt + slot of S, one logit out of every
-// sstride) and the largest value, at the resolution of the top 13 key bits, that at least rw of
-// them reach.  Bisection on the key bits; the count is a compare per sample and one warp
-// reduction per bit.
+// The warp's sample of logits -- NSEC aligned 32-byte sectors (8 logits each) per lane: sample
+// x * nt + slot of S, one sector out of every sec_stride -- and the largest value, at the
+// resolution of the top 13 key bits, that at least rw of them reach.  Whole sectors, because the
+// logits of a long context do not all stay in L2 and DRAM serves a scattered 4-byte read at
+// the price of a sector.  Bisection on the key bits; the count is a compare per sample and one
+// warp reduction per bit.
 constexpr int kThrBits = 13;
-template <int NX>
-__device__ __forceinline__ uint32_t sample_quantile(const float* g, int S, int sstride, int nt, int slot, int rw) {
-  uint32_t u[NX];
+template <int NSEC>
+__device__ __forceinline__ uint32_t sample_quantile(const float* gal, int S, int sec_stride, int nt, int slot, int rw) {
+  uint32_t u[8 * NSEC];
 #pragma unroll
-  for (int x = 0; x < NX; ++x) {
+  for (int x = 0; x < NSEC; ++x) {
     const int sidx = x * nt + slot;
-    u[x] = sidx < S ? float_to_key(__ldcg(g + (long long)sidx * sstride + ((sidx * 5) & 15))) : 0u;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    const bool ok = sidx < S;
+    if (ok) {
+      const float4* src = reinterpret_cast<const float4*>(gal + ((long long)sidx * sec_stride + ((sidx * 5) & 15)) * 8);
+      a = __ldcg(src);
+      b = __ldcg(src + 1);
+    }
+    u[8 * x + 0] = ok ? float_to_key(a.x) : 0u;
+    u[8 * x + 1] = ok ? float_to_key(a.y) : 0u;
+    u[8 * x + 2] = ok ? float_to_key(a.z) : 0u;
+    u[8 * x + 3] = ok ? float_to_key(a.w) : 0u;
+    u[8 * x + 4] = ok ? float_to_key(b.x) : 0u;
+    u[8 * x + 5] = ok ? float_to_key(b.y) : 0u;
+    u[8 * x + 6] = ok ? float_to_key(b.z) : 0u;
+    u[8 * x + 7] = ok ? float_to_key(b.w) : 0u;
   }
   uint32_t prefix = 0u;
 #pragma unroll 1
@@ -237,7 +253,28 @@ __device__ __forceinline__ uint32_t sample_quantile(const float* g, int S, int s
     const uint32_t trial = prefix | (1u << bit);
     int cnt = 0;
 #pragma unroll
-    for (int x = 0; x < NX; ++x) cnt += u[x] >= trial ? 1 : 0;
+    for (int x = 0; x < 8 * NSEC; ++x) cnt += u[x] >= trial ? 1 : 0;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (cnt >= rw) prefix = trial;
+  }
+  return prefix;
+}
+
+// The same for a short range (at most one sampled sector per two lanes): the two lanes of a pair
+// take one half of a sector each, so that every lane of the warp holds four logits.
+__device__ __forceinline__ uint32_t sample_quantile_half(const float* gal, int S, int sec_stride, int nw, int rw) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int sidx = (lane >> 1) * nw + warp;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool ok = sidx < S;
+  if (ok) a = __ldcg(reinterpret_cast<const float4*>(gal + ((long long)sidx * sec_stride + ((sidx * 5) & 15)) * 8) + (lane & 1));
+  const uint32_t u0 = ok ? float_to_key(a.x) : 0u, u1 = ok ? float_to_key(a.y) : 0u;
+  const uint32_t u2 = ok ? float_to_key(a.z) : 0u, u3 = ok ? float_to_key(a.w) : 0u;
+  uint32_t prefix = 0u;
+#pragma unroll 1
+  for (int bit = 31; bit > 31 - kThrBits; --bit) {
+    const uint32_t trial = prefix | (1u << bit);
+    int cnt = (u0 >= trial ? 1 : 0) + (u1 >= trial ? 1 : 0) + (u2 >= trial ? 1 : 0) + (u3 >= trial ? 1 : 0);
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     if (cnt >= rw) prefix = trial;
   }
@@ -440,22 +477,26 @@ __global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams 
     // the histograms of the four 8-bit passes of step 3 (the barrier after step 2 covers this)
     for (int i = tid; i < kHistWords; i += nt) hist[i] = 0u;
     // 1. conservative threshold from a sample (or -inf: list everything).  Every warp takes a
-    //    stratified 1-in-16 sample spread over the whole range (at most 16 logits per thread)
+    //    stratified 1-in-16 sample of 32-byte sectors spread over the whole range
     //    and finds, by bisection on the top 13 key bits, the value that
     //    1.75 k/16 + 16 sampled logits of the CTA would reach if all warps saw the same
     //    distribution; the lower median of the warps' values is the threshold.
     float thr = -INFINITY;
     if (n > p.cand_cap) {
       const int nw = nt >> 5;
-      const int sstride = max(kSampleStride, (n + 16 * nt - 1) / (16 * nt));
-      const int S = n / sstride;
-      const int nx = (S + nt - 1) / nt;            // <= 16
+      // whole 32-byte sectors, one out of every sec_stride (>= 16: a 1-in-16 sample), at most two
+      // per thread
+      const int a8 = (8 - (int)(((long long)unit * p.ld + lo) & 7)) & 7;
+      const int nsec = (n - a8) >> 3;
+      const int sec_stride = max(kSampleStride, (nsec + 2 * nt - 1) / (2 * nt));
+      const int S = nsec / sec_stride;               // sampled sectors
       const int slot = lane * nw + warp;
-      const int want = (int)((7ll * kk * S) / (4ll * n)) + 16;
+      const int want = (int)((7ll * kk * 8 * S) / (4ll * n)) + 16;
       const int rw = (want + nw - 1) / nw;
       uint32_t prefix;
-      if (nx <= 4) prefix = sample_quantile<4>(g, S, sstride, nt, slot, rw);
-      else prefix = sample_quantile<16>(g, S, sstride, nt, slot, rw);
+      if (2 * S <= nt) prefix = sample_quantile_half(g + a8, S, sec_stride, nw, rw);
+      else if (S <= nt) prefix = sample_quantile<1>(g + a8, S, sec_stride, nt, slot, rw);
+      else prefix = sample_quantile<2>(g + a8, S, sec_stride, nt, slot, rw);
       if (lane == 0) misc[80 + warp] = prefix;
       __syncthreads();
       const uint32_t mine = lane < nw ? misc[80 + lane] : 0xffffffffu;
