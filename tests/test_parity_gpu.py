@@ -651,3 +651,37 @@ def test_non_finite_keys_stay_contained(cuda_device):
     for a, b_ in zip(*outs):
         assert torch.equal(a[1], b_[1])                 # the other sequence
         assert torch.equal(a[0, gq:], b_[0, gq:])       # the other KV head of the same sequence
+
+
+# ------------------------------------------------------------ seeded random schedules end to end
+def _random_workload(seed):
+    g = np.random.default_rng(seed)
+    hkv = int(g.choice([1, 2, 4]))
+    gq = int(g.choice([1, 2, 4, 8]))
+    layer_group = int(g.choice([1, 2]))
+    refresh = int(g.choice([1, 2, 3, 4]))
+    context = int(g.integers(300, 5000))
+    paged = bool(g.integers(0, 2))
+    ragged = bool(g.integers(0, 2))
+    kw = dict(layers=2 * layer_group, layer_group=layer_group, batch=int(g.integers(1, 4)), q_heads=hkv * gq,
+              kv_heads=hkv, context=context, steps=int(g.integers(2, 6)), refresh=refresh,
+              top_k=int(g.choice([0, 1, 7, 64, 200, 700])), window=int(g.choice([0, 1, 16, 100, 600])),
+              sinks=int(g.choice([0, 1, 4, 33])), dilate_r=int(g.choice([0, 1, 2])),
+              heavy_hitters=int(g.choice([0, 8])), decay_span=int(g.choice([0, 64])), seed=1000 + seed,
+              halo=float(g.choice([0.0, 0.7])), q_scale=float(g.choice([1.0, 3.0])),
+              page_size=16 if paged else 0, min_context=max(40, context // 3) if ragged else 0,
+              psaw_layer_start=int(g.choice([0, 0, 1, 2])))
+    if kw["heavy_hitters"] and context - kw["window"] - kw["decay_span"] - kw["sinks"] < 16:
+        kw["heavy_hitters"] = 0
+    return small(f"random{seed}", **kw), paged, bool(g.integers(0, 2)) and gq > 1
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", list(range(14)))
+def test_random_schedules(cuda_device, seed):
+    """Seeded random shapes and budgets (zero and oversized budgets, windows longer than the
+    context, one or several layer groups, paged and ragged caches, sliding windows, group-shared
+    sets): every unit of every (layer, step) against the oracle."""
+    w, paged, group_sets = _random_workload(seed)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=group_sets)
+    assert st["checked"] == w.layers * w.steps * w.batch * w.q_heads
