@@ -685,3 +685,51 @@ def test_random_schedules(cuda_device, seed):
     w, paged, group_sets = _random_workload(seed)
     st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=group_sets)
     assert st["checked"] == w.layers * w.steps * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
+def test_group_sets_stage_calls(cuda_device):
+    """The stage-by-stage entry points with group-shared sets: prhs_score_topk hands every head
+    of a group the group's S* (ranked by the group maximum), prhs_build_index_set the group's
+    set, and the explicit-list attention over it equals the fused step."""
+    w = small(q_heads=8, kv_heads=2, context=3000, top_k=96, seed=91)
+    gq = 4
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = W.seq_lens_at(w, 0)
+    ctx = H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device, flags=P.PRHS_GROUP_SETS)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    oi = torch.empty(w.batch, w.q_heads, w.top_k, dtype=torch.int32, device=cuda_device)
+    oc = torch.empty(w.batch, w.q_heads, dtype=torch.int32, device=cuda_device)
+    ol = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    ctx.score_topk(0, 0, q, view, sched, w.batch, oi, oc, ol)
+    assert ctx.check() == 0
+    qh = H.np32(q)
+    for b in range(w.batch):
+        t = int(t_host[b])
+        for kvh in range(w.kv_heads):
+            heads = [O.dense_scores(qh[b, kvh * gq + j], H.np32(k[b, kvh]), t) for j in range(gq)]
+            ag = O.group_logits(heads)
+            want = O.topk_middle(ag, t, w.sinks, w.window, w.top_k)
+            for j in range(gq):
+                h = kvh * gq + j
+                got = oi[b, h, : int(oc[b, h])].cpu().numpy().astype(np.int64)
+                H.check_topk_legal(ag, got, want, f"unit ({b},{h})")
+                assert torch.equal(oi[b, h], oi[b, kvh * gq])
+                assert abs(float(ol[b, h]) - O.logsumexp(heads[j])) <= 1e-4      # log-sum-exp stays per head
+    cap = ctx.index_capacity
+    idx = torch.empty(w.batch, w.q_heads, cap, dtype=torch.int32, device=cuda_device)
+    cnt = torch.empty(w.batch, w.q_heads, dtype=torch.int32, device=cuda_device)
+    ctx.build_index_set(0, 0, sched, view, w.batch, idx, cnt)
+    out_a = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    out_b = torch.empty_like(out_a)
+    ctx.sparse_decode_attn(q, view, idx, cnt, w.batch, out_a)
+    ctx.decode_step(0, 0, sched, q, view, w.batch, out_b)
+    assert ctx.check() == 0
+    for b in range(w.batch):
+        for h in range(w.q_heads):
+            assert int(cnt[b, h]) == int(cnt[b, h - h % gq])
+            assert torch.equal(idx[b, h, : int(cnt[b, h])], idx[b, h - h % gq, : int(cnt[b, h])])
+    assert float((out_a.float() - out_b.float()).abs().max()) <= 2e-2     # different kernels, same set
+    ctx.close()
