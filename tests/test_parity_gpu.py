@@ -733,3 +733,49 @@ def test_group_sets_stage_calls(cuda_device):
             assert torch.equal(idx[b, h, : int(cnt[b, h])], idx[b, h - h % gq, : int(cnt[b, h])])
     assert float((out_a.float() - out_b.float()).abs().max()) <= 2e-2     # different kernels, same set
     ctx.close()
+
+
+@pytest.mark.gpu
+def test_decode_step_in_a_cuda_graph(cuda_device):
+    """prhs_decode_step only enqueues work (no allocation, no synchronisation), so a step can be
+    captured into a CUDA graph and replayed: lengths and queries live in device buffers that the
+    caller updates between replays.  A retrieval step and a sharing step are captured once and
+    replayed over two blocks; results equal the direct calls bit for bit."""
+    w = small(steps=8, refresh=4, context=2600, seed=95)
+    k, v = W.make_kv(w, cuda_device)
+    q_all = W.make_queries(w, cuda_device)[0]
+    sched = H.make_sched(w, cuda_device)
+    direct = []
+    ctx = H.make_ctx(w)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    for n in range(w.steps):
+        view = P.make_view(k, v, W.seq_lens_at(w, n).to(cuda_device), max_seq_len=w.capacity)
+        ctx.decode_step(0, n, sched, q_all[n].contiguous(), view, w.batch, out)
+        direct.append(out.clone())
+    assert ctx.check() == 0
+    ctx.close()
+
+    ctx = H.make_ctx(w)
+    q_buf = torch.empty_like(q_all[0]).contiguous()
+    t_buf = torch.zeros(w.batch, dtype=torch.int32, device=cuda_device)
+    out_g = torch.empty_like(out)
+    view = P.make_view(k, v, t_buf, max_seq_len=w.capacity)
+    side = torch.cuda.Stream()
+    graphs = {}
+    with torch.cuda.stream(side):
+        for kind, step in (("retrieve", 0), ("share", 1)):
+            q_buf.copy_(q_all[step]); t_buf.copy_(W.seq_lens_at(w, step).to(cuda_device))
+            ctx.decode_step(0, step, sched, q_buf, view, w.batch, out_g, stream=side)     # warm-up outside capture
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                ctx.decode_step(0, step, sched, q_buf, view, w.batch, out_g, stream=torch.cuda.current_stream())
+            graphs[kind] = g
+    torch.cuda.synchronize()
+    for n in range(w.steps):
+        q_buf.copy_(q_all[n]); t_buf.copy_(W.seq_lens_at(w, n).to(cuda_device))
+        graphs["retrieve" if n % w.refresh == 0 else "share"].replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out_g, direct[n]), f"step {n}"
+    assert ctx.check() == 0
+    ctx.close()
