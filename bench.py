@@ -252,10 +252,49 @@ def run_cuda(args):
     sampler = ClockSampler(local, uuid=str(torch.cuda.get_device_properties(dev).uuid), period=0.002)
     sampler.start()
     launches0 = ctx.launch_count
+    # The K timed steps are captured once into a CUDA graph (prhs_decode_step only enqueues work) and
+    # the timed region is one replay of it: the same kernels on the same inputs without the
+    # per-launch host work.  --no-graph, or a failed capture, times direct launches instead.
+    graph = None
+    if not args.no_graph and not args.path_only and L > 1:      # (the capture counts the K steps' launches)
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            cap0 = ctx.launch_count
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                # thread-local capture mode: other threads (the clock sampler, a process group's
+                # watchdog) may touch the CUDA runtime while the steps are being captured
+                with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+                    cap = torch.cuda.current_stream()
+                    for i in range(Wn, Wn + Kn):
+                        ctx.decode_step(i % L, i // L, sched, q_all[i % L, i // L], views[i % L][i // L], B, out,
+                                        stream=cap)
+            torch.cuda.synchronize()
+            graph_launches = ctx.launch_count - cap0          # kernel nodes of the graph = launches per replay
+            graph.replay()            # untimed: the first replay also uploads the graph
+            torch.cuda.synchronize()
+            for i in range(Wn):       # back to the state the timed steps start from
+                step_device(i)
+        except Exception as e:                                                  # pragma: no cover
+            print(f"bench: CUDA graph capture failed ({e}); timing direct launches", file=sys.stderr)
+            graph = None
+            torch.cuda.synchronize()
+            for i in range(Wn):
+                step_device(i)
+    launches0 = ctx.launch_count
     barrier()
-    ms = timed_steps(Wn, Kn, step_device)
+    if graph is not None:
+        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_ev.record(stream)
+        graph.replay()
+        b_ev.record(stream)
+        torch.cuda.synchronize()
+        ms = [a_ev.elapsed_time(b_ev) / Kn] * Kn
+    else:
+        ms = timed_steps(Wn, Kn, step_device)
     barrier()
-    launches = ctx.launch_count - launches0
+    launches = graph_launches if graph is not None else ctx.launch_count - launches0
     dev_flags = ctx.check()
     assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
     total_ms = sum(ms)
@@ -392,6 +431,8 @@ def run_cuda(args):
         "config": workload_config(w, {
             "parallelism": f"replicas x{world} (no collective)",
             "cache_copies": L,
+            "launch": ("the K timed steps are one replay of a CUDA graph captured from the same prhs_decode_step calls"
+                       if graph is not None else "direct launches"),
             "kernel_timing": "event pairs inside the library around every launch, on a back-to-back replay of the "
                              "same K steps (the timed region itself carries no instrumentation)",
             "l2": (f"no flush: {L} independent copies of the layer's cache (4.3 GB each) visited round-robin, "
@@ -434,6 +475,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling captures)")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="time direct launches instead of one replay of a CUDA graph of the K steps")
     ap.add_argument("--rotate", type=int, default=4,
                     help="independent copies of the layer cache visited round-robin (1 = flush L2 instead)")
     ap.add_argument("--path-only", action="store_true", help="skip the dense, e2e and CPU legs")
