@@ -779,3 +779,16 @@ def test_decode_step_in_a_cuda_graph(cuda_device):
         assert torch.equal(out_g, direct[n]), f"step {n}"
     assert ctx.check() == 0
     ctx.close()
+
+
+@pytest.mark.gpu
+def test_group_sets_long_and_paged_sampled(cuda_device):
+    # the group-shared variant at the 128K shape and at the ragged paged serving mix
+    w = W.C4_LLAMA3_128K.scaled(steps=5)
+    units = [(0, 0), (1, 13), (3, 31)]
+    st = H.run_schedule_parity(w, cuda_device, units, group_sets=True)
+    assert st["checked"] == 5 * len(units) and not st["select_fallback"]
+    w = W.C5_SERVING.scaled(layers=4, steps=5, batch=6)
+    units = [(0, 0), (2, 9), (5, 31), (3, 16)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3], paged=True, group_sets=True)
+    assert st["checked"] == 5 * 3 * len(units)
