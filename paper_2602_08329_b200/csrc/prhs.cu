@@ -365,10 +365,12 @@ prhs_status do_retrieval(prhs_ctx* c, int layer, int step, const void* q, const 
     // One CTA of 512 threads per unit, two per SM: the kernel is a chain of short phases and wide
     // CTAs shorten it.  Where that would leave a second, partly filled wave (between two and four
     // units per SM) 256-thread CTAs, four to an SM, take all units in one wave instead (the 512
-    // units of a 16 x 32-head batch: 66 us against 74 us).
+    // units of a 16 x 32-head batch: 66 us against 74 us); with at most one unit per SM the CTA
+    // takes all 1024 threads (128 units of 131 K logits: 53 us against 63 us).
     const int units = batch * c->cfg.num_q_heads / p.unit_mul;
     int threads = kSelMaxThreads;
     if (units > 2 * c->sm_count && units <= 4 * c->sm_count && c->sel_smem <= 56 * 1024) threads = kSelMaxThreads / 2;
+    if (units <= c->sm_count) threads = 2 * kSelMaxThreads;     // one CTA per SM at most: the widest CTA
     LaunchScope ls(c, PRHS_KIND_SELECT, st);
     select_kernel<<<units, threads, c->sel_smem, st>>>(p);
   }

@@ -1,7 +1,7 @@
 // Retrieval pass, part 2: exact top-k over the middle range (Sec. 4.1 "Selection
 // Criteria"), descending-logit order with ties broken by lower position, then the
 // neighbour dilation of Eq. 10.  One CTA per (sequence, query head); any multiple of 32 threads
-// up to 512 works, 512 is what the library launches.
+// up to 1024 works; the library launches 512, or 256 / 1024 when that fills the SMs better.
 //
 // Fast path: every warp takes a stratified 1-in-16 sample of the unit's logits and finds by
 // bisection on the top 13 key bits (a compare per sample and one warp reduction per bit) the
@@ -416,7 +416,7 @@ __device__ __forceinline__ void block_merge_sort_desc(unsigned long long* buf, u
   }
 }
 
-__global__ void __launch_bounds__(kSelMaxThreads, 2) select_kernel(SelectParams p) {
+__global__ void __launch_bounds__(2 * kSelMaxThreads, 1) select_kernel(SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem_raw);                     // kHistWords
   uint32_t* misc = hist + kHistWords;                                         // kSelMiscWords
