@@ -320,6 +320,27 @@ const char* prhs_kernel_kind_name(int32_t kind);
 /* Number of kernels this context has launched since creation (host-side counter). */
 int64_t prhs_launch_count(const prhs_ctx* ctx);
 
+/* Diagnostic for callers that build their own lists for prhs_sparse_decode_attn: checks on the
+ * device that every (b, h) list is strictly ascending (hence free of duplicates), lies inside
+ * [0, t_b) and is no longer than idx_stride.  host_num_bad receives the number of offending
+ * units, host_bad_units (host int32 [batch][Hq], or NULL) a 0 / 1 mark per unit.  The attention
+ * kernels skip and flag out-of-range entries on their own; order and uniqueness are only
+ * checked here.  Synchronises the stream. */
+prhs_status prhs_validate_index_lists(prhs_ctx* ctx, const prhs_kv_view* kv, const int32_t* idx,
+                                      const int32_t* count, int32_t idx_stride, int32_t batch,
+                                      int32_t* host_bad_units, int32_t* host_num_bad, void* stream);
+
+/* Checkpoint of the shared-set state (no counterpart in the paper): everything a context carries
+ * from one decode step to the next -- the stored S*, S^ and their sizes per (layer group,
+ * sequence, head, slot), the lengths at the last retrieval, the cosine gate's block history and
+ * decisions, and where every layer group stands in its schedule -- as one flat host buffer of
+ * prhs_state_bytes() bytes.  Import restores it into a context created with the SAME
+ * prhs_config (PRHS_ERR_INVALID_ARG otherwise); decoding then continues as if uninterrupted,
+ * bit for bit.  The KV cache itself belongs to the caller.  Both calls synchronise the stream. */
+int64_t prhs_state_bytes(const prhs_ctx* ctx);
+prhs_status prhs_state_export(prhs_ctx* ctx, void* host_buf, int64_t bytes, void* stream);
+prhs_status prhs_state_import(prhs_ctx* ctx, const void* host_buf, int64_t bytes, void* stream);
+
 /* Self-test of the failure path of the TMA kernels (no counterpart in the paper): launches one
  * thread that waits, with the given budget in SM cycles (1 .. 2e8, about 0.1 s), on a barrier
  * that nothing completes.  The wait must give up: *host_gave_up = 1, PRHS_FLAG_TIMEOUT is set in

@@ -28,7 +28,7 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_sparse_decode_attn", "prhs_dense_decode_attn", "prhs_decode_step",
            "prhs_decode_step_host", "prhs_decode_step_host_async", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
-           "prhs_launch_count", "prhs_selftest_wait", "prhs_last_error", "prhs_version", "prhs_profile_begin",
+           "prhs_launch_count", "prhs_selftest_wait", "prhs_state_bytes", "prhs_state_export", "prhs_state_import", "prhs_validate_index_lists", "prhs_last_error", "prhs_version", "prhs_profile_begin",
            "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate"]
 NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
@@ -99,6 +99,10 @@ def load() -> C.CDLL:
         "prhs_profile_end": (st, [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]),
         "prhs_kernel_kind_name": (C.c_char_p, [i32]),
         "prhs_launch_count": (C.c_int64, [vp]),
+        "prhs_validate_index_lists": (st, [vp, C.POINTER(KvView), vp, vp, i32, i32, vp, C.POINTER(C.c_int32), vp]),
+        "prhs_state_bytes": (C.c_int64, [vp]),
+        "prhs_state_export": (st, [vp, vp, C.c_int64, vp]),
+        "prhs_state_import": (st, [vp, vp, C.c_int64, vp]),
         "prhs_selftest_wait": (st, [vp, C.c_int64, C.POINTER(C.c_int32), vp]),
         "prhs_last_error": (C.c_char_p, [vp]),
         "prhs_version": (C.c_char_p, []),
@@ -264,6 +268,24 @@ class Context:
         self._ck(self.lib.prhs_profile_end(self.h, _stream(stream), ms, n))
         return {self.lib.prhs_kernel_kind_name(i).decode(): (float(ms[i]), int(n[i]))
                 for i in range(KERNEL_KINDS)}
+
+    def validate_index_lists(self, view, idx, count, batch, stream=None):
+        """(number of bad units, CPU int32 [batch][Hq] marks) for explicit index lists."""
+        marks = torch.empty(batch, self.cfg.num_q_heads, dtype=torch.int32)
+        nbad = C.c_int32(-1)
+        self._ck(self.lib.prhs_validate_index_lists(self.h, C.byref(view), _ptr(idx), _ptr(count), idx.shape[-1],
+                                                    batch, marks.data_ptr(), C.byref(nbad), _stream(stream)))
+        return nbad.value, marks
+
+    def state_export(self, stream=None) -> torch.Tensor:
+        """The shared-set state as a flat CPU uint8 tensor (see prhs_state_export)."""
+        buf = torch.empty(self.lib.prhs_state_bytes(self.h), dtype=torch.uint8)
+        self._ck(self.lib.prhs_state_export(self.h, buf.data_ptr(), buf.numel(), _stream(stream)))
+        return buf
+
+    def state_import(self, buf: torch.Tensor, stream=None):
+        assert buf.dtype == torch.uint8 and buf.device.type == "cpu" and buf.is_contiguous()
+        self._ck(self.lib.prhs_state_import(self.h, buf.data_ptr(), buf.numel(), _stream(stream)))
 
     def selftest_wait(self, budget_cycles=1_000_000, stream=None) -> int:
         gave_up = C.c_int32(-1)

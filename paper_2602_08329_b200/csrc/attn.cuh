@@ -975,6 +975,30 @@ __global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunk
   }
   lse_full[i] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
 }
+// Diagnostic: is every unit's index list strictly ascending (hence unique), inside [0, t_b) and
+// no longer than its stride?  One warp per (b, h); bad[unit] = 1 where it is not, *nbad counts.
+__global__ void __launch_bounds__(128)
+validate_lists_kernel(const int* __restrict__ idx, const int* __restrict__ count, int idx_stride,
+                      const int* __restrict__ seq_lens, int num_q_heads, int units, int* bad, int* nbad) {
+  const int unit = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (unit >= units) return;
+  const int t = __ldg(seq_lens + unit / num_q_heads);
+  const int n = __ldg(count + unit);
+  const int* l = idx + (long long)unit * idx_stride;
+  bool ok = n >= 0 && n <= idx_stride;
+  const int m = min(max(n, 0), idx_stride);
+  for (int i = lane; i < m; i += 32) {
+    const int x = __ldg(l + i);
+    if (x < 0 || x >= t) ok = false;
+    if (i > 0 && __ldg(l + i - 1) >= x) ok = false;
+  }
+  ok = __all_sync(0xffffffffu, ok);
+  if (lane == 0) {
+    bad[unit] = ok ? 0 : 1;
+    if (!ok) atomicAdd(nbad, 1);
+  }
+}
+
 // One launch that takes a decode step's inputs straight from PINNED, device-mapped host memory:
 // the queries into the staging buffer, the new K and V rows into the cache at position t_b - 1,
 // the lengths into the device array.  Replaces four host-to-device copies and the append

@@ -465,6 +465,113 @@ prhs_status prhs_selftest_wait(prhs_ctx* ctx, int64_t budget_cycles, int32_t* ho
   return PRHS_OK;
 }
 
+prhs_status prhs_validate_index_lists(prhs_ctx* ctx, const prhs_kv_view* kv, const int32_t* idx,
+                                      const int32_t* count, int32_t idx_stride, int32_t batch,
+                                      int32_t* host_bad_units, int32_t* host_num_bad, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!kv || !kv->seq_lens || !idx || !count || !host_num_bad) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (idx_stride < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "idx_stride must be >= 1");
+  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
+  cudaStream_t st = as_stream(stream);
+  const int units = batch * ctx->cfg.num_q_heads;
+  int* bad = ctx->count;                       // [units] scratch of the context
+  int* nbad = reinterpret_cast<int*>(ctx->tickets);   // zero between launches; restored below
+  {
+    LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+    validate_lists_kernel<<<(units + 3) / 4, 128, 0, st>>>(idx, count, idx_stride, kv->seq_lens,
+                                                           ctx->cfg.num_q_heads, units, bad, nbad);
+  }
+  PRHS_CUDA(ctx, cudaGetLastError());
+  PRHS_CUDA(ctx, cudaMemcpyAsync(host_num_bad, nbad, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (host_bad_units)
+    PRHS_CUDA(ctx, cudaMemcpyAsync(host_bad_units, bad, (size_t)units * sizeof(int), cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(ctx, cudaMemsetAsync(nbad, 0, sizeof(int), st));
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+// ---- checkpoint of the shared-set state --------------------------------------------------
+namespace {
+constexpr uint32_t kStateMagic = 0x50724853u;   // "PrHS"
+constexpr uint32_t kStateVersion = 1u;
+struct StateHeader {
+  uint32_t magic, version;
+  prhs_config cfg;
+  int32_t num_groups, slots, last_layer_group, last_share_gq;
+};
+struct StatePart { void* dev; size_t bytes; };
+std::vector<StatePart> state_parts(prhs_ctx* c) {
+  const size_t U = units_max(c), G = c->num_groups, SL = c->slots, mk = c->cfg.max_k, hc = c->shat_cap;
+  return {{c->sstar_desc, G * U * SL * mk * sizeof(int)},   {c->sstar_asc, G * U * SL * mk * sizeof(int)},
+          {c->shat_asc, G * U * SL * hc * sizeof(int)},     {c->n_star, G * U * SL * sizeof(int)},
+          {c->n_hat, G * U * SL * sizeof(int)},             {c->anchor_t, G * c->cfg.max_batch * sizeof(int)},
+          {c->qhist, G * U * SL * kHeadDim * sizeof(__nv_bfloat16)}, {c->set_of_pos, G * U * SL * sizeof(int)},
+          {c->nsets, G * U * sizeof(int)},                  {c->g_need, G * U * sizeof(int)},
+          {c->g_slot, G * U * sizeof(int)},                 {c->g_ref, G * U * sizeof(int)}};
+}
+size_t state_total(prhs_ctx* c) {
+  size_t n = sizeof(StateHeader) + 2 * (size_t)c->num_groups * sizeof(int32_t);
+  for (const StatePart& p : state_parts(c)) n += (p.bytes + 15) & ~(size_t)15;
+  return n;
+}
+}  // namespace
+
+int64_t prhs_state_bytes(const prhs_ctx* ctx) { return ctx ? (int64_t)state_total(const_cast<prhs_ctx*>(ctx)) : 0; }
+
+prhs_status prhs_state_export(prhs_ctx* ctx, void* host_buf, int64_t bytes, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!host_buf) return fail(ctx, PRHS_ERR_INVALID_ARG, "state export: NULL buffer");
+  if (bytes < (int64_t)state_total(ctx)) return fail(ctx, PRHS_ERR_CAPACITY, "state export: buffer below prhs_state_bytes()");
+  cudaStream_t st = as_stream(stream);
+  unsigned char* o = static_cast<unsigned char*>(host_buf);
+  StateHeader h{kStateMagic, kStateVersion, ctx->cfg, ctx->num_groups, ctx->slots, ctx->last_layer_group,
+                ctx->last_share_gq};
+  std::memcpy(o, &h, sizeof(h));
+  o += sizeof(h);
+  std::memcpy(o, ctx->anchor_step.data(), ctx->num_groups * sizeof(int32_t));
+  o += ctx->num_groups * sizeof(int32_t);
+  std::memcpy(o, ctx->gate_step.data(), ctx->num_groups * sizeof(int32_t));
+  o += ctx->num_groups * sizeof(int32_t);
+  for (const StatePart& p : state_parts(ctx)) {
+    PRHS_CUDA(ctx, cudaMemcpyAsync(o, p.dev, p.bytes, cudaMemcpyDeviceToHost, st));
+    o += (p.bytes + 15) & ~(size_t)15;
+  }
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  return PRHS_OK;
+}
+
+prhs_status prhs_state_import(prhs_ctx* ctx, const void* host_buf, int64_t bytes, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!host_buf) return fail(ctx, PRHS_ERR_INVALID_ARG, "state import: NULL buffer");
+  if (bytes < (int64_t)sizeof(StateHeader)) return fail(ctx, PRHS_ERR_INVALID_ARG, "state import: truncated buffer");
+  const unsigned char* in = static_cast<const unsigned char*>(host_buf);
+  StateHeader h;
+  std::memcpy(&h, in, sizeof(h));
+  if (h.magic != kStateMagic || h.version != kStateVersion)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "state import: not a state buffer of this library version");
+  if (std::memcmp(&h.cfg, &ctx->cfg, sizeof(prhs_config)) != 0 || h.num_groups != ctx->num_groups ||
+      h.slots != ctx->slots)
+    return fail(ctx, PRHS_ERR_INVALID_ARG, "state import: the buffer was exported from a different configuration");
+  if (bytes < (int64_t)state_total(ctx)) return fail(ctx, PRHS_ERR_INVALID_ARG, "state import: truncated buffer");
+  cudaStream_t st = as_stream(stream);
+  in += sizeof(h);
+  std::memcpy(ctx->anchor_step.data(), in, ctx->num_groups * sizeof(int32_t));
+  in += ctx->num_groups * sizeof(int32_t);
+  std::memcpy(ctx->gate_step.data(), in, ctx->num_groups * sizeof(int32_t));
+  in += ctx->num_groups * sizeof(int32_t);
+  for (const StatePart& p : state_parts(ctx)) {
+    PRHS_CUDA(ctx, cudaMemcpyAsync(p.dev, in, p.bytes, cudaMemcpyHostToDevice, st));
+    in += (p.bytes + 15) & ~(size_t)15;
+  }
+  PRHS_CUDA(ctx, cudaStreamSynchronize(st));
+  ctx->last_layer_group = h.last_layer_group;
+  ctx->last_share_gq = h.last_share_gq;
+  ctx->last_set = SetRef{};
+  ctx->last_seq_lens = nullptr;
+  ctx->last_batch = 0;
+  return PRHS_OK;
+}
+
 int32_t prhs_index_capacity(const prhs_ctx* ctx) { return ctx ? ctx->idx_cap : 0; }
 
 int32_t prhs_scores_ld(const prhs_ctx* ctx) { return ctx ? ctx->ld : 0; }

@@ -792,3 +792,80 @@ def test_group_sets_long_and_paged_sampled(cuda_device):
     units = [(0, 0), (2, 9), (5, 31), (3, 16)]
     st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3], paged=True, group_sets=True)
     assert st["checked"] == 5 * 3 * len(units)
+
+
+# ----------------------------------------------------------------- checkpoint of the set state
+@pytest.mark.gpu
+@pytest.mark.parametrize("gated", [False, True])
+def test_state_export_import_resumes_bit_for_bit(cuda_device, gated):
+    """Export the shared-set state in the middle of a block, import it into a fresh context and
+    continue there: outputs and index sets equal those of the uninterrupted context, for the
+    fixed schedule (with layer groups) and for the cosine gate (block history included)."""
+    w = small(layers=4, layer_group=2, steps=9, refresh=4, q_heads=8, kv_heads=2, context=2100, seed=97,
+              sigma=0.7 if gated else 0.05, sim_threshold=0.8 if gated else None)
+    kv = {l: (k, v) for l, k, v in W.make_layer_kv(w, cuda_device)}
+    q = W.make_queries(w, cuda_device)
+    sched = H.make_sched(w, cuda_device)
+    ctx_a, ctx_b = H.make_ctx(w), None
+    out_a = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    out_b = torch.empty_like(out_a)
+    cut = 6          # after step 5: the second block is two steps old
+    for n in range(w.steps):
+        view_t = W.seq_lens_at(w, n).to(cuda_device)
+        if n == cut:
+            blob = ctx_a.state_export()
+            assert blob.numel() == ctx_a.lib.prhs_state_bytes(ctx_a.h)
+            ctx_b = H.make_ctx(w)
+            ctx_b.state_import(blob)
+            with pytest.raises(P.PrhsError):                 # another configuration refuses the buffer
+                other = H.make_ctx(w.scaled(top_k=w.top_k + 8))
+                try:
+                    other.state_import(blob)
+                finally:
+                    other.close()
+        for l in range(w.layers):
+            view = P.make_view(kv[l][0], kv[l][1], view_t, max_seq_len=w.capacity)
+            ctx_a.decode_step(l, n, sched, q[l, n].contiguous(), view, w.batch, out_a)
+            if ctx_b is not None:
+                ctx_b.decode_step(l, n, sched, q[l, n].contiguous(), view, w.batch, out_b)
+                assert torch.equal(out_a, out_b), f"layer {l} step {n}"
+                ia, ca = ctx_a.get_index_set(w.batch)
+                ib, cb = ctx_b.get_index_set(w.batch)
+                assert torch.equal(ca, cb)
+                for b in range(w.batch):
+                    for h in range(w.q_heads):
+                        assert torch.equal(ia[b, h, : int(ca[b, h])], ib[b, h, : int(cb[b, h])])
+    assert ctx_a.check() == 0 and ctx_b.check() == 0
+    ctx_a.close(); ctx_b.close()
+
+
+@pytest.mark.gpu
+def test_validate_index_lists(cuda_device):
+    w = small(context=2000, seed=98)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = W.seq_lens_at(w, 0).to(cuda_device)
+    view = P.make_view(k, v, t_dev, max_seq_len=w.capacity)
+    ctx = H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    ctx.decode_step(0, 0, sched, q, view, w.batch, out)
+    cap = ctx.index_capacity
+    idx = torch.empty(w.batch, w.q_heads, cap, dtype=torch.int32, device=cuda_device)
+    cnt = torch.empty(w.batch, w.q_heads, dtype=torch.int32, device=cuda_device)
+    ctx.build_index_set(0, 0, sched, view, w.batch, idx, cnt)
+    nbad, marks = ctx.validate_index_lists(view, idx, cnt, w.batch)
+    assert nbad == 0 and int(marks.sum()) == 0                   # the library's own lists are clean
+    bad = idx.clone()
+    bad[0, 1, 5] = bad[0, 1, 4]                                   # a duplicate
+    bad[1, 0, 3], bad[1, 0, 2] = idx[1, 0, 2].item(), idx[1, 0, 3].item()    # out of order
+    bad[1, 3, 0] = -7                                             # out of range
+    cnt2 = cnt.clone()
+    cnt2[0, 2] = cap + 1                                          # longer than the stride
+    nbad, marks = ctx.validate_index_lists(view, bad, cnt2, w.batch)
+    assert nbad == 4
+    assert marks.tolist() == [[0, 1, 1, 0], [1, 0, 0, 1]]
+    ctx.decode_step(0, 1, sched, q, P.make_view(k, v, W.seq_lens_at(w, 1).to(cuda_device), max_seq_len=w.capacity),
+                    w.batch, out)                                 # the scratch it borrowed is back in order
+    assert ctx.check() == 0
+    ctx.close()
