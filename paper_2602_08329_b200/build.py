@@ -29,10 +29,11 @@ def stale() -> bool:
     return any(os.path.getmtime(s) > t for s in sources())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, nvtx: bool = False) -> str:
+    """nvtx=True (`--nvtx`) puts every launch in an NVTX range named after its stage."""
     if not force and not stale():
         return LIB
-    cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + (["-DPRHS_NVTX", "-ldl"] if nvtx else []) + \
           ["-o", LIB, os.path.join(CSRC, "prhs.cu")]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
@@ -43,4 +44,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, nvtx="--nvtx" in sys.argv))

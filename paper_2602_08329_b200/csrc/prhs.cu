@@ -10,6 +10,10 @@
 #include <string>
 #include <vector>
 
+#ifdef PRHS_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 #include "attn.cuh"
 #include "common.cuh"
 #include "attn_group.cuh"
@@ -157,11 +161,20 @@ prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
 }
 
 // Brackets one kernel launch: counts it and, in profiling mode, records an event pair.
+// With -DPRHS_NVTX every launch also sits in an NVTX range named after its kind (a timeline tool
+// then shows the stages of a step); off by default.
+#ifdef PRHS_NVTX
+static const char* const kKindNames[PRHS_KERNEL_KINDS] = {"prhs score", "prhs select", "prhs build_set",
+                                                          "prhs attn_sparse", "prhs attn_dense", "prhs misc"};
+#endif
 struct LaunchScope {
   prhs_ctx* c;
   cudaStream_t st;
   int slot = -1;
   LaunchScope(prhs_ctx* ctx, int kind, cudaStream_t stream) : c(ctx), st(stream) {
+#ifdef PRHS_NVTX
+    nvtxRangePushA(kKindNames[kind]);
+#endif
     c->launches++;
     if (c->prof_on && c->prof_used < (int)c->prof.size()) {
       slot = c->prof_used++;
@@ -171,6 +184,9 @@ struct LaunchScope {
   }
   ~LaunchScope() {
     if (slot >= 0) cudaEventRecord(c->prof[slot].b, st);
+#ifdef PRHS_NVTX
+    nvtxRangePop();
+#endif
   }
 };
 
