@@ -328,6 +328,18 @@ def run_cuda(args):
         step_device(i)
         _, cnt = ctx.get_index_set(B)
         counts.append(int(cnt.sum()))
+    # ---- dropped attention mass of the sets in use (Sec. 2.3), untimed: the same steps with the
+    # diagnostic on (a full log-sum-exp pass on the sharing steps)
+    deltas = []
+    if not args.path_only:
+        sched_d = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
+                                  flags=P.PRHS_WANT_DELTA)
+        dlt = torch.empty(B, Hq, dtype=torch.float32, device=dev)
+        rewind()
+        for i in range(Wn, Wn + Kn):
+            ctx.decode_step(i % L, i // L, sched_d, q_all[i % L, i // L], views[i % L][i // L], B, out, dlt)
+            deltas.append(dlt.clone())
+        deltas = torch.stack(deltas)
     t_cpu = t_all.cpu()
     score_bytes = [int(t_cpu[i // L].sum()) * Hkv * 256 for i in range(Wn, Wn + Kn) if is_refresh(i)]
     gather_bytes = [c * 512 for c in counts]
@@ -448,6 +460,9 @@ def run_cuda(args):
         "path_achieved_gbs": path_gbs, "path_frac_of_measured_peak": path_gbs / hbm_peak,
         "path_frac_of_8tbs": path_gbs / 8000.0,
         "mean_set_size": sum(counts) / (len(counts) * B * Hq),
+        "delta": {"mean": float(deltas.mean()), "max": float(deltas.max()),
+                  "note": "dropped attention mass over all (step, sequence, head) of the timed steps; synthetic "
+                          "keys at q_scale 1 have far flatter attention than a trained model"},
         "retrieval_ratio": len(score_bytes) / Kn,
         "select_fallback": bool(dev_flags & P.PRHS_FLAG_SELECT_FALLBACK),
         "roofline": roofline, "kernels": kernels,
