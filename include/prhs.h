@@ -16,13 +16,16 @@
  *   - head_dim is 128.  q, K, V and attention outputs are bf16; logits, log-sum-exps and
  *     delta are fp32; indices and counts are int32.
  *   - Query head h uses KV head h / (num_q_heads / num_kv_heads).  Index sets are per
- *     (sequence, query head).
+ *     (sequence, query head), as in the paper; PRHS_GROUP_SETS is a labelled variant with one
+ *     set per (sequence, KV head).
  *   - "device" pointers are CUDA device memory owned by the caller unless stated; "host"
  *     pointers are ordinary (preferably pinned) host memory.  The library never frees or
  *     keeps caller memory beyond the call (asynchronous work on `stream` excepted).
  *   - Every call validates its arguments on the host and returns a prhs_status; nothing
- *     traps, asserts or spins on the device.  Device-side anomalies (an index outside
- *     [0, t_b), a candidate overflow) are recorded in a flag word read by prhs_check().
+ *     traps or asserts on the device, no kernel waits on another kernel or CTA, and the only
+ *     waits there are (on the copy engine's barriers) are bounded.  Device-side anomalies (an
+ *     index outside [0, t_b), a page id outside the pool, a wait that ran out) are recorded in
+ *     a flag word read by prhs_check().
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default
  *     stream) and is asynchronous unless stated.  Workspaces and the shared-set state are
  *     allocated in prhs_create(); no call below allocates.
