@@ -17,4 +17,6 @@ def cuda_device():
     import torch
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
+    from paper_2602_08329_b200 import build
+    build.build()          # no-op when libprhs.so is newer than its sources
     return torch.device("cuda:0")
