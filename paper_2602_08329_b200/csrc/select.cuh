@@ -491,8 +491,14 @@ __global__ void __launch_bounds__(2 * kSelMaxThreads, 1) select_kernel(SelectPar
       const int sec_stride = max(kSampleStride, (nsec + 2 * nt - 1) / (2 * nt));
       const int S = nsec / sec_stride;               // sampled sectors
       const int slot = lane * nw + warp;
-      const int want = (int)((7ll * kk * 8 * S) / (4ll * n)) + 16;
-      const int rw = (want + nw - 1) / nw;
+      // sampled logits that should reach the threshold: 1.75 x the expected number above the
+      // k-th logit, plus 16; but no more than would fill 85 % of the list (a long context with a
+      // large budget leaves little room: better a thinner margin than a certain overflow)
+      int want = (int)((7ll * kk * 8 * S) / (4ll * n)) + 16;
+      const int room = (int)((17ll * p.cand_cap * 8 * S) / (20ll * n));
+      const bool tight = want > room;
+      if (tight) want = max(room, (int)((8ll * kk * S) / n) + 1);
+      const int rw = tight ? max(1, want / nw) : (want + nw - 1) / nw;   // per warp; rounded towards the room
       uint32_t prefix;
       if (2 * S <= nt) prefix = sample_quantile_half(g + a8, S, sec_stride, nw, rw);
       else if (S <= nt) prefix = sample_quantile<1>(g + a8, S, sec_stride, nt, slot, rw);

@@ -869,3 +869,14 @@ def test_validate_index_lists(cuda_device):
                     w.batch, out)                                 # the scratch it borrowed is back in order
     assert ctx.check() == 0
     ctx.close()
+
+
+@pytest.mark.gpu
+def test_maximum_context_length(cuda_device):
+    """One sequence at the library's largest context (2^20 positions, 4096 winners): the sparse
+    sample, the single-bitmap layout and a million-row tensor map, against the oracle."""
+    n = (1 << 20) - 8
+    w = small("max_context", context=n, steps=2, refresh=2, batch=1, q_heads=2, kv_heads=1, top_k=4096,
+              window=256, sinks=4, heavy_hitters=64, decay_span=512, seed=99)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), check_scores=True)
+    assert st["checked"] == 2 * 2 and not st["select_fallback"]
