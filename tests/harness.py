@@ -112,23 +112,25 @@ class _HostSlices:
 
 
 def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, want_delta=True,
-                        paged=False, check_scores=True, group_sets=False):
+                        paged=False, check_scores=True, group_sets=False, dilate_anchor=False, dilate_m=-1):
     """Drive prhs_decode_step over the workload's schedule and compare sampled (b, h) units.
 
     The oracle follows the same schedule.  Where the GPU retrieved, its S* is first checked
     for legality against the oracle's own top-k (near-ties at the k-th logit only) and then
     handed to the oracle as an override, so that every later comparison in the block
     (dilation, shared sets, attention, delta) is exact.
-    `group_sets` runs the labelled variant with one set per KV head (ranking by the group's
+    `dilate_anchor` makes the retrieving call attend over the dilated set too; `dilate_m` fixes the
+    number of dilated winners instead of k/3.  `group_sets` runs the labelled variant with one set per KV head (ranking by the group's
     maximum logit) on both sides.
     Returns a dict of summary statistics.
     """
     layers = list(range(w.layers)) if layers is None else layers
     steps = w.steps if steps is None else steps
-    ctx = make_ctx(w)
-    flags = (P.PRHS_WANT_DELTA if want_delta else 0) | (P.PRHS_GROUP_SETS if group_sets else 0)
-    sched = make_sched(w, device, flags=flags)
-    osched = oracle_sched(w, group_sets=group_sets)
+    ctx = make_ctx(w, max_dilate_m=dilate_m)
+    flags = ((P.PRHS_WANT_DELTA if want_delta else 0) | (P.PRHS_GROUP_SETS if group_sets else 0) |
+             (P.PRHS_DILATE_ANCHOR if dilate_anchor else 0))
+    sched = make_sched(w, device, flags=flags, dilate_m=dilate_m)
+    osched = oracle_sched(w, group_sets=group_sets, dilate_anchor=dilate_anchor, dilate_m=dilate_m)
     orc = O.PrhsOracle(osched, w.q_heads, w.kv_heads)
     q_all = W.make_queries(w, device)
     kv = {l: (k, v) for l, k, v in W.make_layer_kv(w, device, layers=layers)}

@@ -880,3 +880,14 @@ def test_maximum_context_length(cuda_device):
               window=256, sinks=4, heavy_hitters=64, decay_span=512, seed=99)
     st = H.run_schedule_parity(w, cuda_device, all_units(w), check_scores=True)
     assert st["checked"] == 2 * 2 and not st["select_fallback"]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("anchor,m,r", [(True, -1, 1), (False, 0, 1), (True, 5, 2), (False, 48, 2), (True, 3, 0)])
+def test_dilation_options(cuda_device, anchor, m, r):
+    # the other reading of who attends over the dilated set (the retrieving call too), and an
+    # explicit number of dilated winners instead of k/3 (none, a few, all of them)
+    w = small(layers=2, layer_group=2, steps=5, refresh=2, q_heads=4, kv_heads=2, context=2300, seed=33, dilate_r=r,
+              halo=0.7)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), dilate_anchor=anchor, dilate_m=m)
+    assert st["checked"] == 2 * 5 * w.batch * w.q_heads
