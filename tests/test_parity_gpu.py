@@ -891,3 +891,23 @@ def test_dilation_options(cuda_device, anchor, m, r):
               halo=0.7)
     st = H.run_schedule_parity(w, cuda_device, all_units(w), dilate_anchor=anchor, dilate_m=m)
     assert st["checked"] == 2 * 5 * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
+def test_per_kernel_profile_counts(cuda_device):
+    w = small(steps=4, refresh=2)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0]
+    ctx = H.make_ctx(w)
+    sched = H.make_sched(w, cuda_device)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    n0 = ctx.launch_count
+    ctx.profile_begin()
+    for n in range(w.steps):
+        view = P.make_view(k, v, W.seq_lens_at(w, n).to(cuda_device), max_seq_len=w.capacity)
+        ctx.decode_step(0, n, sched, q[n].contiguous(), view, w.batch, out)
+    prof = ctx.profile_end()
+    assert {name: cnt for name, (ms, cnt) in prof.items() if cnt} == {"score": 2, "select": 2, "attn_sparse": 4}
+    assert all(ms > 0 for ms, cnt in prof.values() if cnt)
+    assert ctx.launch_count - n0 == 8
+    ctx.close()
