@@ -216,7 +216,7 @@ score_tma_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     const int lm_mi = lane >> 3, lm_r = lane & 7;
     for (int j = 0; j < nstages; ++j) {
       const int slot = j % kSTStages;
-      // every lane polls; the verdict is made uniform so that the warp leaves the loop together
+      // every lane polls; the outcome is made uniform so that the warp leaves the loop together
       if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8 * slot, (j / kSTStages) & 1, &sh_abort))) {
         if (lane == 0) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; }
         break;
