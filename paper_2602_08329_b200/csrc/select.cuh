@@ -482,7 +482,9 @@ __global__ void __launch_bounds__(2 * kSelMaxThreads, 1) select_kernel(SelectPar
     //    1.75 k/16 + 16 sampled logits of the CTA would reach if all warps saw the same
     //    distribution; the lower median of the warps' values is the threshold.
     float thr = -INFINITY;
-    if (n > p.cand_cap) {
+    // sample whenever listing every candidate would be much more than the ~2 k the threshold lets
+    // through (always when they would not fit)
+    if (n > p.cand_cap || (n >= 2048 && n > 4 * kk)) {
       const int nw = nt >> 5;
       // whole 32-byte sectors, one out of every sec_stride (>= 16: a 1-in-16 sample), at most two
       // per thread
