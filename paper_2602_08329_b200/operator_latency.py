@@ -1,6 +1,7 @@
 """Attention-operator latency of the library on the shapes of the paper's efficiency study.
 
     python -m paper_2602_08329_b200.operator_latency            # Table-3 shapes
+    python -m paper_2602_08329_b200.operator_latency --graph    # the same, blocks of s steps replayed from CUDA graphs
     python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C5 shapes
     python -m paper_2602_08329_b200.operator_latency --configs --group-sets   # one set per KV head (variant)
 
@@ -101,7 +102,74 @@ def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6, group_sets
             "unique_bytes": unique, "key_bytes": key_bytes}
 
 
-def table3(dev):
+def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6):
+    """Per-step device time (us) of a whole block of s decode steps (one retrieval, s - 1 sharing
+    steps) and of s dense steps, each block replayed from a CUDA graph: what a decode loop pays
+    once the per-launch host work is out of the way.  Blocks of independent cache copies are
+    replayed in turn."""
+    w = w.scaled(layers=copies, steps=s)
+    kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
+    q = W.make_queries(w, dev)
+    B, Hq = w.batch, w.q_heads
+    ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, w.top_k, w.window, w.sinks, max_dilate_r=w.dilate_r)
+    sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=s, dilate_r=w.dilate_r)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    lens = [W.seq_lens_at(w, n).to(dev) for n in range(s)]
+    views = [[P.make_view(kv[l][0], kv[l][1], lens[n], max_seq_len=w.capacity) for n in range(s)] for l in range(copies)]
+    side = torch.cuda.Stream()
+    graphs = {"sparse": [], "dense": []}
+    with torch.cuda.stream(side):
+        for l in range(copies):
+            for kind in ("sparse", "dense"):
+                def block(stream):
+                    for n in range(s):
+                        if kind == "sparse":
+                            ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out, stream=stream)
+                        else:
+                            ctx.dense_decode_attn(q[l, n], views[l][n], B, out, stream=stream)
+                block(side)
+                side.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                    block(torch.cuda.current_stream())
+                graphs[kind].append(g)
+    torch.cuda.synchronize()
+    res = {}
+    stream = torch.cuda.current_stream()
+    for kind in ("sparse", "dense"):
+        ts = []
+        for r in range(reps):
+            for g in graphs[kind]:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                g.replay()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if r > 0:
+                    ts.append(a.elapsed_time(b) * 1e3 / s)
+        res[kind] = statistics.median(ts)
+    assert ctx.check() == 0
+    ctx.close()
+    return res
+
+
+def table3(dev, graph=False):
+    if graph:
+        print("| BS | seqlen | k | dense us / step | s=8 us / step | s=16 us / step | dense / s=8 | dense / s=16 "
+              "| paper Flash / CPE-8 / CPE-16 ms (A100), ratios |")
+        print("|---|---|---|---|---|---|---|---|---|")
+        for batch in (8, 16):
+            for n in (1024, 2048, 4096):
+                k = n // 8 - 80
+                w = W.Workload(f"table3_b{batch}_{n}", layers=1, batch=batch, q_heads=32, kv_heads=32, context=n,
+                               steps=4, top_k=k, window=64, sinks=16, refresh=8, heavy_hitters=16,
+                               decay_span=min(512, n // 8), seed=100 + batch + n)
+                r8, r16 = time_blocks(w, dev, 8), time_blocks(w, dev, 16)
+                pf, p8, p16 = PAPER_TABLE3_MS[(batch, n)]
+                print(f"| {batch} | {n} | {k} | {r16['dense']:.1f} | {r8['sparse']:.1f} | {r16['sparse']:.1f} | "
+                      f"{r8['dense'] / r8['sparse']:.2f}x | {r16['dense'] / r16['sparse']:.2f}x | "
+                      f"{pf} / {p8} / {p16}, {pf / p8:.1f}x / {pf / p16:.1f}x |")
+        return
     print("| BS | seqlen | k | dense us | retrieval step us | sharing step us | amortised s=8 us | amortised s=16 us "
           "| dense / s=16 | paper Flash / CPE-8 / CPE-16 ms (A100) |")
     print("|---|---|---|---|---|---|---|---|---|---|")
@@ -140,6 +208,8 @@ def configs(dev, group_sets=False, only=None, batch=0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C5 shapes instead")
+    ap.add_argument("--graph", action="store_true",
+                    help="Table-3 shapes: whole blocks of s steps replayed from CUDA graphs (per-step time)")
     ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
     ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
     ap.add_argument("--group-sets", action="store_true",
@@ -152,7 +222,7 @@ def main():
     if args.configs:
         configs(dev, args.group_sets, args.only, args.batch)
     else:
-        table3(dev)
+        table3(dev, args.graph)
 
 
 if __name__ == "__main__":
