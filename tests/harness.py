@@ -112,13 +112,15 @@ class _HostSlices:
 
 
 def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, want_delta=True,
-                        paged=False, check_scores=True, group_sets=False, dilate_anchor=False, dilate_m=-1):
+                        paged=False, check_scores=True, group_sets=False, dilate_anchor=False, dilate_m=-1,
+                        ctx_over=None):
     """Drive prhs_decode_step over the workload's schedule and compare sampled (b, h) units.
 
     The oracle follows the same schedule.  Where the GPU retrieved, its S* is first checked
     for legality against the oracle's own top-k (near-ties at the k-th logit only) and then
     handed to the oracle as an override, so that every later comparison in the block
     (dilation, shared sets, attention, delta) is exact.
+    `ctx_over` overrides sizes of the context (a context larger than the workload).
     `dilate_anchor` makes the retrieving call attend over the dilated set too; `dilate_m` fixes the
     number of dilated winners instead of k/3.  `group_sets` runs the labelled variant with one set per KV head (ranking by the group's
     maximum logit) on both sides.
@@ -126,7 +128,7 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
     """
     layers = list(range(w.layers)) if layers is None else layers
     steps = w.steps if steps is None else steps
-    ctx = make_ctx(w, max_dilate_m=dilate_m)
+    ctx = make_ctx(w, max_dilate_m=dilate_m, **(ctx_over or {}))
     flags = ((P.PRHS_WANT_DELTA if want_delta else 0) | (P.PRHS_GROUP_SETS if group_sets else 0) |
              (P.PRHS_DILATE_ANCHOR if dilate_anchor else 0))
     sched = make_sched(w, device, flags=flags, dilate_m=dilate_m)

@@ -911,3 +911,17 @@ def test_per_kernel_profile_counts(cuda_device):
     assert all(ms > 0 for ms, cnt in prof.values() if cnt)
     assert ctx.launch_count - n0 == 8
     ctx.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("gated", [False, True])
+def test_context_larger_than_the_workload(cuda_device, gated):
+    # a context dimensioned for more sequences, layers, longer contexts and larger budgets than
+    # the calls use: state and workspaces are indexed by the configured maxima
+    w = small(layers=2, layer_group=2, steps=5, refresh=2, q_heads=8, kv_heads=2, context=1900, seed=44,
+              sim_threshold=0.8 if gated else None, sigma=0.6 if gated else 0.05)
+    over = dict(max_batch=w.batch + 3, num_layers=6, max_context=w.capacity + 5000, max_k=w.top_k + 100,
+                max_window=w.window + 9, max_sinks=w.sinks + 3, max_dilate_r=2, min_layer_group=1,
+                max_block_sets=4 if gated else 1)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), ctx_over=over, group_sets=not gated)
+    assert st["checked"] == 2 * 5 * w.batch * w.q_heads
