@@ -115,22 +115,22 @@ def job_throughput(world: int, batch: int, steps: int, max_ms: float) -> float:
 
 
 # ---------------------------------------------------------------------- the CPU oracle arm
-def oracle_throughput(w: W.Workload, steps: int, warmup: int, heads_per_step: int):
+def oracle_throughput(w: W.Workload, steps: int, warmup: int, heads_per_step: int, seqs: int = 1):
     """Time the CPU oracle, unmodified, on a bounded sample of the workload.
 
-    One sequence of the batch is generated on the CPU; each step runs `heads_per_step` of its
-    heads through the oracle's decode step (retrieval on the first step of a block), and the
+    `seqs` sequences of the batch are generated on the CPU; each step runs `heads_per_step` heads of
+    each through the oracle's decode step (retrieval on the first step of a block), and the
     step time is scaled to the full batch x heads.  Returns (tokens/s, ms per scaled step,
     threads, sample description).
     """
     from oracle import prhs_oracle as O
-    ws = w.scaled(batch=1, steps=warmup + steps)
+    ws = w.scaled(batch=seqs, steps=warmup + steps)
     k, v = W.make_kv(ws, "cpu")
     q = W.make_queries(ws, "cpu")[0]
     K, V, Q = k.float().numpy(), v.float().numpy(), q.float().numpy()
     orc = O.PrhsOracle(O.Schedule(top_k=w.top_k, window=w.window, sinks=w.sinks,
                                   refresh_interval=w.refresh, dilate_r=w.dilate_r), w.q_heads, w.kv_heads)
-    units = [(0, h) for h in range(min(heads_per_step, w.q_heads))]
+    units = [(b, h) for b in range(seqs) for h in range(min(heads_per_step, w.q_heads))]
     scale = (w.batch * w.q_heads) / len(units)
     total = 0.0
     for n in range(warmup + steps):
@@ -431,8 +431,9 @@ def run_cuda(args):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
+        # about 12 s of CPU work: every (sequence, head) unit of the batch, four blocks of steps
         cval, cms, threads, sample = oracle_throughput(W.C2_LLAMA2_7B, steps=4 * w.refresh, warmup=0,
-                                                       heads_per_step=Hq)
+                                                       heads_per_step=Hq, seqs=B)
         cpu = {"value": cval, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                "ms_per_step": cms}
 
