@@ -102,20 +102,35 @@ def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6, group_sets
             "unique_bytes": unique, "key_bytes": key_bytes}
 
 
-def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6):
+def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6, group_sets: bool = False):
     """Per-step device time (us) of a whole block of s decode steps (one retrieval, s - 1 sharing
     steps) and of s dense steps, each block replayed from a CUDA graph: what a decode loop pays
     once the per-launch host work is out of the way.  Blocks of independent cache copies are
     replayed in turn."""
     w = w.scaled(layers=copies, steps=s)
-    kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
+    table = None
+    if w.page_size:
+        table, pool = W.make_page_table(w)
+        kv = []
+        for _, k, v in W.make_layer_kv(w, dev):       # page one copy at a time to bound memory
+            kv.append((W.to_paged(w, k, table, pool), W.to_paged(w, v, table, pool)))
+            del k, v
+        table = table.to(dev)
+    else:
+        kv = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
     q = W.make_queries(w, dev)
     B, Hq = w.batch, w.q_heads
-    ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, w.top_k, w.window, w.sinks, max_dilate_r=w.dilate_r)
-    sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=s, dilate_r=w.dilate_r)
+    kps = W.top_k_per_seq(w)
+    max_k = max(w.top_k, int(w.k_frac * w.context))
+    ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
+                    page_size=w.page_size)
+    sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=s, dilate_r=w.dilate_r,
+                            top_k_per_seq=None if kps is None else kps.to(dev),
+                            flags=P.PRHS_GROUP_SETS if group_sets else 0)
     out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     lens = [W.seq_lens_at(w, n).to(dev) for n in range(s)]
-    views = [[P.make_view(kv[l][0], kv[l][1], lens[n], max_seq_len=w.capacity) for n in range(s)] for l in range(copies)]
+    views = [[P.make_view(kv[l][0], kv[l][1], lens[n], page_table=table, max_seq_len=w.capacity) for n in range(s)]
+             for l in range(copies)]
     side = torch.cuda.Stream()
     graphs = {"sparse": [], "dense": []}
     with torch.cuda.stream(side):
@@ -186,6 +201,23 @@ def table3(dev, graph=False):
                   f"{am[8]:.1f} | {am[16]:.1f} | {r['dense_us'] / am[16]:.2f}x | {pf} / {p8} / {p16} |")
 
 
+def configs_graph(dev, group_sets=False, only=None, batch=0):
+    print("| config | steps per retrieval (s x G_L) | dense us / step | sparse us / step | dense / sparse |")
+    print("|---|---|---|---|---|")
+    for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
+        if only and w.name != only:
+            continue
+        if batch:
+            w = w.scaled(batch=batch)
+        period = w.refresh * w.layer_group
+        # a follower layer's step costs what a sharing step costs: one block of `period` steps
+        r = time_blocks(w.scaled(layer_group=1), dev, period, copies=4 if w.context < 50000 else 2,
+                        group_sets=group_sets)
+        print(f"| {w.name} | {period} | {r['dense']:.1f} | {r['sparse']:.1f} | {r['dense'] / r['sparse']:.2f}x |",
+              flush=True)
+        torch.cuda.empty_cache()
+
+
 def configs(dev, group_sets=False, only=None, batch=0):
     print("| config | dense us | retrieval step us | sharing step us | amortised (config's s, G_L) us | "
           "mean set size | dense / amortised | sharing step GB/s logical / unique | retrieval step kernels us |")
@@ -209,7 +241,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", action="store_true", help="time the benchmark's C2..C5 shapes instead")
     ap.add_argument("--graph", action="store_true",
-                    help="Table-3 shapes: whole blocks of s steps replayed from CUDA graphs (per-step time)")
+                    help="whole blocks of steps (one retrieval and the sharing steps that follow) replayed from "
+                         "CUDA graphs: time per step")
     ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
     ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
     ap.add_argument("--group-sets", action="store_true",
@@ -220,7 +253,7 @@ def main():
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     if args.configs:
-        configs(dev, args.group_sets, args.only, args.batch)
+        (configs_graph if args.graph else configs)(dev, args.group_sets, args.only, args.batch)
     else:
         table3(dev, args.graph)
 
