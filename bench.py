@@ -11,9 +11,18 @@ gathered attention).  The workload is the LLaMA-2-7B-shaped single layer at 32K 
 four independent copies of that layer's cache are visited round-robin so that no step finds
 its rows in L2.
 
+The timed window always holds whole blocks of the schedule: --warmup and --steps are rounded up
+to multiples of (cache copies x refresh interval), so that one step in `refresh` retrieves
+whatever the arguments (the line reports the rounded figures as `steps` / `warmup` and the
+arguments as `steps_requested` / `warmup_requested`).  The window is timed --repeats times (each
+repeat is the same K steps, starting from a block boundary of every cache copy, so it needs no
+state from the one before); `value` comes from the median repeat.
+
 Prints ONE JSON line.  `value` is attention-only decode throughput in tokens/s (batch tokens
 per step / device time per step) with every input resident in HBM; `e2e` is the same metric
-through the host-buffer entry point with the per-step host<->device copies timed.
+through the host-buffer entry point with the per-step host<->device copies timed;
+`other_configs` holds the same measurement, per layer-step, for the other full-size
+configurations (Mistral-shaped layer group, 128K context, paged serving mix).
 """
 from __future__ import annotations
 
@@ -114,6 +123,14 @@ def job_throughput(world: int, batch: int, steps: int, max_ms: float) -> float:
     return world * batch * steps / (max_ms * 1e-3)
 
 
+def aligned_window(warmup: int, steps: int, period: int):
+    """(warm-up, steps) rounded up to whole blocks: multiples of `period` = cache copies x refresh
+    interval, at least one block each.  A window like that starts on a block boundary of every
+    cache copy and holds exactly one retrieval per `refresh` steps, whatever was asked for."""
+    up = lambda x: max(1, -(-x // period)) * period
+    return up(warmup), up(steps)
+
+
 # ---------------------------------------------------------------------- the CPU oracle arm
 def oracle_throughput(w: W.Workload, steps: int, warmup: int, heads_per_step: int, seqs: int = 1):
     """Time the CPU oracle, unmodified, on a bounded sample of the workload.
@@ -164,9 +181,12 @@ def run_reference(args):
     if rank != 0:
         return 0
     w = W.C2_LLAMA2_7B
-    val, ms, threads, sample = oracle_throughput(w, args.steps, args.warmup, heads_per_step=8)
+    # whole blocks of the schedule here too (the oracle decodes one cache: a block is `refresh` steps)
+    warmup, steps = aligned_window(args.warmup, args.steps, w.refresh)
+    val, ms, threads, sample = oracle_throughput(w, steps, warmup, heads_per_step=8)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "steps": steps, "warmup": warmup, "steps_requested": args.steps, "warmup_requested": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": workload_config(w),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
@@ -195,14 +215,20 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    Wn, Kn = args.warmup, args.steps
     # Step i of the run is decode step i // L of cache i % L: L independent copies of the
     # single-layer workload are visited round-robin, so every step finds its K/V rows cold in
     # L2 (each copy is 4.3 GB) without a flush kernel between steps, and launches stay
     # back to back as in a real decode loop.  L = 1 falls back to flushing L2 between steps.
     L = max(1, args.rotate)
-    n_dec = (Wn + Kn + L - 1) // L
-    w = W.C2_LLAMA2_7B.scaled(steps=n_dec, layers=L, seed=W.C2_LLAMA2_7B.seed + 97 * rank)
+    base = W.C2_LLAMA2_7B
+    # whole blocks only: a window of any multiple of L x s steps that starts on a multiple of
+    # L x s holds exactly one retrieval per s steps, and every sharing step in it finds the
+    # set that its own block's retrieval (also in the window) stored
+    period = L * base.refresh
+    Wn, Kn = aligned_window(args.warmup, args.steps, period)
+    R = max(1, args.repeats)
+    n_dec = (Wn + Kn) // L
+    w = base.scaled(steps=n_dec, layers=L, seed=base.seed + 97 * rank)
     if args.batch:
         w = w.scaled(batch=args.batch)      # smaller case for profiler captures only
     kv_layers = [(k, v) for _, k, v in W.make_layer_kv(w, dev)]
@@ -247,15 +273,17 @@ def run_cuda(args):
     def is_refresh(i):
         return (i // L) % w.refresh == 0
 
+    assert sum(is_refresh(i) for i in range(Wn, Wn + Kn)) * w.refresh == Kn     # one retrieval per s steps
+
     # ---- warm-up, then the timed region
     timed_steps(0, Wn, step_device)
     sampler = ClockSampler(local, uuid=str(torch.cuda.get_device_properties(dev).uuid), period=0.002)
     sampler.start()
-    launches0 = ctx.launch_count
     # The K timed steps are captured once into a CUDA graph (prhs_decode_step only enqueues work) and
-    # the timed region is one replay of it: the same kernels on the same inputs without the
-    # per-launch host work.  --no-graph, or a failed capture, times direct launches instead.
+    # a repeat of the timed region is one replay of it: the same kernels on the same inputs without
+    # the per-launch host work.  --no-graph, or a failed capture, times direct launches instead.
     graph = None
+    graph_launches = 0
     if not args.no_graph and not args.path_only and L > 1:      # (the capture counts the K steps' launches)
         try:
             side = torch.cuda.Stream()
@@ -274,48 +302,41 @@ def run_cuda(args):
             graph_launches = ctx.launch_count - cap0          # kernel nodes of the graph = launches per replay
             graph.replay()            # untimed: the first replay also uploads the graph
             torch.cuda.synchronize()
-            for i in range(Wn):       # back to the state the timed steps start from
-                step_device(i)
         except Exception as e:                                                  # pragma: no cover
             print(f"bench: CUDA graph capture failed ({e}); timing direct launches", file=sys.stderr)
             graph = None
             torch.cuda.synchronize()
-            for i in range(Wn):
-                step_device(i)
     launches0 = ctx.launch_count
     barrier()
-    if graph is not None:
-        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a_ev.record(stream)
-        graph.replay()
-        b_ev.record(stream)
-        torch.cuda.synchronize()
-        ms = [a_ev.elapsed_time(b_ev) / Kn] * Kn
-    else:
-        ms = timed_steps(Wn, Kn, step_device)
+    rep_ms = []                       # device time of each repeat of the K steps
+    for _ in range(R):
+        if graph is not None:
+            a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_ev.record(stream)
+            graph.replay()
+            b_ev.record(stream)
+            torch.cuda.synchronize()
+            rep_ms.append(a_ev.elapsed_time(b_ev))
+        else:
+            rep_ms.append(sum(timed_steps(Wn, Kn, step_device)))
     barrier()
-    launches = graph_launches if graph is not None else ctx.launch_count - launches0
+    launches = R * graph_launches if graph is not None else ctx.launch_count - launches0
     dev_flags = ctx.check()
     assert dev_flags & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
-    total_ms = sum(ms)
+    total_ms = statistics.median(rep_ms)
     total_ms_max = reduce_max_ms(total_ms, dist, dev)
     value = job_throughput(world, B, Kn, total_ms_max)
 
-    def rewind():
-        """Replay the warm-up steps so that the shared-set state is the one step Wn expects."""
-        for i in range(Wn):
-            step_device(i)
-
+    # Nothing to restore between the legs below: each starts at step Wn, a block boundary of every
+    # cache copy, where the first thing each copy does is retrieve.
     # per-kernel durations: the same K steps once more, back to back, with an event pair recorded
     # inside the library around every launch (kept out of the timed region above, where the 24
     # extra event pairs cost about 9 us per step)
-    rewind()
     ctx.profile_begin(8 * Kn + 16)
     timed_steps(Wn, Kn, step_device)
     prof = ctx.profile_end()
 
     # per-step times of the same steps (event pair per step), to tell retrieval from sharing steps
-    rewind()
     ms_each = timed_steps(Wn, Kn, step_device, per_step=True)
 
     refresh_ms = [m for i, m in enumerate(ms_each) if is_refresh(Wn + i)]
@@ -323,7 +344,6 @@ def run_cuda(args):
 
     # ---- algorithmic bytes: K once on retrieval steps, gathered K/V rows on every step
     counts = []
-    rewind()
     for i in range(Wn, Wn + Kn):                          # untimed replay to read the set sizes
         step_device(i)
         _, cnt = ctx.get_index_set(B)
@@ -335,7 +355,6 @@ def run_cuda(args):
         sched_d = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
                                   flags=P.PRHS_WANT_DELTA)
         dlt = torch.empty(B, Hq, dtype=torch.float32, device=dev)
-        rewind()
         for i in range(Wn, Wn + Kn):
             ctx.decode_step(i % L, i // L, sched_d, q_all[i % L, i // L], views[i % L][i // L], B, out, dlt)
             deltas.append(dlt.clone())
@@ -377,7 +396,7 @@ def run_cuda(args):
         return 0
 
     # ---- in-library dense flash-decode baseline, same protocol
-    nd = min(4, Kn)
+    nd = min(8, Kn)
     dense_ms = timed_steps(Wn, nd, lambda i: ctx.dense_decode_attn(q_all[i % L, i // L], views[i % L][i // L],
                                                                  B, out))
     dense_us = 1e3 * statistics.median(dense_ms[1:] or dense_ms)
@@ -401,9 +420,8 @@ def run_cuda(args):
         hq, hk, hv, ht = host[i - Wn]
         ctx.decode_step_host(i % L, i // L, sched, hq, hk, hv, ht, views_h[i % L], B, host_out)
 
-    rewind()
     barrier()
-    e2e_ms = timed_steps(Wn, Kn, step_host)
+    e2e_reps = [sum(timed_steps(Wn, Kn, step_host)) for _ in range(3)]
     barrier()
     # the same through the entry point that does not synchronise after every step (a caller with
     # other layers to enqueue): inputs and outputs still cross the host link every step, the host
@@ -412,13 +430,12 @@ def run_cuda(args):
         hq, hk, hv, ht = host[i - Wn]
         ctx.decode_step_host(i % L, i // L, sched, hq, hk, hv, ht, views_h[i % L], B, host_out, sync=False)
 
-    rewind()
     barrier()
-    e2e_async_ms = timed_steps(Wn, Kn, step_host_async)
+    e2e_async_reps = [sum(timed_steps(Wn, Kn, step_host_async)) for _ in range(3)]
     barrier()
-    e2e_async_max_ms = reduce_max_ms(sum(e2e_async_ms), dist, dev)
+    e2e_async_max_ms = reduce_max_ms(statistics.median(e2e_async_reps), dist, dev)
     clocks = sampler.stop()
-    e2e_max_ms = reduce_max_ms(sum(e2e_ms), dist, dev)
+    e2e_max_ms = reduce_max_ms(statistics.median(e2e_reps), dist, dev)
     e2e_value = job_throughput(world, B, Kn, e2e_max_ms)
     h2d = B * Hq * 256 + 2 * B * Hkv * 256 + B * 4
     d2h = B * Hq * 256
@@ -428,6 +445,22 @@ def run_cuda(args):
         if dist is not None:
             dist.destroy_process_group()
         return 0
+
+    # ---- the other full-size configurations, each timed as its own schedule runs it (one layer
+    # group, or independent copies of a single layer), per layer-step
+    other = None
+    if world == 1 and not args.no_other_configs and not args.batch:
+        from paper_2602_08329_b200 import operator_latency as OL
+        ctx.close()
+        del kv_layers, views, views_h, q_all, graph
+        torch.cuda.empty_cache()
+        other = {}
+        for ow in (W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
+            try:
+                other[ow.name] = OL.config_summary(ow, dev, hbm_peak_gbs=hbm_peak)
+            except Exception as e:                                              # pragma: no cover
+                other[ow.name] = {"error": f"{type(e).__name__}: {e}"}
+                torch.cuda.empty_cache()
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -439,13 +472,19 @@ def run_cuda(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": Kn, "warmup": Wn,
-        "ms_per_step": total_ms_max / Kn, "higher_is_better": True, "scaling": "weak",
+        "steps_requested": args.steps, "warmup_requested": args.warmup,
+        "window": f"whole blocks: steps and warm-up rounded up to multiples of {period} "
+                  f"({L} cache copies x refresh interval {w.refresh})",
+        "repeats": R, "ms_per_step": total_ms_max / Kn,
+        "ms_per_step_min_max": [min(rep_ms) / Kn, max(rep_ms) / Kn],
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
         "config": workload_config(w, {
             "parallelism": f"replicas x{world} (no collective)",
             "cache_copies": L,
-            "launch": ("the K timed steps are one replay of a CUDA graph captured from the same prhs_decode_step calls"
-                       if graph is not None else "direct launches"),
+            "launch": ("each repeat of the K timed steps is one replay of a CUDA graph captured from the same "
+                       "prhs_decode_step calls; value = median repeat"
+                       if graph is not None else "direct launches; value = median repeat"),
             "kernel_timing": "event pairs inside the library around every launch, on a back-to-back replay of the "
                              "same K steps (the timed region itself carries no instrumentation)",
             "l2": (f"no flush: {L} independent copies of the layer's cache (4.3 GB each) visited round-robin, "
@@ -474,7 +513,8 @@ def run_cuda(args):
                           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                           "ms_per_step": e2e_async_max_ms / Kn,
                           "note": "prhs_decode_step_host_async: same copies every step, one wait after the K steps"},
-        "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+        "gpu_launches": launches, "gpu_launches_per_repeat": launches // R, "clocks": clocks,
+        "cpu_baseline": cpu, "other_configs": other,
     }
     print(json.dumps(line))
     ctx.close()
@@ -496,6 +536,10 @@ def main():
     ap.add_argument("--rotate", type=int, default=4,
                     help="independent copies of the layer cache visited round-robin (1 = flush L2 instead)")
     ap.add_argument("--path-only", action="store_true", help="skip the dense, e2e and CPU legs")
+    ap.add_argument("--repeats", type=int, default=10,
+                    help="how many times the K timed steps are run; the line reports the median repeat")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the per-layer-step summaries of the other full-size configurations")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         print("warning: fewer than 3 warm-up steps", file=sys.stderr)

@@ -70,7 +70,15 @@ typedef struct {
   int32_t min_layer_group; /* smallest layer_group that will be used (sizes the state); >= 1 */
   int32_t max_block_sets;  /* sets kept per (b, h) and block, 1..64; 1 unless the cosine gate is
                               used, which needs max_block_sets >= refresh_interval              */
+  uint32_t flags;          /* PRHS_CFG_* below; 0 = defaults                                    */
 } prhs_config;
+
+/* Configuration flags */
+#define PRHS_CFG_NO_TMA 1u /* retrieval scoring never uses the tensor-memory-accelerator kernels: the
+                              key stream is staged by the cp.async ring kernel instead, which is what
+                              the library falls back to on its own when the driver does not export
+                              cuTensorMapEncodeTiled or the cache spans 2^31 rows or more.  Same
+                              results; for testing that path and for comparing the two. */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at
@@ -203,7 +211,10 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
  *     each call first clears the tickets it will use (a memset node on `stream`).  Two calls
  *     whose kernels may overlap on the GPU (different streams, no ordering) race on it:
  *     serialise them.
- *   - An index outside [0, t_b) is skipped; the anomaly word is not reported by this call.
+ *   - The first call on a device may come from several host threads at once (the set-up is
+ *     guarded); the GPU-side sharing rule above is what callers have to respect.
+ *   - An index outside [0, t_b) or a page id outside the pool is skipped and recorded in the
+ *     array's anomaly word, which prhs_noalloc_check() reports.
  * Arguments as prhs_sparse_decode_attn, with the head counts passed explicitly.
  * Errors go to prhs_last_error(NULL). */
 #define PRHS_NOALLOC_MAX_UNITS 1024
@@ -212,6 +223,12 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
                                             const int32_t* count, int32_t idx_stride, int32_t batch,
                                             int32_t num_q_heads, int32_t num_kv_heads, void* out,
                                             float* out_lse, void* stream);
+
+/* Companion of prhs_sparse_decode_attn_noalloc (the paper has no counterpart): synchronises
+ * `stream`, reads the anomaly word the allocation-free calls on the current device share, and
+ * clears it.  *out_flags (may be NULL) receives the PRHS_FLAG_* bits; the return value is
+ * PRHS_ERR_DEVICE_FLAG if any was set, else PRHS_OK.  Allocates nothing. */
+prhs_status prhs_noalloc_check(void* stream, uint32_t* out_flags);
 
 /* Dense flash-decoding baseline (Eq. 2): attention over all i < t_b. Same outputs. */
 prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv,

@@ -22,6 +22,7 @@ PRHS_DILATE_ANCHOR = 1
 PRHS_WANT_DELTA = 2
 PRHS_GROUP_SETS = 4
 PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TIMEOUT = 1, 2, 4, 8
+PRHS_CFG_NO_TMA = 1
 
 # every symbol include/prhs.h declares
 EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_set",
@@ -29,7 +30,8 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_decode_step_host", "prhs_decode_step_host_async", "prhs_delta", "prhs_index_capacity", "prhs_get_index_set",
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
            "prhs_launch_count", "prhs_selftest_wait", "prhs_state_bytes", "prhs_state_export", "prhs_state_import", "prhs_validate_index_lists", "prhs_last_error", "prhs_version", "prhs_profile_begin",
-           "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate"]
+           "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate",
+           "prhs_noalloc_check"]
 NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
 
@@ -44,7 +46,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_layers", "max_batch", "num_q_heads", "num_kv_heads", "head_dim", "max_context",
         "page_size", "max_k", "max_window", "max_sinks", "max_dilate_r", "max_dilate_m",
-        "min_layer_group", "max_block_sets")]
+        "min_layer_group", "max_block_sets")] + [("flags", C.c_uint32)]
 
 
 class KvView(C.Structure):
@@ -83,6 +85,7 @@ def load() -> C.CDLL:
         "prhs_sparse_decode_attn": (st, [vp, vp, C.POINTER(KvView), vp, vp, i32, i32, vp, vp, vp]),
         "prhs_dense_decode_attn": (st, [vp, vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_sparse_decode_attn_noalloc": (st, [vp, C.POINTER(KvView), vp, vp, i32, i32, i32, i32, vp, vp, vp]),
+        "prhs_noalloc_check": (st, [vp, C.POINTER(C.c_uint32)]),
         "prhs_decode_step": (st, [vp, i32, i32, C.POINTER(Schedule), vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_decode_step_host": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32, vp, vp]),
         "prhs_decode_step_host_async": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32,
@@ -155,11 +158,11 @@ class Context:
 
     def __init__(self, num_layers, max_batch, num_q_heads, num_kv_heads, max_context, max_k,
                  max_window, max_sinks, max_dilate_r=1, max_dilate_m=-1, page_size=0,
-                 min_layer_group=1, head_dim=128, max_block_sets=1):
+                 min_layer_group=1, head_dim=128, max_block_sets=1, flags=0):
         self.lib = load()
         self.cfg = Config(num_layers, max_batch, num_q_heads, num_kv_heads, head_dim, max_context,
                           page_size, max_k, max_window, max_sinks, max_dilate_r, max_dilate_m,
-                          min_layer_group, max_block_sets)
+                          min_layer_group, max_block_sets, flags)
         h = C.c_void_p()
         rc = self.lib.prhs_create(C.byref(self.cfg), C.byref(h))
         if rc != PRHS_OK:
@@ -312,6 +315,20 @@ def sparse_decode_attn_noalloc(q, view, idx, count, batch, num_q_heads, num_kv_h
                                              _stream(stream))
     if rc != PRHS_OK:
         raise PrhsError(rc, lib.prhs_last_error(None).decode())
+
+
+def noalloc_check(stream=None) -> int:
+    """Report and clear the anomaly word of the allocation-free calls on the current device.
+
+    Returns 0 when clean; raises PrhsError (PRHS_ERR_DEVICE_FLAG) when a call skipped an index
+    outside [0, t_b) or a page id outside the pool.  Synchronises the stream.
+    """
+    lib = load()
+    flags = C.c_uint32(0)
+    rc = lib.prhs_noalloc_check(_stream(stream), C.byref(flags))
+    if rc != PRHS_OK:
+        raise PrhsError(rc, lib.prhs_last_error(None).decode())
+    return flags.value
 
 
 def version() -> str:

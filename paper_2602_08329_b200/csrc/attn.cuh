@@ -952,13 +952,6 @@ gate_kernel(const __nv_bfloat16* __restrict__ q, int units, int pos, float tau, 
   }
 }
 
-// delta = 1 - exp(lse_C - lse_full)  (Sec. 2.3), one thread per (b, h).
-__global__ void delta_kernel(const float* __restrict__ lse_c, const float* __restrict__ lse_full,
-                             float* __restrict__ out, int n) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = (lse_c[i] == -INFINITY) ? 1.f : -expm1f(lse_c[i] - lse_full[i]);
-}
-
 // Reduce the scoring pass' per-chunk (m, l) partials to lse_full (used when no selection runs).
 __global__ void lse_reduce_kernel(const float2* __restrict__ part_ml, int nchunks, int chunk_rows,
                                   const int* __restrict__ seq_lens, int num_q_heads,

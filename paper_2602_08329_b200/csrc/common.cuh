@@ -29,21 +29,6 @@ struct KvDev {
   int num_pages;
 };
 
-// Element offset of row `i` of (b, kvh); -1 (and a flag) for a page id out of range.
-__device__ __forceinline__ long long row_offset(const KvDev& kv, int b, int kvh, int i,
-                                                uint32_t* flags) {
-  if (kv.page_table != nullptr) {
-    int page = __ldg(kv.page_table + (long long)b * kv.page_table_stride + (i >> kPageShift));
-    if ((unsigned)page >= (unsigned)kv.num_pages) {
-      atomicOr(flags, kFlagBadPage);
-      return -1;
-    }
-    return (long long)page * kv.stride_outer + (long long)kvh * kv.stride_head +
-           (long long)(i & ((1 << kPageShift) - 1)) * kHeadDim;
-  }
-  return (long long)b * kv.stride_outer + (long long)kvh * kv.stride_head + (long long)i * kHeadDim;
-}
-
 // Which stored middle set a (b, h) unit attends over.  Sets live in slots: [unit][slot][stride]
 // for S* (ascending) and for the dilated S^; a unit uses S* only on the step that retrieved
 // it (and not even then with PRHS_DILATE_ANCHOR), else S^ (Def. 3.2).
@@ -87,37 +72,6 @@ __device__ __forceinline__ int psaw_start(double c, int t) {
 // bf16 pair (packed in 32 bits) -> two floats; exact.
 __device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
-
-// 16-byte read-only load that does not allocate in L1 (streamed once).
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
-
-// Dot product of 8 bf16 (one uint4) with 8 floats.
-__device__ __forceinline__ float dot8(const uint4& kx, const float* q) {
-  float s = bf_lo(kx.x) * q[0];
-  s = fmaf(bf_hi(kx.x), q[1], s);
-  s = fmaf(bf_lo(kx.y), q[2], s);
-  s = fmaf(bf_hi(kx.y), q[3], s);
-  s = fmaf(bf_lo(kx.z), q[4], s);
-  s = fmaf(bf_hi(kx.z), q[5], s);
-  s = fmaf(bf_lo(kx.w), q[6], s);
-  s = fmaf(bf_hi(kx.w), q[7], s);
-  return s;
-}
-
-// Sum over the 16 lanes of a half-warp (all 16 lanes receive the total).
-__device__ __forceinline__ float half_warp_sum(float s) {
-  s += __shfl_xor_sync(0xffffffffu, s, 8);
-  s += __shfl_xor_sync(0xffffffffu, s, 4);
-  s += __shfl_xor_sync(0xffffffffu, s, 2);
-  s += __shfl_xor_sync(0xffffffffu, s, 1);
-  return s;
-}
 
 // Order-preserving map fp32 -> uint32: larger float <=> larger key (-0 < +0, NaNs at the ends).
 __device__ __forceinline__ uint32_t float_to_key(float f) {

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -155,6 +156,9 @@ prhs_status check_sched(prhs_ctx* ctx, const prhs_schedule* s) {
   if (s->top_k > ctx->cfg.max_k || s->window > ctx->cfg.max_window || s->sinks > ctx->cfg.max_sinks ||
       s->dilate_r > ctx->cfg.max_dilate_r || (s->dilate_m >= 0 && s->dilate_m > ctx->max_m))
     return fail(ctx, PRHS_ERR_CAPACITY, "schedule: budget exceeds the configured maximum");
+  // m = floor(k / 3) by default (Sec. 5.1): the dilated set must fit what the context was sized for
+  if (s->dilate_m < 0 && (s->top_k_per_seq ? ctx->cfg.max_k : s->top_k) / 3 > ctx->max_m)
+    return fail(ctx, PRHS_ERR_CAPACITY, "schedule: floor(k / 3) dilated winners exceed max_dilate_m");
   if ((s->flags & PRHS_GROUP_SETS) && s->sim_threshold > -1.f)
     return fail(ctx, PRHS_ERR_UNSUPPORTED, "schedule: the cosine gate is per head, group-shared sets are per KV head");
   return PRHS_OK;
@@ -228,7 +232,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + kSTStageRows - 1) & ~(kSTStageRows - 1);
   sp.flags = c->flags;
   bool tma_done = false;
-  if (c->encode_tiled) {
+  if (c->encode_tiled && !(c->cfg.flags & PRHS_CFG_NO_TMA)) {
     // K as a 2-D tensor [rows][128] bf16.  Contiguous cache: rows past the last sequence's max
     // length are out of bounds for the copy engine (zero fill), rows in between belong to the
     // cache; a copy brings 64 rows.  Paged cache: the rows of the page pool; a copy brings the
@@ -607,6 +611,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
   if (cfg->max_context > kMaxContext) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context above 2^20");
   if (cfg->max_k > 65536) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_k above 65536");
+  if (cfg->flags & ~PRHS_CFG_NO_TMA) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
 
   prhs_ctx* c = new (std::nothrow) prhs_ctx();
   if (!c) return fail(nullptr, PRHS_ERR_OOM, "host allocation failed");
@@ -796,13 +801,46 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
                      nullptr, nullptr, as_stream(stream));
 }
 
+namespace {
+// Per-device set-up state of the allocation-free entry points (no allocation): the scratch
+// array's device address, SM count, resident CTAs per SM.  Guarded by a mutex so that two host
+// threads may make the first call on a device at the same time.
+struct NoAllocDev { unsigned char* scratch = nullptr; int sm_count = 0; int ctas_per_sm = 0; };
+NoAllocDev g_noalloc_dev[64];
+std::mutex g_noalloc_mutex;
+
+// Resolves the state of the current device, doing the one-time set-up on the first call there.
+prhs_status noalloc_device(NoAllocDev** out) {
+  int dev = -1;
+  PRHS_CUDA(nullptr, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "noalloc: device ordinal above 63");
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  NoAllocDev& ds = g_noalloc_dev[dev];
+  if (!ds.scratch) {
+    // first call on this device, with this device current: in host code the array's name is a
+    // stand-in, its device address has to be asked for
+    unsigned char* ptr = nullptr;
+    PRHS_CUDA(nullptr, cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch));
+    PRHS_CUDA(nullptr, cudaFuncSetAttribute(gather_attn_mma_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes));
+    PRHS_CUDA(nullptr, cudaDeviceGetAttribute(&ds.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    PRHS_CUDA(nullptr, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ds.ctas_per_sm, gather_attn_mma_kernel,
+                                                                     kTThreads, kTSmemBytes));
+    if (ds.ctas_per_sm < 1) ds.ctas_per_sm = 1;
+    ds.scratch = ptr;
+  }
+  *out = &ds;
+  return PRHS_OK;
+}
+inline unsigned int* noalloc_tickets(const NoAllocDev& ds) {
+  return reinterpret_cast<unsigned int*>(ds.scratch + kNoAllocPartialFloats * sizeof(float));
+}
+}  // namespace
+
 prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* kv, const int32_t* idx,
                                             const int32_t* count, int32_t idx_stride, int32_t batch,
                                             int32_t num_q_heads, int32_t num_kv_heads, void* out,
                                             float* out_lse, void* stream) {
-  // per-device set-up state (no allocation): scratch address, SM count, resident CTAs per SM
-  struct DevState { unsigned char* scratch = nullptr; int sm_count = 0; int ctas_per_sm = 0; };
-  static DevState dev_state[64];
   if (!q || !kv || !kv->k || !kv->v || !kv->seq_lens || !idx || !count || !out)
     return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: NULL pointer");
   if (batch < 1 || num_q_heads < 1 || num_kv_heads < 1 || num_q_heads % num_kv_heads || idx_stride < 1)
@@ -815,22 +853,10 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
     return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: strides must be positive multiples of 128 elements, bases 16-byte aligned");
   if (kv->page_table && (kv->page_table_stride < 1 || kv->num_pages < 1))
     return fail(nullptr, PRHS_ERR_INVALID_ARG, "noalloc: bad page table stride or pool size");
-  int dev = -1;
-  PRHS_CUDA(nullptr, cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "noalloc: device ordinal above 63");
-  DevState& ds = dev_state[dev];
-  if (!ds.scratch) {
-    // first call on this device, with this device current
-    unsigned char* ptr = nullptr;
-    PRHS_CUDA(nullptr, cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch));
-    PRHS_CUDA(nullptr, cudaFuncSetAttribute(gather_attn_mma_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes));
-    PRHS_CUDA(nullptr, cudaDeviceGetAttribute(&ds.sm_count, cudaDevAttrMultiProcessorCount, dev));
-    PRHS_CUDA(nullptr, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ds.ctas_per_sm, gather_attn_mma_kernel,
-                                                                     kTThreads, kTSmemBytes));
-    if (ds.ctas_per_sm < 1) ds.ctas_per_sm = 1;
-    ds.scratch = ptr;
-  }
+  NoAllocDev* dsp = nullptr;
+  prhs_status rc = noalloc_device(&dsp);
+  if (rc != PRHS_OK) return rc;
+  const NoAllocDev& ds = *dsp;
   cudaStream_t st = as_stream(stream);
   const int units = batch * num_q_heads;
   // same split rule as the context-based call, capped by the static capacity
@@ -845,7 +871,7 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
     if (cost < best_cost * 0.999) { best_cost = cost; splits = s; }
   }
   float* partials = reinterpret_cast<float*>(ds.scratch);
-  unsigned int* tickets = reinterpret_cast<unsigned int*>(ds.scratch + kNoAllocPartialFloats * sizeof(float));
+  unsigned int* tickets = noalloc_tickets(ds);
   uint32_t* flag_word = tickets + PRHS_NOALLOC_MAX_UNITS;
   // the array keeps the last call's contents: tickets must start at zero
   PRHS_CUDA(nullptr, cudaMemsetAsync(tickets, 0, (size_t)units * sizeof(unsigned int), st));
@@ -875,6 +901,26 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
   p.flags = flag_word;
   gather_attn_mma_kernel<<<dim3(splits, num_q_heads, batch), kTThreads, kTSmemBytes, st>>>(p);
   PRHS_CUDA(nullptr, cudaGetLastError());
+  return PRHS_OK;
+}
+
+prhs_status prhs_noalloc_check(void* stream, uint32_t* out_flags) {
+  NoAllocDev* dsp = nullptr;
+  prhs_status rc = noalloc_device(&dsp);
+  if (rc != PRHS_OK) return rc;
+  cudaStream_t st = as_stream(stream);
+  uint32_t* flag_word = noalloc_tickets(*dsp) + PRHS_NOALLOC_MAX_UNITS;
+  uint32_t f = 0;
+  PRHS_CUDA(nullptr, cudaMemcpyAsync(&f, flag_word, sizeof(f), cudaMemcpyDeviceToHost, st));
+  PRHS_CUDA(nullptr, cudaStreamSynchronize(st));
+  if (out_flags) *out_flags = f;
+  if (f) {
+    PRHS_CUDA(nullptr, cudaMemsetAsync(flag_word, 0, sizeof(uint32_t), st));
+    PRHS_CUDA(nullptr, cudaStreamSynchronize(st));
+    char buf[96];
+    snprintf(buf, sizeof buf, "noalloc: device flag word 0x%x", f);
+    return fail(nullptr, PRHS_ERR_DEVICE_FLAG, buf);
+  }
   return PRHS_OK;
 }
 
@@ -979,10 +1025,25 @@ prhs_status decode_step_host_impl(prhs_ctx* ctx, int32_t layer, int32_t step, co
   if (!host_q || !host_new_k || !host_new_v || !host_seq_lens || !host_out || !kv)
     return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
   if (kv->page_table) return fail(ctx, PRHS_ERR_UNSUPPORTED, "host entry point needs a contiguous cache");
-  if (batch < 1 || batch > ctx->cfg.max_batch) return fail(ctx, PRHS_ERR_CAPACITY, "batch out of range");
-  for (int b = 0; b < batch; ++b)
-    if (host_seq_lens[b] < 1 || host_seq_lens[b] > ctx->cfg.max_context)
-      return fail(ctx, PRHS_ERR_INVALID_ARG, "seq_lens entry out of range");
+  // everything prhs_decode_step would reject is rejected here, before the cache is written
+  prhs_status vrc = check_sched(ctx, sched);
+  if (vrc != PRHS_OK) return vrc;
+  vrc = check_layer(ctx, layer, step, sched);
+  if (vrc != PRHS_OK) return vrc;
+  {
+    KvDev unused;
+    int cap = 0;
+    vrc = check_view(ctx, kv, batch, &unused, &cap);
+    if (vrc != PRHS_OK) return vrc;
+    // the new row lands at position t_b - 1 of the (b, kvh) slice: it must lie inside the capacity
+    // the view declares and inside the slice itself (a slice ends where the next head or sequence begins)
+    const long long slice_rows = std::min(kv->stride_head, kv->stride_outer) / kHeadDim;
+    for (int b = 0; b < batch; ++b) {
+      if (host_seq_lens[b] < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "seq_lens entry below 1");
+      if (host_seq_lens[b] > cap || host_seq_lens[b] > slice_rows)
+        return fail(ctx, PRHS_ERR_CAPACITY, "seq_lens entry exceeds the cache capacity (max_seq_len, strides)");
+    }
+  }
   cudaStream_t st = as_stream(stream);
   const size_t qb = (size_t)batch * ctx->cfg.num_q_heads * kRowBytes;
   const size_t kb = (size_t)batch * ctx->cfg.num_kv_heads * kRowBytes;

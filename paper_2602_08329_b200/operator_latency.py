@@ -4,6 +4,7 @@
     python -m paper_2602_08329_b200.operator_latency --graph    # the same, blocks of s steps replayed from CUDA graphs
     python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C5 shapes
     python -m paper_2602_08329_b200.operator_latency --configs --group-sets   # one set per KV head (variant)
+    python -m paper_2602_08329_b200.operator_latency --configs --summary  # JSON: time, bytes, roofline per layer-step
 
 The paper (Sec. 5.4, Table 3) times one attention layer of LLaMA-2-7B-Chat (32 MHA heads,
 head_dim 128) in decode at batch 8 / 16 and 1k-4k cached tokens, token sparsity 1/8, block
@@ -29,6 +30,14 @@ PAPER_TABLE3_MS = {  # (batch, seqlen): (Flash, CPE-8, CPE-16) in ms on an A100 
     (8, 1024): (0.230, 0.092, 0.078), (8, 2048): (0.830, 0.144, 0.095), (8, 4096): (1.630, 0.506, 0.469),
     (16, 1024): (0.440, 0.089, 0.075), (16, 2048): (1.630, 0.196, 0.165), (16, 4096): (3.230, 0.904, 0.821),
 }
+
+
+def table3_workload(batch: int, n: int, s: int = 8) -> W.Workload:
+    """The Table-3 shape (batch, n cached tokens) with the budgets of Sec. 5.3.2 scaled to the
+    length: C_sink 16, C_local 64, k = n/8 - 80 (432 at 4k); one MHA layer of 32 heads."""
+    return W.Workload(f"table3_b{batch}_{n}", layers=1, batch=batch, q_heads=32, kv_heads=32, context=n,
+                      steps=4, top_k=n // 8 - 80, window=64, sinks=16, refresh=s, heavy_hitters=16,
+                      decay_span=min(512, n // 8), seed=100 + batch + n)
 
 
 def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6, group_sets: bool = False):
@@ -168,6 +177,172 @@ def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6, grou
     return res
 
 
+def _make_caches(w: W.Workload, dev):
+    """(kv list per layer, page table on the device or None): the workload's caches, paged if it asks."""
+    if w.page_size:
+        table, pool = W.make_page_table(w)
+        kv = []
+        for _, k, v in W.make_layer_kv(w, dev):       # page one layer at a time to bound memory
+            kv.append((W.to_paged(w, k, table, pool), W.to_paged(w, v, table, pool)))
+            del k, v
+        return kv, table.to(dev)
+    return [(k, v) for _, k, v in W.make_layer_kv(w, dev)], None
+
+
+def _set_bytes(idx, cnt, w: W.Workload):
+    """(logical, unique) bytes a step must gather for the lists (idx, cnt): every listed row once per
+    query head, and once per KV head for the union over the heads of a group; 512 B per row (K + V)."""
+    B, Hq, cap = idx.shape
+    G = Hq // w.kv_heads
+    valid = torch.arange(cap)[None, None, :] < cnt[:, :, None]
+    mark = torch.zeros(B * w.kv_heads, w.capacity + 1, dtype=torch.bool)
+    unit = (torch.arange(B)[:, None] * w.kv_heads + torch.arange(Hq)[None, :] // G)[:, :, None].expand_as(idx)
+    mark[unit[valid].long(), idx[valid].long()] = True
+    return int(cnt.sum()) * 512, int(mark.sum()) * 512
+
+
+def config_summary(w: W.Workload, dev, reps: int = 7, copies: int = 4, group_sets: bool = False,
+                   hbm_peak_gbs: float | None = None) -> dict:
+    """One configuration of the benchmark, timed as its schedule runs it.
+
+    A block is one retrieval period: s decode steps of every layer of ONE layer group (the
+    configuration's G_L layers, each with its own cache; the first layer retrieves on the
+    block's first step, every other layer-step shares), or, for a single-layer configuration,
+    s decode steps of `copies` independent copies of the layer (each retrieves once).  Either
+    way consecutive layer-steps touch different caches, so no step finds its rows in L2.  The
+    block is captured into a CUDA graph once and replayed `reps` times (median); the dense
+    baseline likewise.  Bytes are the algorithmic bytes of the path: K once per retrieval and
+    the gathered K/V rows of every layer-step, logical (per query head) and unique (per KV head).
+    """
+    s = w.refresh
+    grouped = w.layer_group > 1
+    NL = w.layer_group if grouped else copies
+    ws = w.scaled(layers=NL, steps=s + 1)
+    kv, table = _make_caches(ws, dev)
+    q = W.make_queries(ws, dev)
+    B, Hq = ws.batch, ws.q_heads
+    kps = W.top_k_per_seq(ws)
+    max_k = max(ws.top_k, int(ws.k_frac * ws.context))
+    ctx = P.Context(NL, B, Hq, ws.kv_heads, ws.capacity, max_k, ws.window, ws.sinks, max_dilate_r=ws.dilate_r,
+                    page_size=ws.page_size, min_layer_group=ws.layer_group)
+    sched = P.make_schedule(ws.top_k, ws.window, ws.sinks, refresh_interval=s, layer_group=ws.layer_group,
+                            dilate_r=ws.dilate_r, top_k_per_seq=None if kps is None else kps.to(dev),
+                            flags=P.PRHS_GROUP_SETS if group_sets else 0)
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    lens = [W.seq_lens_at(ws, n).to(dev) for n in range(s)]
+    views = [[P.make_view(kv[l][0], kv[l][1], lens[n], page_table=table, max_seq_len=ws.capacity)
+              for n in range(s)] for l in range(NL)]
+    order = [(l, n) for n in range(s) for l in range(NL)]
+
+    def block(kind, stream=None):
+        for l, n in order:
+            if kind == "sparse":
+                ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out, stream=stream)
+            else:
+                ctx.dense_decode_attn(q[l, n], views[l][n], B, out, stream=stream)
+
+    # ---- bytes and per-step times from one directly launched block (an event pair per layer-step)
+    stream = torch.cuda.current_stream()
+    block("sparse")
+    torch.cuda.synchronize()
+    step_us, sizes, key_bytes = {}, {}, 0
+    evs = []
+    ctx.profile_begin(16 * len(order))
+    for l, n in order:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out)
+        b.record(stream)
+        evs.append((a, b))
+    prof = ctx.profile_end()
+    torch.cuda.synchronize()
+    retr = [(l, n) for l, n in order if n == 0 and (l % ws.layer_group == 0)]
+    times = {ln: a.elapsed_time(b) * 1e3 for ln, (a, b) in zip(order, evs)}
+    share = [ln for ln in order if ln not in retr]
+    step_us["retrieval"] = statistics.median(times[ln] for ln in retr)
+    step_us["sharing"] = statistics.median(times[ln] for ln in share) if share else None
+    kernels = {name: ms * 1e3 / cnt for name, (ms, cnt) in prof.items() if cnt}
+    # set sizes: the retrieving call (undilated set) and a sharing call (dilated set)
+    ctx.decode_step(0, 0, sched, q[0, 0], views[0][0], B, out)
+    idx_s, cnt_s = ctx.get_index_set(B)
+    sizes["retrieval"] = _set_bytes(idx_s, cnt_s, ws)
+    sizes["sharing"] = (0, 0)
+    if share:
+        l, n = (1, 0) if grouped else (0, 1)      # a follower layer, or the layer's next step
+        ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out)
+        idx_s, cnt_s = ctx.get_index_set(B)
+        sizes["sharing"] = _set_bytes(idx_s, cnt_s, ws)
+    key_bytes = int(lens[0].sum()) * ws.kv_heads * 256
+    n_retr, n_steps = len(retr), len(order)
+    per_step = {kind: (n_retr * (key_bytes + sizes["retrieval"][i]) + (n_steps - n_retr) * sizes["sharing"][i]) / n_steps
+                for i, kind in enumerate(("logical", "unique"))}
+    dense_bytes = int(lens[0].sum()) * ws.kv_heads * 512
+
+    # ---- whole blocks replayed from CUDA graphs
+    side = torch.cuda.Stream()
+    graphs = {}
+    with torch.cuda.stream(side):
+        for kind in ("sparse", "dense"):
+            block(kind, side)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                block(kind, torch.cuda.current_stream())
+            graphs[kind] = g
+    torch.cuda.synchronize()
+    us = {}
+    for kind in ("sparse", "dense"):
+        graphs[kind].replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            graphs[kind].replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3 / n_steps)
+        us[kind] = (statistics.median(ts), min(ts), max(ts))
+    flags = ctx.check()
+    ctx.close()
+    del kv, views, graphs
+    torch.cuda.empty_cache()
+    res = {
+        "workload": ws.name, "batch": B, "q_heads": Hq, "kv_heads": ws.kv_heads, "context": ws.context,
+        "refresh_interval": s, "layer_group": ws.layer_group, "paged": bool(ws.page_size),
+        "caches": f"{NL} layers of one layer group" if grouped else f"{NL} independent copies of the layer",
+        "layer_steps_per_retrieval": n_steps // n_retr,
+        "us_per_layer_step": us["sparse"][0], "us_per_layer_step_min_max": list(us["sparse"][1:]),
+        "dense_us_per_layer_step": us["dense"][0], "dense_over_sparse": us["dense"][0] / us["sparse"][0],
+        "retrieval_step_us": step_us["retrieval"], "sharing_step_us": step_us["sharing"],
+        "retrieval_step_kernels_us": {k: round(v, 1) for k, v in kernels.items()},
+        "key_bytes_per_retrieval": key_bytes,
+        "gather_bytes_logical": {"retrieval_step": sizes["retrieval"][0], "sharing_step": sizes["sharing"][0]},
+        "gather_bytes_unique": {"retrieval_step": sizes["retrieval"][1], "sharing_step": sizes["sharing"][1]},
+        "bytes_per_layer_step_logical": per_step["logical"], "bytes_per_layer_step_unique": per_step["unique"],
+        "dense_bytes_per_layer_step": dense_bytes, "dense_gbs": dense_bytes / us["dense"][0] / 1e3,
+        "mean_set_size_sharing": float(cnt_s.float().mean()),
+        "select_fallback": bool(flags & P.PRHS_FLAG_SELECT_FALLBACK),
+    }
+    for kind in ("logical", "unique"):
+        gbs = per_step[kind] / us["sparse"][0] / 1e3
+        res[f"achieved_gbs_{kind}"] = gbs
+        res[f"frac_of_8tbs_{kind}"] = gbs / 8000.0
+        if hbm_peak_gbs:
+            res[f"frac_of_measured_peak_{kind}"] = gbs / hbm_peak_gbs
+    return res
+
+
+def configs_summary(dev, group_sets=False, only=None, batch=0):
+    import json
+    for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
+        if only and w.name != only:
+            continue
+        if batch:
+            w = w.scaled(batch=batch)
+        print(json.dumps(config_summary(w, dev, group_sets=group_sets)), flush=True)
+
+
 def table3(dev, graph=False):
     if graph:
         print("| BS | seqlen | k | dense us / step | s=8 us / step | s=16 us / step | dense / s=8 | dense / s=16 "
@@ -175,10 +350,8 @@ def table3(dev, graph=False):
         print("|---|---|---|---|---|---|---|---|---|")
         for batch in (8, 16):
             for n in (1024, 2048, 4096):
-                k = n // 8 - 80
-                w = W.Workload(f"table3_b{batch}_{n}", layers=1, batch=batch, q_heads=32, kv_heads=32, context=n,
-                               steps=4, top_k=k, window=64, sinks=16, refresh=8, heavy_hitters=16,
-                               decay_span=min(512, n // 8), seed=100 + batch + n)
+                w = table3_workload(batch, n)
+                k = w.top_k
                 r8, r16 = time_blocks(w, dev, 8), time_blocks(w, dev, 16)
                 pf, p8, p16 = PAPER_TABLE3_MS[(batch, n)]
                 print(f"| {batch} | {n} | {k} | {r16['dense']:.1f} | {r8['sparse']:.1f} | {r16['sparse']:.1f} | "
@@ -190,10 +363,8 @@ def table3(dev, graph=False):
     print("|---|---|---|---|---|---|---|---|---|---|")
     for batch in (8, 16):
         for n in (1024, 2048, 4096):
-            k = n // 8 - 80
-            w = W.Workload(f"table3_b{batch}_{n}", layers=1, batch=batch, q_heads=32, kv_heads=32, context=n,
-                           steps=4, top_k=k, window=64, sinks=16, refresh=8, heavy_hitters=16,
-                           decay_span=min(512, n // 8), seed=100 + batch + n)
+            w = table3_workload(batch, n)
+            k = w.top_k
             r = time_workload(w, dev)
             am = {s: (r["refresh_us"] + (s - 1) * r["shared_us"]) / s for s in (8, 16)}
             pf, p8, p16 = PAPER_TABLE3_MS[(batch, n)]
@@ -243,6 +414,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="whole blocks of steps (one retrieval and the sharing steps that follow) replayed from "
                          "CUDA graphs: time per step")
+    ap.add_argument("--summary", action="store_true",
+                    help="with --configs: one JSON line per configuration, timed as its own schedule runs it (layer "
+                         "groups included): time, bytes and roofline fractions per layer-step")
     ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
     ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
     ap.add_argument("--group-sets", action="store_true",
@@ -252,7 +426,9 @@ def main():
         raise SystemExit("needs a CUDA device")
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
-    if args.configs:
+    if args.configs and args.summary:
+        configs_summary(dev, args.group_sets, args.only, args.batch)
+    elif args.configs:
         (configs_graph if args.graph else configs)(dev, args.group_sets, args.only, args.batch)
     else:
         table3(dev, args.graph)

@@ -7,6 +7,9 @@ Tolerances (bf16 inputs, fp32 accumulation on the GPU, float64 in the oracle):
   attention y     max-abs 2e-2 against the oracle evaluated on the GPU's own index set
   delta           1e-4 absolute
   logits          1e-4 absolute + 1e-5 relative (fp32 accumulation order)
+  order inside S* two winners may appear in either order only if their oracle logits differ by
+                  no more than twice the logit tolerance (each side's fp32 logit is within one
+                  tolerance of the exact value); the order fixes the top-m of Eq. 10
 """
 from __future__ import annotations
 
@@ -20,6 +23,7 @@ from paper_2602_08329_b200 import workloads as W
 Y_TOL = 2e-2
 DELTA_TOL = 1e-4
 TIE_REL = 1e-3
+LOGIT_ATOL, LOGIT_RTOL = 1e-4, 1e-5
 SIM_TOL = 1e-4          # a cosine similarity this close to tau may fall either way (fp32 vs float64)
 
 
@@ -31,8 +35,15 @@ def tie_band(a_ref: float) -> float:
     return TIE_REL * max(abs(a_ref), 1e-3)
 
 
+def order_band(a_ref: float) -> float:
+    """How far apart two oracle logits may lie for the kernel to rank them the other way round."""
+    return 2.0 * (LOGIT_ATOL + LOGIT_RTOL * abs(a_ref))
+
+
 def check_topk_legal(a32: np.ndarray, got_desc: np.ndarray, want_desc: np.ndarray, where=""):
-    """`got_desc` must equal the oracle's S* except for near-ties with the k-th logit."""
+    """`got_desc` must equal the oracle's S* except for near-ties with the k-th logit (membership:
+    the 1e-3 relative band), and be in the oracle's order except between logits that the fp32
+    accumulation order cannot tell apart (order: twice the logit tolerance)."""
     assert len(got_desc) == len(want_desc), f"{where}: |S*| {len(got_desc)} != {len(want_desc)}"
     if len(want_desc) == 0:
         return
@@ -42,14 +53,15 @@ def check_topk_legal(a32: np.ndarray, got_desc: np.ndarray, want_desc: np.ndarra
     for i in diff:
         assert abs(float(a32[i]) - a_k) <= tie_band(a_k), \
             f"{where}: position {i} logit {a32[i]} differs from the oracle set beyond the tie band of {a_k}"
-    # descending order (ties by lower position) up to the same band
+    # descending order (ties by lower position), up to what the logit tolerance allows
     ag = a32[got_desc].astype(np.float64)
-    assert np.all(np.diff(ag) <= tie_band(a_k)), f"{where}: S* not in descending-logit order"
+    bands = 2.0 * (LOGIT_ATOL + LOGIT_RTOL * np.abs(ag[:-1]))
+    assert np.all(np.diff(ag) <= bands), f"{where}: S* not in descending-logit order"
     if len(diff) == 0:
         same = got_desc == want_desc
         for j in np.nonzero(~same)[0]:
-            assert abs(float(a32[got_desc[j]]) - float(a32[want_desc[j]])) <= tie_band(a32[want_desc[j]]), \
-                f"{where}: order differs at rank {j} beyond a near-tie"
+            assert abs(float(a32[got_desc[j]]) - float(a32[want_desc[j]])) <= order_band(a32[want_desc[j]]), \
+                f"{where}: order differs at rank {j} beyond what the logit tolerance allows"
 
 
 def make_ctx(w: W.Workload, **over):
@@ -218,7 +230,7 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                     stats["near_tie_sets"] += int(before > 0)
                     if check_scores:
                         sg = scores[b, hs, :t].numpy()
-                        assert np.allclose(sg, a32, atol=1e-4, rtol=1e-5), f"{where}: logits differ"
+                        assert np.allclose(sg, a32, atol=LOGIT_ATOL, rtol=LOGIT_RTOL), f"{where}: logits differ"
                     over_s[(b, hs)] = got         # legal: the oracle adopts it
             ref = orc.decode_step(l, n, qh, Ks, Vs, t_host.numpy(), units=units, want_delta=want_delta,
                                   override_s_star=over_s, override_ref=over_ref)

@@ -35,7 +35,7 @@ def test_library_exports_every_declared_symbol(lib):
 def test_version_and_struct_layout(lib):
     assert P.version().startswith("prhs-b200")
     # the ctypes mirrors must have the C layout the header implies (LP64)
-    assert ctypes.sizeof(P.Config) == 14 * 4
+    assert ctypes.sizeof(P.Config) == 15 * 4
     assert ctypes.sizeof(P.KvView) == 64
     assert ctypes.sizeof(P.Schedule) == 64
     assert P.KvView.seq_lens.offset == 48 and P.Schedule.top_k_per_seq.offset == 16
@@ -44,11 +44,11 @@ def test_version_and_struct_layout(lib):
 
 def test_create_validates_before_touching_the_device(lib):
     h = ctypes.c_void_p()
-    bad = P.Config(1, 1, 4, 2, 64, 1000, 0, 16, 16, 4, 1, -1, 1, 1)          # head_dim 64
+    bad = P.Config(1, 1, 4, 2, 64, 1000, 0, 16, 16, 4, 1, -1, 1, 1, 0)          # head_dim 64
     assert lib.prhs_create(ctypes.byref(bad), ctypes.byref(h)) == 2 and not h.value
-    bad = P.Config(1, 1, 4, 3, 128, 1000, 0, 16, 16, 4, 1, -1, 1, 1)         # Hkv does not divide Hq
+    bad = P.Config(1, 1, 4, 3, 128, 1000, 0, 16, 16, 4, 1, -1, 1, 1, 0)         # Hkv does not divide Hq
     assert lib.prhs_create(ctypes.byref(bad), ctypes.byref(h)) == 1
-    bad = P.Config(1, 1, 4, 2, 128, 1000, 8, 16, 16, 4, 1, -1, 1, 1)         # page size 8
+    bad = P.Config(1, 1, 4, 2, 128, 1000, 8, 16, 16, 4, 1, -1, 1, 1, 0)         # page size 8
     assert lib.prhs_create(ctypes.byref(bad), ctypes.byref(h)) == 2
     assert b"page_size" in lib.prhs_last_error(None)
     assert lib.prhs_create(None, ctypes.byref(h)) == 1

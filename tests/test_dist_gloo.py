@@ -54,3 +54,19 @@ def test_reference_arm_other_ranks_exit_without_work():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        capture_output=True, text=True, env=env, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_timed_window_is_whole_blocks_whatever_the_arguments():
+    import bench
+    L, s = 4, 4                                            # cache copies, refresh interval
+    for warm, steps in [(5, 20), (4, 16), (0, 1), (3, 17), (16, 32), (33, 7)]:
+        Wn, Kn = bench.aligned_window(warm, steps, L * s)
+        assert Wn >= max(warm, 1) and Kn >= max(steps, 1)
+        assert Wn % (L * s) == 0 and Kn % (L * s) == 0
+        # step i is decode step i // L of cache i % L: it retrieves iff (i // L) % s == 0
+        retrievals = sum((i // L) % s == 0 for i in range(Wn, Wn + Kn))
+        assert retrievals * s == Kn                        # the schedule's steady state, exactly
+        for l in range(L):                                 # every cache's first step in the window retrieves
+            first = next(i for i in range(Wn, Wn + Kn) if i % L == l)
+            assert (first // L) % s == 0
+    assert bench.aligned_window(5, 20, 16) == (16, 32)

@@ -3,6 +3,18 @@
 Small cases compare every element; the benchmark's full-size configurations compare sampled
 (sequence, head) units that the oracle computes one by one, in the launch configuration the
 benchmark times.  Tolerances are stated in tests/harness.py.
+
+The selection kernel's CTA width follows the number of (sequence, head) units, so the
+full-size tests are chosen to cover every width at the batch the configuration really uses:
+  1024 threads (at most one unit per SM)   test_c4_long_context_sampled (4 x 32 = 128 units),
+                                           test_c3_stack_slice_sampled (batch 4)
+  512 threads                              test_c2_full_size_sampled (8 x 32 = 256 units),
+                                           test_c5_full_batch_sampled (64 x 32 = 2048 units, a
+                                           multi-wave grid of every kernel)
+  256 threads (two to four units per SM)   test_c3_full_batch_sampled (16 x 32 = 512 units),
+                                           test_table3_operator_shapes[16-4096-16]
+Retrieval scoring runs the TMA kernels everywhere except in the test_score_ring_* tests, which
+create their contexts with PRHS_CFG_NO_TMA.
 """
 import math
 
@@ -385,6 +397,79 @@ def test_c5_serving_mix_sampled(cuda_device):
     assert st["checked"] == 5 * 3 * len(units)
 
 
+def test_c3_full_batch_sampled(cuda_device):
+    # the Mistral-shaped stack at its real batch of 16 (512 selection units: the 256-thread
+    # launch of the selection kernel), two layer groups, leaders and followers
+    w = W.C3_MISTRAL.scaled(layers=8, steps=6)
+    units = [(0, 0), (5, 9), (11, 22), (15, 31)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1, 3, 4, 7])
+    assert st["checked"] == 6 * 5 * len(units)
+    assert not st["select_fallback"]
+
+
+def test_c5_full_batch_sampled(cuda_device):
+    # the serving mix at its real batch of 64 ragged, paged sequences (2048 selection units,
+    # k_b = floor(0.03 N_b)): the leader and one follower of a layer group
+    w = W.C5_SERVING.scaled(layers=4, steps=5)
+    units = [(0, 0), (17, 9), (40, 31), (63, 16), (29, 4)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1], paged=True)
+    assert st["checked"] == 5 * 2 * len(units)
+    assert not st["select_fallback"]
+
+
+# ----------------------------------------- the paper's operator-benchmark shapes (Sec. 5.4, Table 3)
+@pytest.mark.parametrize("batch,n,s", [(16, 4096, 16), (8, 1024, 8)])
+def test_table3_operator_shapes(cuda_device, batch, n, s):
+    # budgets of Sec. 5.3.2 (C_sink 16, C_local 64, k = n/8 - 80 = 432 at 4k), blocks of s steps:
+    # one whole block and the start of the next
+    from paper_2602_08329_b200 import operator_latency as OL
+    w = OL.table3_workload(batch, n, s).scaled(steps=s + 2)
+    assert (w.sinks, w.window) == (16, 64) and w.top_k == (432 if n == 4096 else 48)
+    g = np.random.default_rng(batch + n)
+    units = sorted({(int(g.integers(batch)), int(g.integers(32))) for _ in range(20)})
+    st = H.run_schedule_parity(w, cuda_device, units)
+    assert st["checked"] == (s + 2) * len(units)
+    assert st["retrievals"] == 2 * len(units) and not st["select_fallback"]
+    assert max(st["set_sizes"]) <= 16 + w.top_k + 2 * (w.top_k // 3) + 64
+
+
+# --------------------------------------------------- retrieval scoring without the TMA kernels
+@pytest.mark.parametrize("paged", [False, True])
+def test_score_ring_small_every_unit(cuda_device, paged):
+    # PRHS_CFG_NO_TMA: the key stream goes through the cp.async ring kernel (what the library
+    # falls back to by itself when the driver offers no tensor-map encoder)
+    w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=3, q_heads=8, kv_heads=2, context=2700,
+              min_context=400 if paged else 0, page_size=16 if paged else 0, seed=17)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, ctx_over=dict(flags=P.PRHS_CFG_NO_TMA))
+    assert st["checked"] == 2 * 4 * w.batch * w.q_heads
+
+
+def test_score_ring_c2_sampled(cuda_device):
+    w = W.C2_LLAMA2_7B.scaled(steps=5)
+    units = [(0, 0), (6, 30), (2, 11)]
+    st = H.run_schedule_parity(w, cuda_device, units, ctx_over=dict(flags=P.PRHS_CFG_NO_TMA))
+    assert st["checked"] == 5 * len(units) and not st["select_fallback"]
+
+
+def test_score_ring_and_tma_logits_agree(cuda_device):
+    # the two scoring kernels on the same inputs: same logits (both within the tolerance of the
+    # oracle, so within twice that of each other) and the same log-sum-exp
+    w = small(batch=2, q_heads=8, kv_heads=2, context=5000, top_k=64, seed=18)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device), max_seq_len=w.capacity)
+    res = []
+    for flags in (0, P.PRHS_CFG_NO_TMA):
+        ctx = H.make_ctx(w, flags=flags)
+        lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+        ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), w.batch, out_lse_full=lse)
+        assert ctx.check() == 0
+        res.append((ctx.get_scores(w.batch)[:, :, : w.context + 1], lse.cpu()))
+        ctx.close()
+    assert torch.allclose(res[0][0], res[1][0], atol=2 * H.LOGIT_ATOL, rtol=2 * H.LOGIT_RTOL)
+    assert torch.allclose(res[0][1], res[1][1], atol=1e-4)
+
+
 # ------------------------------------------------------------------- host-buffer entry point
 @pytest.mark.parametrize("pinned", [True, False])
 def test_decode_step_host_buffers(cuda_device, pinned):
@@ -455,6 +540,59 @@ def test_host_side_errors(cuda_device):
         P.Context(1, 1, 4, 2, 1000, 16, 16, 4, head_dim=64)
     assert e.value.status == 2
     ctx.decode_step(0, 0, good, q, view, w.batch, out)                                   # still usable
+    assert ctx.check() == 0
+    ctx.close()
+
+
+def test_host_entry_point_rejects_rows_beyond_the_cache(cuda_device):
+    """A context dimensioned for longer sequences than the cache holds: the host-buffer entry
+    point must refuse a length whose new row would land outside the cache, before it writes
+    anything (the cache and the device lengths stay as they were)."""
+    w = small(steps=2)
+    k, v = W.make_kv(w, cuda_device)
+    k0, v0 = k.clone(), v.clone()
+    ctx = H.make_ctx(w, max_context=w.capacity + 4000)
+    sched = H.make_sched(w, cuda_device)
+    t_dev = torch.full((w.batch,), 7, dtype=torch.int32, device=cuda_device)
+    g = torch.Generator().manual_seed(5)
+    hq = torch.randn(w.batch, w.q_heads, 128, generator=g).to(torch.bfloat16).pin_memory()
+    hk = torch.randn(w.batch, w.kv_heads, 128, generator=g).to(torch.bfloat16).pin_memory()
+    hout = torch.zeros(w.batch, w.q_heads, 128, dtype=torch.bfloat16).pin_memory()
+
+    def status(t_list, view, **kw):
+        ht = torch.tensor(t_list, dtype=torch.int32).pin_memory()
+        with pytest.raises(P.PrhsError) as e:
+            ctx.decode_step_host(0, 0, kw.get("sched", sched), hq, hk, hk, ht, view, w.batch, hout)
+        return e.value.status
+
+    full = P.make_view(k, v, t_dev)                                # max_seq_len 0: the context's maximum
+    assert status([w.capacity + 1, 10], full) == 6                 # beyond the (b, kvh) slice (strides)
+    assert status([10, w.capacity + 3999], full) == 6
+    short = P.make_view(k, v, t_dev, max_seq_len=1000)
+    assert status([1001, 10], short) == 6                          # beyond the capacity the view declares
+    assert status([0, 10], full) == 1
+    assert status([10, 10], full, sched=H.make_sched(w, cuda_device, top_k=w.top_k + 1)) == 6   # bad schedule
+    torch.cuda.synchronize()
+    assert torch.equal(k, k0) and torch.equal(v, v0) and bool((t_dev == 7).all())   # nothing was written
+    ht = torch.tensor([w.capacity, 1000], dtype=torch.int32).pin_memory()           # the largest legal length
+    ctx.decode_step_host(0, 0, sched, hq, hk, hk, ht, full, w.batch, hout)
+    assert ctx.check() == 0 and torch.equal(t_dev.cpu(), ht)
+    ctx.close()
+
+
+def test_default_dilation_count_must_fit_the_context(cuda_device):
+    # m = floor(k / 3) by default: a context created for fewer dilated winners refuses the schedule
+    # instead of truncating the dilated set
+    w = small()
+    ctx = H.make_ctx(w, max_dilate_m=3)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device))
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    with pytest.raises(P.PrhsError) as e:
+        ctx.decode_step(0, 0, H.make_sched(w, cuda_device), q, view, w.batch, out)      # 48 / 3 = 16 > 3
+    assert e.value.status == 6
+    ctx.decode_step(0, 0, H.make_sched(w, cuda_device, dilate_m=3), q, view, w.batch, out)
     assert ctx.check() == 0
     ctx.close()
 
