@@ -446,13 +446,17 @@ def run_cuda(args):
             dist.destroy_process_group()
         return 0
 
+    launch_desc = ("each repeat of the K timed steps is one replay of a CUDA graph captured from the same "
+                   "prhs_decode_step calls; value = median repeat"
+                   if graph is not None else "direct launches; value = median repeat")
     # ---- the other full-size configurations, each timed as its own schedule runs it (one layer
     # group, or independent copies of a single layer), per layer-step
     other = None
     if world == 1 and not args.no_other_configs and not args.batch:
         from paper_2602_08329_b200 import operator_latency as OL
         ctx.close()
-        del kv_layers, views, views_h, q_all, graph
+        ctx = None
+        del kv_layers, views, views_h, q_all, graph, host
         torch.cuda.empty_cache()
         other = {}
         for ow in (W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
@@ -482,9 +486,7 @@ def run_cuda(args):
         "config": workload_config(w, {
             "parallelism": f"replicas x{world} (no collective)",
             "cache_copies": L,
-            "launch": ("each repeat of the K timed steps is one replay of a CUDA graph captured from the same "
-                       "prhs_decode_step calls; value = median repeat"
-                       if graph is not None else "direct launches; value = median repeat"),
+            "launch": launch_desc,
             "kernel_timing": "event pairs inside the library around every launch, on a back-to-back replay of the "
                              "same K steps (the timed region itself carries no instrumentation)",
             "l2": (f"no flush: {L} independent copies of the layer's cache (4.3 GB each) visited round-robin, "
@@ -517,7 +519,8 @@ def run_cuda(args):
         "cpu_baseline": cpu, "other_configs": other,
     }
     print(json.dumps(line))
-    ctx.close()
+    if ctx is not None:
+        ctx.close()
     if dist is not None:
         dist.destroy_process_group()
     return 0

@@ -53,7 +53,7 @@ build_set_kernel(SetRef ref, const int* __restrict__ seq_lens, int num_q_heads,
 }
 
 // ------------------------------------------------------------ gathered / dense attention
-constexpr int kPartStride = kHeadDim + 2;         // o[128] (unnormalised), m, l per split
+constexpr int kPartStride = kHeadDim + 4;         // o[128] (unnormalised), m, l, l~ per split (+ padding)
 
 struct AttnParams {
   const __nv_bfloat16* q;   // [B][Hq][128]
@@ -67,7 +67,7 @@ struct AttnParams {
   // idx == nullptr and set.star == nullptr: all positions [0, t) (dense baseline)
   int num_q_heads, group_size;
   int splits;
-  float* partials;          // [B][Hq][splits][kPartStride]
+  float* partials;          // [B][Hq][splits][kPartStride]: o, m, l, l~ (see below)
   unsigned int* tickets;    // [B][Hq], zero on entry, zero again on exit
   __nv_bfloat16* out;       // [B][Hq][128]
   float* out_lse;           // [B][Hq] or nullptr
@@ -154,6 +154,11 @@ __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit
 //               16 n-tiles x 1 k-step; lanes 0-3 hold the 128 output columns.
 // Index sets are per query head, so only one of the 16 tile rows carries data; the tensor
 // cores are used for their instruction economy, not their FLOPs.
+// The weights enter the P V product rounded to bf16.  Two sums of them are kept: l, of the fp32
+// weights, gives the log-sum-exp (and through it delta) at full precision; l~, of the weights
+// as rounded, divides the output, so that the output is a convex combination of the value rows
+// with consistently normalised weights (where one key dominates, its weight stays 1 instead of
+// carrying the rounding error of its bf16 image).
 constexpr int kTWarps = 4;
 constexpr int kTThreads = kTWarps * 32;
 constexpr int kTStageRows = 16;
@@ -217,7 +222,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
 #pragma unroll
   for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; }
   float z0 = 0.f, z1 = 0.f;            // accumulator rows 8..15: always zero
-  float m = -INFINITY, l = 0.f;
+  float m = -INFINITY, l = 0.f, lt = 0.f;     // lt: the sum of the weights as rounded to bf16
 
   // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane.  Each level is
   // produced one step before it is consumed, so that no load is waited for where it is issued:
@@ -362,6 +367,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
       const float corr = exp2f(m - mn);     // m = -inf on the first real stage: corr = 0
       m = mn;
       l *= corr;
+      lt *= corr;
 #pragma unroll
       for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
     }
@@ -369,6 +375,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
       const float p0 = exp2f(s0 - m), p1 = exp2f(s1 - m), p2 = exp2f(s2 - m), p3 = exp2f(s3 - m);
       l += (p0 + p1) + (p2 + p3);
       const uint32_t ap0 = pack_bf16x2(p0, p1), ap2 = pack_bf16x2(p2, p3);
+      lt += (bf_lo(ap0) + bf_hi(ap0)) + (bf_lo(ap2) + bf_hi(ap2));
       // ---- O += P V
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
@@ -388,33 +395,36 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   cp_async_wait<0>();
   l += __shfl_xor_sync(0xffffffffu, l, 1);
   l += __shfl_xor_sync(0xffffffffu, l, 2);
+  lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+  lt += __shfl_xor_sync(0xffffffffu, lt, 2);
 
   // ---- combine the warps of this CTA (lanes 0-3 hold row 0: columns 8*nt + 2*tg, +1)
   __shared__ float sm_o[kTWarps][kHeadDim];
-  __shared__ float sm_m[kTWarps], sm_l[kTWarps];
+  __shared__ float sm_m[kTWarps], sm_l[kTWarps], sm_lt[kTWarps];
   __shared__ bool is_last;
   if (g == 0) {
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt)
       *reinterpret_cast<float2*>(&sm_o[warp][nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
   }
-  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; sm_lt[warp] = lt; }
   __syncthreads();
   {
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w]);
-    float acc = 0.f, L = 0.f;
+    float acc = 0.f, L = 0.f, Lt = 0.f;
     if (M != -INFINITY) {
 #pragma unroll
       for (int w = 0; w < kTWarps; ++w) {
         const float scw = exp2f(sm_m[w] - M);
         acc = fmaf(sm_o[w][tid], scw, acc);
         L = fmaf(sm_l[w], scw, L);
+        Lt = fmaf(sm_lt[w], scw, Lt);
       }
     }
     if (p.splits == 1) {
-      p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+      p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(Lt > 0.f ? acc / Lt : 0.f);
       if (tid == 0) {
         const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
         if (p.out_lse) p.out_lse[unit] = lse;
@@ -424,7 +434,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
     }
     float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
     part[tid] = acc;
-    if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
+    if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; part[kHeadDim + 2] = Lt; }
   }
   __threadfence();
   __syncthreads();
@@ -439,15 +449,16 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   const float* base = p.partials + (long long)unit * p.splits * kPartStride;
   float M = -INFINITY;
   for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
-  float acc = 0.f, L = 0.f;
+  float acc = 0.f, L = 0.f, Lt = 0.f;
   if (M != -INFINITY) {
     for (int sp = 0; sp < p.splits; ++sp) {
       const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
       acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
       L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
+      Lt = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 2), scw, Lt);
     }
   }
-  p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(Lt > 0.f ? acc / Lt : 0.f);
   if (tid == 0) {
     const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     if (p.out_lse) p.out_lse[unit] = lse;
@@ -476,7 +487,7 @@ __device__ __forceinline__ void mma_bf16_full(float (&d)[4], uint32_t a0, uint32
 // lane's four keys (rows 2tg, 2tg+1, 8+2tg, 9+2tg of the stage) are real.
 __device__ __forceinline__ void group_stage(uint32_t kt, uint32_t vt, const uint32_t (&aq)[8][4], bool v0, bool v1,
                                             bool v2, bool v3, float (&o)[16][4], float& m0, float& l0, float& m1,
-                                            float& l1) {
+                                            float& l1, float& lt0, float& lt1) {
   const int lane = threadIdx.x & 31;
   const int lm_mi = lane >> 3, lm_r = lane & 7;
   const int vrow = (lm_mi & 1) * 8 + lm_r;
@@ -513,6 +524,7 @@ __device__ __forceinline__ void group_stage(uint32_t kt, uint32_t vt, const uint
     const float c1 = (n1 == -INFINITY) ? 1.f : exp2f(m1 - n1);
     m0 = n0; m1 = n1;
     l0 *= c0; l1 *= c1;
+    lt0 *= c0; lt1 *= c1;
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= c0; o[nt][1] *= c0; o[nt][2] *= c1; o[nt][3] *= c1; }
   }
@@ -526,6 +538,8 @@ __device__ __forceinline__ void group_stage(uint32_t kt, uint32_t vt, const uint
   l1 += (pw[1][0] + pw[1][1]) + (pw[1][2] + pw[1][3]);
   const uint32_t a0 = pack_bf16x2(pw[0][0], pw[0][1]), a1 = pack_bf16x2(pw[1][0], pw[1][1]);
   const uint32_t a2 = pack_bf16x2(pw[0][2], pw[0][3]), a3 = pack_bf16x2(pw[1][2], pw[1][3]);
+  lt0 += (bf_lo(a0) + bf_hi(a0)) + (bf_lo(a2) + bf_hi(a2));      // the weights as the MMA sees them
+  lt1 += (bf_lo(a1) + bf_hi(a1)) + (bf_lo(a3) + bf_hi(a3));
   // ---- O += P V
 #pragma unroll
   for (int np = 0; np < 8; ++np) {
@@ -542,17 +556,22 @@ __device__ __forceinline__ void group_stage(uint32_t kt, uint32_t vt, const uint
 // is free by now and holds [warp][head][128] floats.
 __device__ __forceinline__ void group_epilogue(const AttnParams& p, unsigned char* g_smem, int b, int head0, int gq,
                                                int split, float (&o)[16][4], float m0, float l0, float m1,
-                                               float l1) {
+                                               float l1, float lt0, float lt1) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  lt0 += __shfl_xor_sync(0xffffffffu, lt0, 1);
+  lt0 += __shfl_xor_sync(0xffffffffu, lt0, 2);
+  lt1 += __shfl_xor_sync(0xffffffffu, lt1, 1);
+  lt1 += __shfl_xor_sync(0xffffffffu, lt1, 2);
   __syncthreads();
   float* sm_o = reinterpret_cast<float*>(g_smem);                       // 4 x 16 x 128 floats = 32 KB
   float* sm_m = sm_o + kTWarps * 16 * kHeadDim;                         // [warp][16]
   float* sm_l = sm_m + kTWarps * 16;
+  float* sm_lt = sm_l + kTWarps * 16;
   __shared__ bool is_last;
 #pragma unroll
   for (int nt = 0; nt < 16; ++nt) {
@@ -560,12 +579,12 @@ __device__ __forceinline__ void group_epilogue(const AttnParams& p, unsigned cha
     *reinterpret_cast<float2*>(&sm_o[(warp * 16 + g + 8) * kHeadDim + nt * 8 + 2 * tg]) = make_float2(o[nt][2], o[nt][3]);
   }
   if (tg == 0) {
-    sm_m[warp * 16 + g] = m0; sm_l[warp * 16 + g] = l0;
-    sm_m[warp * 16 + g + 8] = m1; sm_l[warp * 16 + g + 8] = l1;
+    sm_m[warp * 16 + g] = m0; sm_l[warp * 16 + g] = l0; sm_lt[warp * 16 + g] = lt0;
+    sm_m[warp * 16 + g + 8] = m1; sm_l[warp * 16 + g + 8] = l1; sm_lt[warp * 16 + g + 8] = lt1;
   }
   __syncthreads();
-  auto finish = [&](int unit, float acc, float M, float L) {
-    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  auto finish = [&](int unit, float acc, float M, float L, float Lt) {
+    p.out[(long long)unit * kHeadDim + tid] = __float2bfloat16_rn(Lt > 0.f ? acc / Lt : 0.f);
     if (tid == 0) {
       const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
       if (p.out_lse) p.out_lse[unit] = lse;
@@ -577,21 +596,22 @@ __device__ __forceinline__ void group_epilogue(const AttnParams& p, unsigned cha
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kTWarps; ++w) M = fmaxf(M, sm_m[w * 16 + j]);
-    float acc = 0.f, L = 0.f;
+    float acc = 0.f, L = 0.f, Lt = 0.f;
     if (M != -INFINITY) {
 #pragma unroll
       for (int w = 0; w < kTWarps; ++w) {
         const float scw = exp2f(sm_m[w * 16 + j] - M);
         acc = fmaf(sm_o[(w * 16 + j) * kHeadDim + tid], scw, acc);
         L = fmaf(sm_l[w * 16 + j], scw, L);
+        Lt = fmaf(sm_lt[w * 16 + j], scw, Lt);
       }
     }
     if (p.splits == 1) {
-      finish(unit, acc, M, L);
+      finish(unit, acc, M, L, Lt);
     } else {
       float* part = p.partials + ((long long)unit * p.splits + split) * kPartStride;
       part[tid] = acc;
-      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; }
+      if (tid == 0) { part[kHeadDim] = M; part[kHeadDim + 1] = L; part[kHeadDim + 2] = Lt; }
     }
   }
   if (p.splits == 1) return;
@@ -611,15 +631,16 @@ __device__ __forceinline__ void group_epilogue(const AttnParams& p, unsigned cha
     const float* base = p.partials + (long long)unit * p.splits * kPartStride;
     float M = -INFINITY;
     for (int sp = 0; sp < p.splits; ++sp) M = fmaxf(M, __ldcg(base + sp * kPartStride + kHeadDim));
-    float acc = 0.f, L = 0.f;
+    float acc = 0.f, L = 0.f, Lt = 0.f;
     if (M != -INFINITY) {
       for (int sp = 0; sp < p.splits; ++sp) {
         const float scw = exp2f(__ldcg(base + sp * kPartStride + kHeadDim) - M);
         acc = fmaf(__ldcg(base + sp * kPartStride + tid), scw, acc);
         L = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 1), scw, L);
+        Lt = fmaf(__ldcg(base + sp * kPartStride + kHeadDim + 2), scw, Lt);
       }
     }
-    finish(unit, acc, M, L);
+    finish(unit, acc, M, L, Lt);
   }
 }
 
@@ -656,6 +677,7 @@ __global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p)
 #pragma unroll
   for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; o[nt][2] = 0.f; o[nt][3] = 0.f; }
   float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // rows g and g + 8
+  float lt0 = 0.f, lt1 = 0.f;
 
   const bool paged = p.kv.page_table != nullptr;
   const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
@@ -702,10 +724,10 @@ __global__ void __launch_bounds__(kTThreads) dense_attn_mma_kernel(AttnParams p)
     const int pos0 = start + i * kTStageRows;
     // keys of this lane: pos0 + 2tg, +1 (n-tile 0) and pos0 + 8 + 2tg, +1 (n-tile 1)
     group_stage(kt, kt + kTTileBytes, aq, pos0 + 2 * tg < end, pos0 + 2 * tg + 1 < end, pos0 + 8 + 2 * tg < end,
-                pos0 + 9 + 2 * tg < end, o, m0, l0, m1, l1);
+                pos0 + 9 + 2 * tg < end, o, m0, l0, m1, l1, lt0, lt1);
   }
   cp_async_wait<0>();
-  group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1);
+  group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1, lt0, lt1);
 }
 
 // ------------------------------------------------------- retrieval scoring, ring variant

@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(kTThreads) gather_group_attn_mma_kernel(AttnPa
 #pragma unroll
   for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; o[nt][2] = 0.f; o[nt][3] = 0.f; }
   float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // rows g and g + 8
+  float lt0 = 0.f, lt1 = 0.f;                                 // sums of the weights as rounded to bf16
 
   // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane; every level is
   // produced one step before it is consumed (see gather_attn_mma_kernel).
@@ -143,10 +144,10 @@ __global__ void __launch_bounds__(kTThreads) gather_group_attn_mma_kernel(AttnPa
     issue(i + kTStages - 1);
     const uint32_t kt = ring + (uint32_t)slot_i * kTStageBytes;
     group_stage(kt, kt + kTTileBytes, aq, (vm >> (2 * tg)) & 1u, (vm >> (2 * tg + 1)) & 1u,
-                (vm >> (8 + 2 * tg)) & 1u, (vm >> (9 + 2 * tg)) & 1u, o, m0, l0, m1, l1);
+                (vm >> (8 + 2 * tg)) & 1u, (vm >> (9 + 2 * tg)) & 1u, o, m0, l0, m1, l1, lt0, lt1);
   }
   cp_async_wait<0>();
-  group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1);
+  group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1, lt0, lt1);
 }
 
 }  // namespace prhs

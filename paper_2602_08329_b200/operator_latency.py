@@ -315,7 +315,7 @@ def config_summary(w: W.Workload, dev, reps: int = 7, copies: int = 4, group_set
         "us_per_layer_step": us["sparse"][0], "us_per_layer_step_min_max": list(us["sparse"][1:]),
         "dense_us_per_layer_step": us["dense"][0], "dense_over_sparse": us["dense"][0] / us["sparse"][0],
         "retrieval_step_us": step_us["retrieval"], "sharing_step_us": step_us["sharing"],
-        "retrieval_step_kernels_us": {k: round(v, 1) for k, v in kernels.items()},
+        "kernel_avg_us_per_launch": {k: round(v, 1) for k, v in kernels.items()},
         "key_bytes_per_retrieval": key_bytes,
         "gather_bytes_logical": {"retrieval_step": sizes["retrieval"][0], "sharing_step": sizes["sharing"][0]},
         "gather_bytes_unique": {"retrieval_step": sizes["retrieval"][1], "sharing_step": sizes["sharing"][1]},

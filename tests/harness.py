@@ -4,7 +4,11 @@ oracle on the same seeded tensors, and compare with the tolerances the benchmark
 Tolerances (bf16 inputs, fp32 accumulation on the GPU, float64 in the oracle):
   index sets      bit-exact, except positions whose oracle logit lies within 1e-3 relative
                   of the k-th (or, for dilation extras, the m-th) largest logit
-  attention y     max-abs 2e-2 against the oracle evaluated on the GPU's own index set
+  attention y     max-abs 2e-2 between the kernel's bf16 output and the oracle's float64 value,
+                  the oracle evaluated on the GPU's own index set.  (The oracle's value is not
+                  rounded to bf16 first: with both sides rounded, a value near a rounding tie at
+                  |y| >= 4, where one bf16 step is 2^-5 = 0.031, can land one whole step apart
+                  although each side is within half a step of the exact result.)
   delta           1e-4 absolute
   logits          1e-4 absolute + 1e-5 relative (fp32 accumulation order)
   order inside S* two winners may appear in either order only if their oracle logits differ by
@@ -245,7 +249,7 @@ def run_schedule_parity(w: W.Workload, device, units, layers=None, steps=None, w
                 C_want = ref["set"][(b, h)]
                 C_got = idx[b, h, : int(cnt[b, h])].numpy().astype(np.int64)
                 assert np.array_equal(C_got, C_want), f"{where}: index set differs"
-                err = float(np.max(np.abs(y_gpu[b, h] - O.bf16_round(ref["y"][(b, h)]))))
+                err = float(np.max(np.abs(y_gpu[b, h] - ref["y"][(b, h)])))
                 assert err <= Y_TOL, f"{where}: attention max-abs error {err}"
                 stats["max_y_err"] = max(stats["max_y_err"], err)
                 stats["set_sizes"].append(len(C_want))
