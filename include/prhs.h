@@ -79,6 +79,14 @@ typedef struct {
                               the library falls back to on its own when the driver does not export
                               cuTensorMapEncodeTiled or the cache spans 2^31 rows or more.  Same
                               results; for testing that path and for comparing the two. */
+#define PRHS_CFG_TMA_GATHER 2u /* the gathered attention (per-head sets) brings its rows in with TMA row
+                              gathers (cp.async.bulk.tensor tile::gather4, four rows per instruction,
+                              no multicast) instead of 16-byte cp.async copies.  Same results.  Off by
+                              default because it measured slower: a tile that ldmatrix reads without
+                              bank conflicts needs the 128-byte swizzle, hence two 64-column boxes per
+                              row, and at that granularity the copy engine falls behind (a sharing step
+                              of the 32K-context layer: 59.9 us against 51.7 us).  Kept so that the
+                              comparison can be repeated (python -m paper_2602_08329_b200.gather_ceiling). */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at
@@ -336,6 +344,18 @@ prhs_status prhs_profile_begin(prhs_ctx* ctx, int32_t max_launches);
 prhs_status prhs_profile_end(prhs_ctx* ctx, void* stream, float* host_ms_per_kind,
                              int64_t* host_launches_per_kind);
 const char* prhs_kernel_kind_name(int32_t kind);
+
+/* Measurement support (no counterpart in the paper): the bare row gather of
+ * prhs_sparse_decode_attn, without its arithmetic.  Fetches the K row and the V row of every
+ * entry of the given lists (same arguments, contiguous caches only) with the work laid out as the
+ * attention kernel lays it out, and discards them.  variant: 0 = plain 16-byte loads into
+ * registers, 1 = 16-byte cp.async copies into a shared-memory ring (the attention kernel's
+ * mechanism), 2 = one 256-byte bulk copy per row, 3 = TMA row gather (tile::gather4, four rows per
+ * instruction).  Timed with CUDA events by the caller, it gives the ceiling each mechanism sets for
+ * the gathered attention on the same index pattern (python -m paper_2602_08329_b200.gather_ceiling).
+ * Out-of-range entries are replaced by a valid row and flagged.  Asynchronous on `stream`. */
+prhs_status prhs_gather_probe(prhs_ctx* ctx, int32_t variant, const prhs_kv_view* kv, const int32_t* idx,
+                              const int32_t* count, int32_t idx_stride, int32_t batch, void* stream);
 
 /* Number of kernels this context has launched since creation (host-side counter). */
 int64_t prhs_launch_count(const prhs_ctx* ctx);

@@ -23,6 +23,7 @@ PRHS_WANT_DELTA = 2
 PRHS_GROUP_SETS = 4
 PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TIMEOUT = 1, 2, 4, 8
 PRHS_CFG_NO_TMA = 1
+PRHS_CFG_TMA_GATHER = 2
 
 # every symbol include/prhs.h declares
 EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_set",
@@ -31,7 +32,7 @@ EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_s
            "prhs_get_shared_set", "prhs_get_scores", "prhs_scores_ld", "prhs_check",
            "prhs_launch_count", "prhs_selftest_wait", "prhs_state_bytes", "prhs_state_export", "prhs_state_import", "prhs_validate_index_lists", "prhs_last_error", "prhs_version", "prhs_profile_begin",
            "prhs_profile_end", "prhs_kernel_kind_name", "prhs_sparse_decode_attn_noalloc", "prhs_get_gate",
-           "prhs_noalloc_check"]
+           "prhs_noalloc_check", "prhs_gather_probe"]
 NOALLOC_MAX_UNITS = 1024
 KERNEL_KINDS = 6
 
@@ -86,6 +87,7 @@ def load() -> C.CDLL:
         "prhs_dense_decode_attn": (st, [vp, vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_sparse_decode_attn_noalloc": (st, [vp, C.POINTER(KvView), vp, vp, i32, i32, i32, i32, vp, vp, vp]),
         "prhs_noalloc_check": (st, [vp, C.POINTER(C.c_uint32)]),
+        "prhs_gather_probe": (st, [vp, i32, C.POINTER(KvView), vp, vp, i32, i32, vp]),
         "prhs_decode_step": (st, [vp, i32, i32, C.POINTER(Schedule), vp, C.POINTER(KvView), i32, vp, vp, vp]),
         "prhs_decode_step_host": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32, vp, vp]),
         "prhs_decode_step_host_async": (st, [vp, i32, i32, C.POINTER(Schedule), vp, vp, vp, vp, C.POINTER(KvView), i32,
@@ -213,6 +215,11 @@ class Context:
         self._ck(self.lib.prhs_sparse_decode_attn(self.h, _ptr(q), C.byref(view), _ptr(idx), _ptr(count),
                                                   idx.shape[-1], batch, _ptr(out), _ptr(out_lse),
                                                   _stream(stream)))
+
+    def gather_probe(self, variant, view, idx, count, batch, stream=None):
+        """The bare row gather of sparse_decode_attn (measurement support; see prhs_gather_probe)."""
+        self._ck(self.lib.prhs_gather_probe(self.h, variant, C.byref(view), _ptr(idx), _ptr(count), idx.shape[-1],
+                                            batch, _stream(stream)))
 
     def dense_decode_attn(self, q, view, batch, out, out_lse=None, stream=None):
         self._ck(self.lib.prhs_dense_decode_attn(self.h, _ptr(q), C.byref(view), batch, _ptr(out),

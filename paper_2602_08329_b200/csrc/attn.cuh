@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   lt += __shfl_xor_sync(0xffffffffu, lt, 2);
 
   // ---- combine the warps of this CTA (lanes 0-3 hold row 0: columns 8*nt + 2*tg, +1)
-  __shared__ float sm_o[kTWarps][kHeadDim];
+  __shared__ __align__(16) float sm_o[kTWarps][kHeadDim];       // written as float2
   __shared__ float sm_m[kTWarps], sm_l[kTWarps], sm_lt[kTWarps];
   __shared__ bool is_last;
   if (g == 0) {

@@ -20,6 +20,8 @@
 #include "attn_group.cuh"
 #include "score_tma.cuh"
 #include "select.cuh"
+#include "gather_probe.cuh"
+#include "attn_tma.cuh"
 
 using namespace prhs;
 
@@ -78,6 +80,11 @@ struct prhs_ctx {
   int last_batch = 0, last_layer_group = 1, last_nchunks = 1;
   // cuTensorMapEncodeTiled, resolved at run time (no link against libcuda); nullptr = no TMA path
   void* encode_tiled = nullptr;
+  // tensor maps of the gathered attention's K and V views (one row by 64 columns per box), kept
+  // from call to call: encoding one costs about a microsecond of host time
+  struct RowMap { const void* base; unsigned long long rows; CUtensorMap map; };
+  std::vector<RowMap> row_maps;
+  size_t row_map_next = 0;
   SetRef last_set{};                // what the last decode step attended over (for diagnostics)
   const int* last_seq_lens = nullptr;
   long long launches = 0;
@@ -213,6 +220,19 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
   return best;
 }
 
+// Split count for the scoring kernels: about 4096 key rows (1 MB) per CTA, several waves of CTAs
+// per launch.  Short CTAs finish at different times, so the SMs never run dry together: a grid of
+// one wave of long CTAs measured 3 to 5 % slower (the 32K-context layer at batch 8: 327 us against
+// 317 us; the ragged paged batch of 64: 747 us against 711 us).  A small batch gets at least two
+// CTAs per resident slot, but no CTA fewer than 256 rows.
+int score_splits(const prhs_ctx* c, int units, int max_t) {
+  const int slots = c->sm_count * 2;
+  int s = (max_t + 4095) / 4096;
+  const int fill = (2 * slots + units - 1) / std::max(units, 1);
+  s = std::max(s, std::min(fill, max_t / 256));
+  return std::max(1, std::min(s, kMaxSplits));
+}
+
 // `sched` != nullptr: a retrieval pass (the fp32 logits are written for the selection kernel);
 // nullptr: only the per-split log-sum-exp partials (the delta diagnostic).
 prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch, int max_t,
@@ -224,7 +244,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.scores = write_scores ? c->scores : nullptr;
   sp.ld = c->ld;
   sp.part_ml = c->part_ml;
-  sp.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_t);
+  sp.splits = score_splits(c, batch * c->cfg.num_kv_heads, max_t);
   sp.num_q_heads = c->cfg.num_q_heads;
   sp.group_size = c->gq;
   sp.need = need;
@@ -276,9 +296,40 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   return PRHS_OK;
 }
 
+// Tensor map of a K or V array viewed as [rows][128] bf16 with a box of ONE row by 64 columns and
+// the 128-byte swizzle: what a tile::gather4 copy of the gathered attention names rows in.
+// false if the driver cannot encode it.
+bool row_gather_map(prhs_ctx* c, const void* base, unsigned long long rows, CUtensorMap* out) {
+  for (const auto& m : c->row_maps)
+    if (m.base == base && m.rows == rows) { *out = m.map; return true; }
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  prhs_ctx::RowMap rm;
+  rm.base = base;
+  rm.rows = rows;
+  const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+  const cuuint64_t gstr[1] = {(cuuint64_t)kRowBytes};
+  const cuuint32_t box[2] = {64u, 1u};
+  const cuuint32_t estr[2] = {1u, 1u};
+  const CUresult cr = reinterpret_cast<EncodeFn>(c->encode_tiled)(
+      &rm.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return false;
+  *out = rm.map;
+  if (c->row_maps.size() < 32) {
+    c->row_maps.push_back(rm);
+  } else {
+    c->row_maps[c->row_map_next] = rm;
+    c->row_map_next = (c->row_map_next + 1) % c->row_maps.size();
+  }
+  return true;
+}
+
 prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
                         int idx_stride, const SetRef& fs, int max_count, int batch, void* out,
-                        float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st) {
+                        float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st, int max_rows) {
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.kv = kv;
@@ -311,8 +362,22 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
     gather_group_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   } else {
     dim3 grid(p.splits, c->cfg.num_q_heads, batch);
+    // rows by 16-byte cp.async copies; by TMA row gather only where the context asks for it
+    // (PRHS_CFG_TMA_GATHER: measured slower, kept for comparison)
+    alignas(64) CUtensorMap tmk, tmv;
+    bool have_maps = false;
+    unsigned long long rows_total = 0;
+    if (c->encode_tiled && (c->cfg.flags & PRHS_CFG_TMA_GATHER) && !(c->cfg.flags & PRHS_CFG_NO_TMA)) {
+      const bool paged = kv.page_table != nullptr;
+      rows_total = (unsigned long long)((paged ? kv.num_pages : batch) - 1) * (unsigned long long)(kv.stride_outer >> 7) +
+                   (unsigned long long)(c->cfg.num_kv_heads - 1) * (unsigned long long)(kv.stride_head >> 7) +
+                   (unsigned long long)(paged ? 16 : max_rows);
+      if (rows_total < (1ull << 31) - 1)
+        have_maps = row_gather_map(c, kv.k, rows_total, &tmk) && row_gather_map(c, kv.v, rows_total, &tmv);
+    }
     LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
-    gather_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
+    if (have_maps) gather_attn_tma_kernel<<<grid, kTThreads, kATSmemBytes, st>>>(tmk, tmv, p, (uint32_t)rows_total);
+    else gather_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   }
   PRHS_CUDA(c, cudaGetLastError());
   return PRHS_OK;
@@ -611,7 +676,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
   if (cfg->max_context > kMaxContext) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context above 2^20");
   if (cfg->max_k > 65536) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_k above 65536");
-  if (cfg->flags & ~PRHS_CFG_NO_TMA) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
+  if (cfg->flags & ~(PRHS_CFG_NO_TMA | PRHS_CFG_TMA_GATHER)) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
 
   prhs_ctx* c = new (std::nothrow) prhs_ctx();
   if (!c) return fail(nullptr, PRHS_ERR_OOM, "host allocation failed");
@@ -676,6 +741,16 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSRSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_attn_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kATSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_probe_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGPSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_probe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGPSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_probe_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGPSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_probe_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGPSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(dense_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess) {
@@ -798,7 +873,7 @@ prhs_status prhs_sparse_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
   return launch_attn(ctx, q, dv, idx, count, idx_stride, SetRef{}, idx_stride, batch, out, out_lse,
-                     nullptr, nullptr, as_stream(stream));
+                     nullptr, nullptr, as_stream(stream), max_t);
 }
 
 namespace {
@@ -924,6 +999,67 @@ prhs_status prhs_noalloc_check(void* stream, uint32_t* out_flags) {
   return PRHS_OK;
 }
 
+prhs_status prhs_gather_probe(prhs_ctx* ctx, int32_t variant, const prhs_kv_view* kv, const int32_t* idx,
+                              const int32_t* count, int32_t idx_stride, int32_t batch, void* stream) {
+  if (!ctx) return PRHS_ERR_INVALID_ARG;
+  if (!idx || !count) return fail(ctx, PRHS_ERR_INVALID_ARG, "NULL pointer");
+  if (idx_stride < 1) return fail(ctx, PRHS_ERR_INVALID_ARG, "idx_stride must be >= 1");
+  if (variant < 0 || variant > 3) return fail(ctx, PRHS_ERR_INVALID_ARG, "gather probe: variant must be 0..3");
+  KvDev dv;
+  int max_t;
+  prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
+  if (rc != PRHS_OK) return rc;
+  if (dv.page_table) return fail(ctx, PRHS_ERR_UNSUPPORTED, "gather probe: contiguous caches only");
+  cudaStream_t st = as_stream(stream);
+  GatherProbeParams p;
+  p.kv = dv;
+  p.idx = idx;
+  p.count = count;
+  p.idx_stride = idx_stride;
+  p.num_q_heads = ctx->cfg.num_q_heads;
+  p.group_size = ctx->gq;
+  p.splits = pick_splits(ctx, batch * ctx->cfg.num_q_heads, idx_stride);
+  p.flags = ctx->flags;
+  p.sink = reinterpret_cast<unsigned int*>(ctx->lse_c);      // any word of the context; never written
+  alignas(64) CUtensorMap tmk, tmv;
+  std::memset(&tmk, 0, sizeof tmk);
+  std::memset(&tmv, 0, sizeof tmv);
+  if (variant == 3) {
+    // K and V as [rows][128] bf16, a box of ONE row: a gather4 copy names four rows and brings 4 boxes
+    if (!ctx->encode_tiled) return fail(ctx, PRHS_ERR_UNSUPPORTED, "gather probe: the driver offers no tensor-map encoder");
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    const unsigned long long rows_total = (unsigned long long)(batch - 1) * (unsigned long long)(dv.stride_outer >> 7) +
+                                          (unsigned long long)(ctx->cfg.num_kv_heads - 1) * (unsigned long long)(dv.stride_head >> 7) +
+                                          (unsigned long long)max_t;
+    if (rows_total >= (1ull << 31)) return fail(ctx, PRHS_ERR_UNSUPPORTED, "gather probe: more than 2^31 rows");
+    const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows_total};
+    const cuuint64_t gstr[1] = {(cuuint64_t)kRowBytes};
+    const cuuint32_t box[2] = {(cuuint32_t)kHeadDim, 1u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    for (int i = 0; i < 2; ++i) {
+      const CUresult cr = reinterpret_cast<EncodeFn>(ctx->encode_tiled)(
+          i == 0 ? &tmk : &tmv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(i == 0 ? dv.k : dv.v),
+          gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (cr != CUDA_SUCCESS) return fail(ctx, PRHS_ERR_CUDA, "gather probe: cuTensorMapEncodeTiled failed");
+    }
+  }
+  const dim3 grid(p.splits, ctx->cfg.num_q_heads, batch);
+  {
+    LaunchScope ls(ctx, PRHS_KIND_MISC, st);
+    switch (variant) {
+      case 0: gather_probe_kernel<0><<<grid, kTThreads, kGPSmemBytes, st>>>(tmk, tmv, p); break;
+      case 1: gather_probe_kernel<1><<<grid, kTThreads, kGPSmemBytes, st>>>(tmk, tmv, p); break;
+      case 2: gather_probe_kernel<2><<<grid, kTThreads, kGPSmemBytes, st>>>(tmk, tmv, p); break;
+      default: gather_probe_kernel<3><<<grid, kTThreads, kGPSmemBytes, st>>>(tmk, tmv, p); break;
+    }
+  }
+  PRHS_CUDA(ctx, cudaGetLastError());
+  return PRHS_OK;
+}
+
 prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, int32_t batch,
                                    void* out, float* out_lse, void* stream) {
   if (!ctx) return PRHS_ERR_INVALID_ARG;
@@ -933,7 +1069,7 @@ prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_v
   prhs_status rc = check_view(ctx, kv, batch, &dv, &max_t);
   if (rc != PRHS_OK) return rc;
   return launch_attn(ctx, q, dv, nullptr, nullptr, 0, SetRef{}, max_t, batch, out, out_lse, nullptr,
-                     nullptr, as_stream(stream));
+                     nullptr, as_stream(stream), max_t);
 }
 
 prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,
@@ -1013,7 +1149,7 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
   ctx->last_seq_lens = dv.seq_lens;
   ctx->last_batch = batch;
   return launch_attn(ctx, q, dv, nullptr, nullptr, 0, fs, ctx->idx_cap, batch, out, ctx->lse_c,
-                     want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr, st);
+                     want_delta ? ctx->lse_full : nullptr, want_delta ? out_delta : nullptr, st, max_t);
 }
 
 namespace {
@@ -1141,7 +1277,7 @@ prhs_status prhs_delta(prhs_ctx* ctx, const void* q, const prhs_kv_view* kv, con
   }
   PRHS_CUDA(ctx, cudaGetLastError());
   return launch_attn(ctx, q, dv, idx, count, idx_stride, SetRef{}, idx_stride, batch, ctx->scratch_out,
-                     ctx->lse_c, ctx->lse_full, out_delta, st);
+                     ctx->lse_c, ctx->lse_full, out_delta, st, max_t);
 }
 
 prhs_status prhs_get_index_set(prhs_ctx* ctx, int32_t batch, int32_t* host_idx, int32_t* host_count,

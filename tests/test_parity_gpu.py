@@ -470,6 +470,92 @@ def test_score_ring_and_tma_logits_agree(cuda_device):
     assert torch.allclose(res[0][1], res[1][1], atol=1e-4)
 
 
+# ------------------------------------------ gathered attention with rows by TMA gather (an option)
+@pytest.mark.parametrize("paged", [False, True])
+def test_tma_gather_attention_small_every_unit(cuda_device, paged):
+    # PRHS_CFG_TMA_GATHER: the same attention with tile::gather4 copies instead of cp.async (off by
+    # default, it measured slower); ragged tails, empty middle sets, out-of-tensor filler rows
+    w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=3, q_heads=8, kv_heads=2, context=2900,
+              min_context=200 if paged else 0, page_size=16 if paged else 0, seed=31, psaw_layer_start=2)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged,
+                               ctx_over=dict(flags=P.PRHS_CFG_TMA_GATHER))
+    assert st["checked"] == 2 * 4 * w.batch * w.q_heads
+
+
+def test_tma_gather_attention_given_sets_and_bad_index(cuda_device):
+    w = small(q_heads=8, kv_heads=4, context=3000, seed=32)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = torch.tensor([2999, 1234], dtype=torch.int32)
+    g = np.random.default_rng(32)
+    cap = 700
+    idx = torch.full((w.batch, w.q_heads, cap), -7, dtype=torch.int32)
+    cnt = torch.zeros(w.batch, w.q_heads, dtype=torch.int32)
+    sets = {}
+    sizes = [0, 1, 15, 16, 17, 255, 256, 257, 511, 640, 700, 33, 300, 64, 129, 5]
+    for b, h in all_units(w):
+        n = min(sizes[(b * w.q_heads + h) % len(sizes)], int(t_host[b]))
+        C = np.sort(g.permutation(int(t_host[b]))[:n])
+        sets[(b, h)] = C
+        idx[b, h, :n] = torch.from_numpy(C.astype(np.int32))
+        cnt[b, h] = n
+    ctx = H.make_ctx(w, flags=P.PRHS_CFG_TMA_GATHER)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    ctx.sparse_decode_attn(q, view, idx.to(cuda_device), cnt.to(cuda_device), w.batch, out, lse)
+    assert ctx.check() == 0
+    y, ls, qh = H.np32(out), H.np32(lse), H.np32(q)
+    for (b, h), C in sets.items():
+        y_ref, lse_ref = O.attn_over_set(qh[b, h], H.np32(k[b, h // 2]), H.np32(v[b, h // 2]), C)
+        assert np.max(np.abs(y[b, h] - y_ref)) <= H.Y_TOL
+        assert (ls[b, h] == -math.inf) if len(C) == 0 else abs(ls[b, h] - lse_ref) <= 1e-4
+    bad = idx.clone()
+    bad[1, 2, 1] = 10 ** 6                                  # skipped (a zero-filled row, masked) and flagged
+    ctx.sparse_decode_attn(q, view, bad.to(cuda_device), cnt.to(cuda_device), w.batch, out, lse)
+    with pytest.raises(P.PrhsError) as e:
+        ctx.check()
+    assert e.value.status == 7
+    C = np.delete(sets[(1, 2)], 1)
+    y_ref, _ = O.attn_over_set(qh[1, 2], H.np32(k[1, 1]), H.np32(v[1, 1]), C)
+    assert np.max(np.abs(H.np32(out)[1, 2] - y_ref)) <= H.Y_TOL
+    ctx.close()
+
+
+# ----------------------------------------------------------- measurement support: the gather probe
+def test_gather_probe_variants_run_clean(cuda_device):
+    # the bare row gather behind `python -m paper_2602_08329_b200.gather_ceiling`: every copy
+    # mechanism over real index lists (ragged tails, an empty list), no anomaly; then a list
+    # with an out-of-range entry, which is replaced and flagged, not read
+    w = small(batch=3, q_heads=8, kv_heads=2, context=4000, seed=29)
+    k, v = W.make_kv(w, cuda_device)
+    t_dev = W.seq_lens_at(w, 0).to(cuda_device)
+    view = P.make_view(k, v, t_dev, max_seq_len=w.capacity)
+    g = np.random.default_rng(29)
+    cap = 900
+    idx = torch.zeros(w.batch, w.q_heads, cap, dtype=torch.int32)
+    cnt = torch.zeros(w.batch, w.q_heads, dtype=torch.int32)
+    for b, h in all_units(w):
+        n = 0 if (b, h) == (1, 1) else int(g.integers(1, cap + 1))
+        idx[b, h, :n] = torch.from_numpy(np.sort(g.permutation(4000)[:n]).astype(np.int32))
+        cnt[b, h] = n
+    idx, cnt = idx.to(cuda_device), cnt.to(cuda_device)
+    ctx = H.make_ctx(w)
+    for variant in range(4):
+        ctx.gather_probe(variant, view, idx, cnt, w.batch)
+        assert ctx.check() == 0, variant
+    bad = idx.clone()
+    bad[2, 3, 0] = 10 ** 6
+    for variant in range(4):
+        ctx.gather_probe(variant, view, bad, cnt, w.batch)
+        with pytest.raises(P.PrhsError) as e:
+            ctx.check()
+        assert e.value.status == 7, variant
+    with pytest.raises(P.PrhsError):
+        ctx.gather_probe(4, view, idx, cnt, w.batch)
+    ctx.close()
+
+
 # ------------------------------------------------------------------- host-buffer entry point
 @pytest.mark.parametrize("pinned", [True, False])
 def test_decode_step_host_buffers(cuda_device, pinned):
