@@ -74,6 +74,11 @@ struct AttnParams {
   const float* lse_full;    // [B][Hq] or nullptr
   float* out_delta;         // [B][Hq] or nullptr: 1 - exp(lse - lse_full)
   uint32_t* flags;
+  // cosine-gated steps launch the attention twice, for the heads that share (beside the retrieval
+  // of the others) and for the heads that retrieved (after it): need_mode 1 = only units with
+  // need[unit] == 0, 2 = only units with need[unit] != 0, 0 = every unit
+  const int* need;
+  int need_mode;
 };
 
 // ---------------------------------------------------------------- cp.async helpers
@@ -193,6 +198,7 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   extern __shared__ __align__(128) unsigned char g_smem[];
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int unit = b * p.num_q_heads + h;
+  if (p.need_mode != 0 && ((__ldg(p.need + unit) != 0) != (p.need_mode == 2))) return;   // the other launch's unit
   const int kvh = h / p.group_size;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;

@@ -53,6 +53,7 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   __shared__ int sh_abort;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int unit = b * p.num_q_heads + h;
+  if (p.need_mode != 0 && ((__ldg(p.need + unit) != 0) != (p.need_mode == 2))) return;   // the other launch's unit
   const int kvh = h / p.group_size;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, tg = lane & 3;

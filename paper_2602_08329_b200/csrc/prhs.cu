@@ -80,6 +80,10 @@ struct prhs_ctx {
   int last_batch = 0, last_layer_group = 1, last_nchunks = 1;
   // cuTensorMapEncodeTiled, resolved at run time (no link against libcuda); nullptr = no TMA path
   void* encode_tiled = nullptr;
+  // cosine-gated steps run the attention of the heads that share on this stream, beside the
+  // scoring and selection of the heads that retrieve on the caller's (Fig. 6: two branches)
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   // tensor maps of the gathered attention's K and V views (one row by 64 columns per box), kept
   // from call to call: encoding one costs about a microsecond of host time
   struct RowMap { const void* base; unsigned long long rows; CUtensorMap map; };
@@ -329,7 +333,8 @@ bool row_gather_map(prhs_ctx* c, const void* base, unsigned long long rows, CUte
 
 prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* idx, const int* count,
                         int idx_stride, const SetRef& fs, int max_count, int batch, void* out,
-                        float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st, int max_rows) {
+                        float* out_lse, const float* lse_full, float* out_delta, cudaStream_t st, int max_rows,
+                        const int* need = nullptr, int need_mode = 0) {
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.kv = kv;
@@ -348,6 +353,8 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
   p.lse_full = lse_full;
   p.out_delta = lse_full ? out_delta : nullptr;
   p.flags = c->flags;
+  p.need = need;
+  p.need_mode = need ? need_mode : 0;
   if (!idx && !fs.star) {
     // dense baseline: one CTA column per KV head, the group's heads share the K/V stream
     p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
@@ -759,6 +766,9 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     if (e == cudaSuccess && nb > 0) c->attn_ctas_per_sm = nb;
   }
 
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
   const size_t U = units_max(c), G = c->num_groups;
   if (e == cudaSuccess) e = dev_alloc(&c->scores, U * c->ld);
   if (e == cudaSuccess) e = dev_alloc(&c->part_ml, U * std::max(c->max_chunks, kMaxSplits));
@@ -820,6 +830,9 @@ prhs_status prhs_destroy(prhs_ctx* c) {
     cudaEventDestroy(r.a);
     cudaEventDestroy(r.b);
   }
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
   delete c;
   return PRHS_OK;
 }
@@ -974,6 +987,8 @@ prhs_status prhs_sparse_decode_attn_noalloc(const void* q, const prhs_kv_view* k
   p.lse_full = nullptr;
   p.out_delta = nullptr;
   p.flags = flag_word;
+  p.need = nullptr;
+  p.need_mode = 0;
   gather_attn_mma_kernel<<<dim3(splits, num_q_heads, batch), kTThreads, kTSmemBytes, st>>>(p);
   PRHS_CUDA(nullptr, cudaGetLastError());
   return PRHS_OK;
@@ -1112,6 +1127,35 @@ prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const p
       }
       PRHS_CUDA(ctx, cudaGetLastError());
       ctx->gate_step[g] = step;
+      if (!want_delta) {
+        // The two branches of Fig. 6.  The heads that share attend over their cached sets on a
+        // second stream while the heads that retrieve are scored and selected on the caller's;
+        // the attention of the retrieving heads follows the selection, and the caller's stream
+        // continues when both branches are done (events; nothing waits on the device).  The
+        // diagnostic (delta) needs every head's full log-sum-exp first: no second branch then.
+        SetRef fs{};
+        rc = pick_middle(ctx, layer, step, sched, &fs);
+        if (rc != PRHS_OK) return rc;
+        ctx->last_set = fs;
+        ctx->last_seq_lens = dv.seq_lens;
+        ctx->last_batch = batch;
+        PRHS_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+        PRHS_CUDA(ctx, cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0));
+        rc = launch_attn(ctx, q, dv, nullptr, nullptr, 0, fs, ctx->idx_cap, batch, out, ctx->lse_c, nullptr, nullptr,
+                         ctx->side_stream, max_t, need, 1);
+        if (rc == PRHS_OK) {
+          PRHS_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side_stream));
+          rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, need, slot,
+                            false, st);
+        }
+        if (rc == PRHS_OK)
+          rc = launch_attn(ctx, q, dv, nullptr, nullptr, 0, fs, ctx->idx_cap, batch, out, ctx->lse_c, nullptr, nullptr,
+                           st, max_t, need, 2);
+        // the side branch joins even after a failed launch, so that a capture in progress stays well formed
+        const cudaError_t je = cudaStreamWaitEvent(st, ctx->ev_join, 0);
+        if (rc == PRHS_OK && je != cudaSuccess) return fail(ctx, PRHS_ERR_CUDA, cudaGetErrorString(je));
+        return rc;
+      }
       rc = do_retrieval(ctx, layer, step, q, dv, max_t, sched, batch, nullptr, nullptr, nullptr, need, slot,
                         want_delta, st);
       if (rc != PRHS_OK) return rc;

@@ -5,6 +5,7 @@
     python -m paper_2602_08329_b200.operator_latency --configs  # the benchmark's C2..C5 shapes
     python -m paper_2602_08329_b200.operator_latency --configs --group-sets   # one set per KV head (variant)
     python -m paper_2602_08329_b200.operator_latency --configs --summary  # JSON: time, bytes, roofline per layer-step
+    python -m paper_2602_08329_b200.operator_latency --gated              # cosine-gated schedule vs fixed at equal rho-hat
 
 The paper (Sec. 5.4, Table 3) times one attention layer of LLaMA-2-7B-Chat (32 MHA heads,
 head_dim 128) in decode at batch 8 / 16 and 1k-4k cached tokens, token sparsity 1/8, block
@@ -333,6 +334,77 @@ def config_summary(w: W.Workload, dev, reps: int = 7, copies: int = 4, group_set
     return res
 
 
+def gated_summary(w: W.Workload, dev, tau: float = 0.8, sigma: float = 0.7, s: int = 16, blocks: int = 2,
+                  copies: int = 2, reps: int = 5) -> dict:
+    """The cosine-gated schedule (Eq. 9) timed against the fixed schedule at the same retrieval ratio.
+
+    `copies` independent caches of the (single-layer) workload decode `blocks` blocks of `s` steps
+    each, round-robin, with sim_threshold = tau and a query drift sigma large enough that a share
+    of the heads fails the similarity test and retrieves inside the block.  The whole run is
+    captured into a CUDA graph and replayed (the decisions depend only on the queries, so every
+    replay takes the same ones); rho-hat is the fraction of (step, head) pairs that retrieved.  The
+    fixed schedule is then timed the same way with the refresh interval nearest to 1 / rho-hat.
+    """
+    T = blocks * s
+    ws = w.scaled(layers=copies, steps=T, layer_group=1, sigma=sigma, refresh=s)
+    kv, table = _make_caches(ws, dev)
+    q = W.make_queries(ws, dev)
+    B, Hq = ws.batch, ws.q_heads
+    out = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    lens = [W.seq_lens_at(ws, n).to(dev) for n in range(T)]
+    views = [[P.make_view(kv[l][0], kv[l][1], lens[n], page_table=table, max_seq_len=ws.capacity)
+              for n in range(T)] for l in range(copies)]
+    order = [(l, n) for n in range(T) for l in range(copies)]
+    stream = torch.cuda.current_stream()
+
+    def run(sim_threshold, refresh):
+        ctx = P.Context(copies, B, Hq, ws.kv_heads, ws.capacity, ws.top_k, ws.window, ws.sinks,
+                        max_dilate_r=ws.dilate_r, page_size=ws.page_size,
+                        max_block_sets=refresh if sim_threshold is not None else 1)
+        sched = P.make_schedule(ws.top_k, ws.window, ws.sinks, refresh_interval=refresh, dilate_r=ws.dilate_r,
+                                sim_threshold=-1.0 if sim_threshold is None else sim_threshold)
+        retrieved = 0
+        for l, n in order:                       # direct pass: warms up and counts the retrievals
+            ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out)
+            if sim_threshold is not None:
+                need, _ = ctx.get_gate(l, B)
+                retrieved += int(need.sum())
+            elif n % refresh == 0:
+                retrieved += B * Hq
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                for l, n in order:
+                    ctx.decode_step(l, n, sched, q[l, n], views[l][n], B, out, stream=torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3 / len(order))
+        assert ctx.check() & ~P.PRHS_FLAG_SELECT_FALLBACK == 0
+        ctx.close()
+        return statistics.median(ts), retrieved / (len(order) * B * Hq)
+
+    gated_us, rho = run(tau, s)
+    s_eq = max(1, round(1.0 / max(rho, 1e-6)))
+    while T % s_eq:                              # whole blocks of the fixed schedule in the same run
+        s_eq -= 1
+    fixed_us, rho_fixed = run(None, s_eq)
+    del kv, views
+    torch.cuda.empty_cache()
+    return {"workload": ws.name, "batch": B, "tau": tau, "sigma": sigma, "block": s, "steps": T, "caches": copies,
+            "rho_hat": rho, "gated_us_per_step": gated_us,
+            "fixed_refresh_interval": s_eq, "fixed_rho_hat": rho_fixed, "fixed_us_per_step": fixed_us,
+            "gated_over_fixed": gated_us / fixed_us}
+
+
 def configs_summary(dev, group_sets=False, only=None, batch=0):
     import json
     for w in (W.C2_LLAMA2_7B, W.C3_MISTRAL, W.C4_LLAMA3_128K, W.C5_SERVING):
@@ -417,6 +489,10 @@ def main():
     ap.add_argument("--summary", action="store_true",
                     help="with --configs: one JSON line per configuration, timed as its own schedule runs it (layer "
                          "groups included): time, bytes and roofline fractions per layer-step")
+    ap.add_argument("--gated", action="store_true",
+                    help="the cosine-gated schedule (tau 0.8) on the c2 shape against the fixed schedule at the same "
+                         "retrieval ratio: one JSON line per query drift sigma")
+    ap.add_argument("--sigmas", default="0.6,0.7,0.75", help="with --gated: query drifts to time")
     ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
     ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
     ap.add_argument("--group-sets", action="store_true",
@@ -426,7 +502,14 @@ def main():
         raise SystemExit("needs a CUDA device")
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
-    if args.configs and args.summary:
+    if args.gated:
+        import json
+        w = W.CONFIGS[args.only] if args.only else W.C2_LLAMA2_7B
+        if args.batch:
+            w = w.scaled(batch=args.batch)
+        for sg in args.sigmas.split(","):
+            print(json.dumps(gated_summary(w, dev, sigma=float(sg))), flush=True)
+    elif args.configs and args.summary:
         configs_summary(dev, args.group_sets, args.only, args.batch)
     elif args.configs:
         (configs_graph if args.graph else configs)(dev, args.group_sets, args.only, args.batch)

@@ -311,6 +311,57 @@ def test_schedule_with_cosine_gate(cuda_device, tau, sigma):
         assert 3 * leaders_heads < st["retrievals"] < 9 * leaders_heads    # a real mix
 
 
+@pytest.mark.parametrize("tau,sigma,paged", [(0.8, 0.7, False), (0.9, 0.45, True), (0.8, 0.3, False), (0.99, 1.5, False)])
+def test_cosine_gate_two_branches(cuda_device, tau, sigma, paged):
+    # without the diagnostic a gated step runs as two branches: the attention of the heads that
+    # share on a second stream, beside the scoring and selection of the heads that retrieve, whose
+    # attention follows (Fig. 6); a real mix, nearly all sharing, all retrieving
+    w = small(layers=4, layer_group=2, steps=9, refresh=4, batch=3, q_heads=8, kv_heads=2, context=2500, seed=27,
+              min_context=600 if paged else 0, page_size=16 if paged else 0, sigma=sigma, sim_threshold=tau)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, want_delta=False)
+    assert st["checked"] == 4 * 9 * w.batch * w.q_heads
+    leaders_heads = 2 * w.batch * w.q_heads
+    if sigma == 0.7:
+        assert 3 * leaders_heads < st["retrievals"] < 9 * leaders_heads
+    if sigma == 1.5:
+        assert st["retrievals"] == 9 * leaders_heads           # no query is that similar: every head retrieves every step
+
+
+def test_cosine_gate_two_branches_in_a_cuda_graph(cuda_device):
+    # the forked branch is captured with the step and joins it: replays equal the direct calls
+    w = small(steps=8, refresh=4, batch=3, q_heads=8, kv_heads=2, context=2400, seed=28, sigma=0.7, sim_threshold=0.8)
+    k, v = W.make_kv(w, cuda_device)
+    q_all = W.make_queries(w, cuda_device)[0]
+    sched = H.make_sched(w, cuda_device)
+    views = [P.make_view(k, v, W.seq_lens_at(w, n).to(cuda_device), max_seq_len=w.capacity) for n in range(w.steps)]
+    out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    ctx = H.make_ctx(w)
+    direct, needs = [], []
+    for n in range(w.steps):
+        ctx.decode_step(0, n, sched, q_all[n], views[n], w.batch, out)
+        direct.append(out.clone())
+        needs.append(ctx.get_gate(0, w.batch)[0].clone())
+    assert ctx.check() == 0
+    assert 0 < int(torch.stack(needs)[1:4].sum()) < 3 * w.batch * w.q_heads          # a mix inside the block
+    side = torch.cuda.Stream()
+    outs = [torch.empty_like(out) for _ in range(w.steps)]
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for n in range(w.steps):
+                ctx.decode_step(0, n, sched, q_all[n], views[n], w.batch, outs[n], stream=torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for n in range(w.steps):
+            assert torch.equal(outs[n], direct[n]), f"step {n}"
+    assert ctx.check() == 0
+    ctx.close()
+
+
 def test_cosine_gate_gqa_paged_with_window(cuda_device):
     w = small(layers=2, layer_group=1, steps=6, refresh=3, batch=3, q_heads=8, kv_heads=1, context=2100,
               min_context=500, page_size=16, top_k=0, k_frac=0.03, seed=16, sigma=0.6, sim_threshold=0.85,
