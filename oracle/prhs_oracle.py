@@ -104,9 +104,8 @@ def topk_middle(a: np.ndarray, t: int, sinks: int, window: int, k: int, psaw_lo:
 
     With a sliding-window start `psaw_lo` (Eq. 11) the candidates are [max(S0, P), t-W).
 
-    Returned in descending-logit order p_1, p_2, ... (Sec. 4.1: "sorted and selected in
-    descending order of attention weight"); equal logits are ordered by lower position
-    first.  Softmax is monotone in the logit, so ranking logits ranks attention weights.
+    Returned in descending-logit order p_1, p_2, ... (Sec. 4.1 ranks the winners by falling
+    attention weight); equal logits are ordered by lower position first.  Softmax is monotone in the logit, so ranking logits ranks attention weights.
     The ranking uses the float32-rounded logits (see module docstring).
     """
     lo, hi = max(sinks, psaw_lo), t - window
@@ -286,8 +285,8 @@ class PrhsOracle:
         the most recent earlier step of the block whose query has cosine similarity > tau,
         and retrieves a new set if there is none.
     A retrieval stores S* and its dilation S^ (Eq. 10).  The retrieving call attends over C
-    built from the undilated S* unless `dilate_anchor` is set (dilation costs budget "during
-    sharing", Sec. 5.2.2); every sharer attends over C built from S^ (Def. 3.2) with its own
+    built from the undilated S* unless `dilate_anchor` is set (Sec. 5.2.2 counts the budget
+    of dilation for the sharing steps); every sharer attends over C built from S^ (Def. 3.2) with its own
     q, K, V.  The other layers of a group follow the decision and the set of its first layer.
 
     `override_ref` / `override_s_star` (per (b, h)) let a test substitute a decision or a

@@ -228,8 +228,10 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
 // per launch.  Short CTAs finish at different times, so the SMs never run dry together: a grid of
 // one wave of long CTAs measured 3 to 5 % slower (the 32K-context layer at batch 8: 327 us against
 // 317 us; the ragged paged batch of 64: 747 us against 711 us).  A small batch gets at least two
-// CTAs per resident slot, but no CTA fewer than 256 rows.
+// CTAs per resident slot, but no CTA fewer than 256 rows.  Contexts of a few thousand keys are
+// bound by latency, not by the stream: they keep the single wave.
 int score_splits(const prhs_ctx* c, int units, int max_t) {
+  if (max_t <= 8192) return pick_splits(c, units, max_t);      // short contexts are bound by latency: one wave
   const int slots = c->sm_count * 2;
   int s = (max_t + 4095) / 4096;
   const int fill = (2 * slots + units - 1) / std::max(units, 1);
