@@ -194,6 +194,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+template <int kValue>
+struct SlotC { static constexpr int value = kValue; };    // a ring slot known at compile time
+
 __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p) {
   extern __shared__ __align__(128) unsigned char g_smem[];
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -280,11 +283,20 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   pg1 = page_of(pos1);
   int pos2 = list_pos(2);
 
-  const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
-  const uint32_t dst_tile = (lane < 16 ? 0u : (uint32_t)kTTileBytes);
-  unsigned long long vmask = 0ull;     // 16 validity bits per ring slot
+  // The copy of row r of a stage: lane p (0-15: K row, 16-31: V row) fills 16-byte position p of the
+  // row with the source chunk p ^ (r & 7), which is the XOR swizzle ldmatrix reads.  Written this
+  // way the destination of a lane is the same in every row and the eight source offsets are
+  // loop invariants: a row costs a shuffle, one multiply-add and the copy.
+  const __nv_bfloat16* srcx[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) srcx[k] = (lane < 16 ? p.kv.k : p.kv.v) + ((((uint32_t)lane & 15u) ^ (uint32_t)k) << 3);
+  const uint32_t dst_lane = (lane < 16 ? 0u : (uint32_t)kTTileBytes) + (((uint32_t)lane & 15u) << 4);
+  uint32_t vmv[kTStages];              // 16 validity bits per ring slot (slots are compile-time below)
+#pragma unroll
+  for (int k = 0; k < kTStages; ++k) vmv[k] = 0u;
 
-  auto issue = [&](int j) {
+  auto issue = [&](int j, auto slot_c) {
+    constexpr int kSlot = decltype(slot_c)::value;
     if (j < nstages) {
       if (j > 0 && (j & 1) == 0) {     // step the row-id pipeline
         const int grp = j >> 1;
@@ -295,43 +307,44 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
         pg1 = page_of(pos1);
         pos2 = list_pos(grp + 2);
       }
-      const int slot_i = j % kTStages;
-      const uint32_t slot = ring + (uint32_t)slot_i * kTStageBytes + dst_tile;
+      // the 16 entries of this stage, brought to lanes 0-15 (odd stages hold them in lanes 16-31)
+      const uint32_t rid_cur = __shfl_sync(0xffffffffu, rid_a, (lane + ((j & 1) << 4)) & 31);
+      const uint32_t slot = ring + (uint32_t)kSlot * kTStageBytes + dst_lane;
       const uint32_t vm = (valid_a >> ((j & 1) * kTStageRows)) & 0xffffu;
       if (vm == 0xffffu) {             // the common case: 16 real rows
 #pragma unroll
         for (int r = 0; r < kTStageRows; ++r) {
-          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
-          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
-          cp_async_16_full(dst, src_base + (size_t)rid * kHeadDim);
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_cur, r);
+          cp_async_16_full(slot + r * kRowBytes, srcx[r & 7] + (size_t)rid * kHeadDim);
         }
       } else {
 #pragma unroll
         for (int r = 0; r < kTStageRows; ++r) {
-          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
-          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
-          cp_async_16(dst, src_base + (size_t)rid * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_cur, r);
+          cp_async_16(slot + r * kRowBytes, srcx[r & 7] + (size_t)rid * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
         }
       }
-      vmask = (vmask & ~(0xffffull << (16 * slot_i))) | ((unsigned long long)vm << (16 * slot_i));
+      vmv[kSlot] = vm;
     }
     cp_async_commit();
   };
 
-#pragma unroll
-  for (int j = 0; j < kTStages - 1; ++j) issue(j);
+  issue(0, SlotC<0>{});
+  issue(1, SlotC<1>{});
+  static_assert(kTStages == 3, "the stage loop below is unrolled over three ring slots");
 
   const float sc = kScale * kLog2e;
   // ldmatrix lane roles
   const int lm_mi = lane >> 3, lm_r = lane & 7;
   const int vrow = (lm_mi & 1) * 8 + lm_r;
-  for (int i = 0; i < nstages; ++i) {
+  // One stage: wait for its copies, refill the slot two stages ahead, S = Q K^T, softmax, O += P V.
+  auto stage = [&](int i, auto slot_c) {
+    constexpr int kSlot = decltype(slot_c)::value;
     cp_async_wait<kTStages - 2>();
     __syncwarp();
-    const int slot_i = i % kTStages;
-    const uint32_t vm = (uint32_t)(vmask >> (16 * slot_i)) & 0xffffu;
-    issue(i + kTStages - 1);
-    const uint32_t kt = ring + (uint32_t)slot_i * kTStageBytes;
+    const uint32_t vm = vmv[kSlot];
+    issue(i + kTStages - 1, SlotC<(kSlot + kTStages - 1) % kTStages>{});
+    const uint32_t kt = ring + (uint32_t)kSlot * kTStageBytes;
     const uint32_t vt = kt + kTTileBytes;
     // ---- S = Q K^T : all K fragments first, then the two accumulator chains interleaved
     uint32_t bk[2][4][4];
@@ -397,6 +410,16 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
         mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[np - 4][2], bv[np - 4][3]);
       }
     }
+  };
+  {
+    int i = 0;
+    for (; i + 2 < nstages; i += 3) {
+      stage(i, SlotC<0>{});
+      stage(i + 1, SlotC<1>{});
+      stage(i + 2, SlotC<2>{});
+    }
+    if (i < nstages) stage(i, SlotC<0>{});
+    if (i + 1 < nstages) stage(i + 1, SlotC<1>{});
   }
   cp_async_wait<0>();
   l += __shfl_xor_sync(0xffffffffu, l, 1);
