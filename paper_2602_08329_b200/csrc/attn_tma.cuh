@@ -89,10 +89,10 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
       aq2[ks] = g == 0 ? __ldg(q32 + ks * 8 + 4 + tg) : 0u;
     }
   }
-  float o[16][2];
+  // O^T += V^T P^T as in gather_attn_mma_kernel: eight 16 x 8 tiles whose column 0 is live
+  float o[8][4];
 #pragma unroll
-  for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; }
-  float z0 = 0.f, z1 = 0.f;            // accumulator rows 8..15: always zero
+  for (int mt = 0; mt < 8; ++mt) { o[mt][0] = 0.f; o[mt][1] = 0.f; o[mt][2] = 0.f; o[mt][3] = 0.f; }
   float m = -INFINITY, l = 0.f, lt = 0.f;
 
   // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane (as in
@@ -200,12 +200,13 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
       }
     }
     float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    float zq[2][2] = {{0.f, 0.f}, {0.f, 0.f}};      // dead accumulator rows, private to each chain
 #pragma unroll
     for (int pp = 0; pp < 4; ++pp) {
-      mma_bf16_row0(s[0][0], s[0][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[0][pp][0], bk[0][pp][1]);
-      mma_bf16_row0(s[1][0], s[1][1], z0, z1, aq0[2 * pp], aq2[2 * pp], bk[1][pp][0], bk[1][pp][1]);
-      mma_bf16_row0(s[0][0], s[0][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[0][pp][2], bk[0][pp][3]);
-      mma_bf16_row0(s[1][0], s[1][1], z0, z1, aq0[2 * pp + 1], aq2[2 * pp + 1], bk[1][pp][2], bk[1][pp][3]);
+      mma_bf16_row0(s[0][0], s[0][1], zq[0][0], zq[0][1], aq0[2 * pp], aq2[2 * pp], bk[0][pp][0], bk[0][pp][1]);
+      mma_bf16_row0(s[1][0], s[1][1], zq[1][0], zq[1][1], aq0[2 * pp], aq2[2 * pp], bk[1][pp][0], bk[1][pp][1]);
+      mma_bf16_row0(s[0][0], s[0][1], zq[0][0], zq[0][1], aq0[2 * pp + 1], aq2[2 * pp + 1], bk[0][pp][2], bk[0][pp][3]);
+      mma_bf16_row0(s[1][0], s[1][1], zq[1][0], zq[1][1], aq0[2 * pp + 1], aq2[2 * pp + 1], bk[1][pp][2], bk[1][pp][3]);
     }
     // the first half of the V fragments, fetched under the softmax arithmetic
     auto v_addr = [&](int np) -> uint32_t {
@@ -233,26 +234,21 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
       l *= corr;
       lt *= corr;
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+      for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= corr; o[mt][1] *= corr; o[mt][2] *= corr; o[mt][3] *= corr; }
     }
     if (m != -INFINITY) {              // warp-uniform; false only while every row so far was invalid
       const float p0 = exp2f(s0 - m), p1 = exp2f(s1 - m), p2 = exp2f(s2 - m), p3 = exp2f(s3 - m);
       l += (p0 + p1) + (p2 + p3);
       const uint32_t ap0 = pack_bf16x2(p0, p1), ap2 = pack_bf16x2(p2, p3);
       lt += (bf_lo(ap0) + bf_hi(ap0)) + (bf_lo(ap2) + bf_hi(ap2));
-      // ---- O += P V
+      // ---- O^T += V^T P^T
 #pragma unroll
-      for (int np = 0; np < 4; ++np) {
-        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[np][0], bv[np][1]);
-        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[np][2], bv[np][3]);
-      }
+      for (int mt = 0; mt < 4; ++mt) mma_bf16_full(o[mt], bv[mt][0], bv[mt][2], bv[mt][1], bv[mt][3], ap0, ap2);
 #pragma unroll
       for (int np = 4; np < 8; ++np) ldmatrix_x4_trans(bv[np - 4], v_addr(np));
 #pragma unroll
-      for (int np = 4; np < 8; ++np) {
-        mma_bf16_row0(o[2 * np][0], o[2 * np][1], z0, z1, ap0, ap2, bv[np - 4][0], bv[np - 4][1]);
-        mma_bf16_row0(o[2 * np + 1][0], o[2 * np + 1][1], z0, z1, ap0, ap2, bv[np - 4][2], bv[np - 4][3]);
-      }
+      for (int mt = 4; mt < 8; ++mt)
+        mma_bf16_full(o[mt], bv[mt - 4][0], bv[mt - 4][2], bv[mt - 4][1], bv[mt - 4][3], ap0, ap2);
     }
   }
   l += __shfl_xor_sync(0xffffffffu, l, 1);
@@ -260,14 +256,16 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   lt += __shfl_xor_sync(0xffffffffu, lt, 1);
   lt += __shfl_xor_sync(0xffffffffu, lt, 2);
 
-  // ---- combine the warps of this CTA (lanes 0-3 hold row 0: columns 8*nt + 2*tg, +1)
+  // ---- combine the warps of this CTA (lanes with tg == 0 hold columns 16*mt + g and 16*mt + g + 8)
   __shared__ __align__(16) float sm_o[kTWarps][kHeadDim];       // written as float2
   __shared__ float sm_m[kTWarps], sm_l[kTWarps], sm_lt[kTWarps];
   __shared__ bool is_last;
-  if (g == 0) {
+  if (tg == 0) {
 #pragma unroll
-    for (int nt = 0; nt < 16; ++nt)
-      *reinterpret_cast<float2*>(&sm_o[warp][nt * 8 + 2 * tg]) = make_float2(o[nt][0], o[nt][1]);
+    for (int mt = 0; mt < 8; ++mt) {
+      sm_o[warp][16 * mt + g] = o[mt][0];
+      sm_o[warp][16 * mt + g + 8] = o[mt][2];
+    }
   }
   if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; sm_lt[warp] = lt; }
   __syncthreads();
