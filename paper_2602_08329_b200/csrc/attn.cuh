@@ -104,10 +104,38 @@ struct ListDesc {
   int count;
 };
 
-// Per-warp set-up of the list descriptor (all 32 lanes call it).  In fused mode the bounds of
-// M inside [vis_lo, wlo) are found by looking at its two ends: dilation can push at most r
-// entries below S0 or into the window; a longer overlap (a sliding window start that moved
-// past many entries, a schedule change inside a block) falls back to a full scan.
+// Entry j of a unit's list, unchecked: for a stored middle entry this is a load whose result the
+// caller must not look at before it needs it (the row-id pipeline issues it a step ahead).
+__device__ __forceinline__ int list_entry(const ListDesc& ld, int j, int end) {
+  if (j >= end) return -1;
+  if (ld.fused) {
+    if (j < ld.s0) return j;
+    if (j < ld.s0 + ld.nmid) return __ldg(ld.list + ld.lo + (j - ld.s0));
+    return ld.wlo + (j - ld.s0 - ld.nmid);
+  }
+  return ld.list ? __ldg(ld.list + j) : j;
+}
+
+// The entry checked (this consumes the load): the position if it is a real row of the sequence,
+// else -1.  A stored middle entry that has moved into the window is left out silently (the window
+// part of the list covers it); a position outside [0, t) is recorded as an anomaly.
+__device__ __forceinline__ int checked_entry(const ListDesc& ld, int pos, int j, int end, int t, uint32_t* flags) {
+  if (j >= end) return -1;
+  if (ld.fused && j >= ld.s0 && j < ld.s0 + ld.nmid && pos >= ld.wlo) return -1;
+  if ((unsigned)pos >= (unsigned)t) {
+    atomicOr(flags, kFlagBadIndex);
+    return -1;
+  }
+  return pos;
+}
+
+// Per-warp set-up of the list descriptor (all 32 lanes call it).  In fused mode the middle part is
+// M without its entries below vis_lo: dilation can push at most r entries below S0, so a look at
+// the first 32 entries (a load that does not wait for the set's size) settles it; a longer overlap
+// (a sliding window start that moved past many entries) falls back to a full scan.  Entries of M
+// that have moved into the window since the set was stored (again at most r, at its end) stay
+// in the list and are masked where they are read: counting them would cost one more round of
+// dependent loads before the first row can be requested.
 __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit, int t) {
   ListDesc d;
   const int lane = threadIdx.x & 31;
@@ -121,25 +149,17 @@ __device__ __forceinline__ ListDesc make_list_desc(const AttnParams& p, int unit
     const int s0 = min(p.set.sinks, t);
     const int vis_lo = max(s0, psaw_start(p.set.psaw_c, t));
     const int wlo = max(max(t - p.set.window, 0), vis_lo);
-    int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && __ldg(M + min(lane, max(nm - 1, 0))) < vis_lo));
-    const int i1 = nm - 32 + lane;
-    int above = __popc(__ballot_sync(0xffffffffu, i1 >= 0 && __ldg(M + max(i1, 0)) >= wlo));
-    if (lo == 32 || above == 32) {      // unusual schedule change inside a block: count everything
-      int c0 = 0, c1 = 0;
-      for (int i = lane; i < nm; i += 32) {
-        const int x = __ldg(M + i);
-        c0 += x < vis_lo;
-        c1 += x >= wlo;
-      }
+    const int head = lane < mstride ? __ldg(M + lane) : 0x7fffffff;     // does not depend on nm
+    int lo = __popc(__ballot_sync(0xffffffffu, lane < nm && head < vis_lo));
+    if (lo == 32) {                     // a sliding window start far into the set: count everything
+      int c0 = 0;
+      for (int i = lane; i < nm; i += 32) c0 += __ldg(M + i) < vis_lo;
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        c0 += __shfl_xor_sync(0xffffffffu, c0, off);
-        c1 += __shfl_xor_sync(0xffffffffu, c1, off);
-      }
-      lo = c0; above = c1;
+      for (int off = 16; off > 0; off >>= 1) c0 += __shfl_xor_sync(0xffffffffu, c0, off);
+      lo = c0;
     }
     d.list = M; d.fused = 1; d.s0 = s0; d.lo = lo; d.wlo = wlo;
-    d.nmid = max(nm - above - lo, 0);
+    d.nmid = max(nm - lo, 0);
     d.count = s0 + d.nmid + (t - wlo);
   } else {
     d.list = nullptr;
@@ -248,23 +268,9 @@ __global__ void __launch_bounds__(kTThreads) gather_attn_mma_kernel(AttnParams p
   //   pos2 : raw list entry of group G+2 (a load from the list, unchecked)
   //   pos1 / pg1 : checked position of group G+1 and, for a paged cache, its raw page id (a load)
   //   rid_a : final row id of group G, the one being issued
-  auto list_pos = [&](int grp) -> int {
-    const int j = start + grp * 32 + lane;
-    if (j >= end) return -1;
-    if (ld.fused) {
-      if (j < ld.s0) return j;
-      if (j < ld.s0 + ld.nmid) return __ldg(ld.list + ld.lo + (j - ld.s0));
-      return ld.wlo + (j - ld.s0 - ld.nmid);
-    }
-    return ld.list ? __ldg(ld.list + j) : j;
-  };
+  auto list_pos = [&](int grp) -> int { return list_entry(ld, start + grp * 32 + lane, end); };
   auto check_pos = [&](int pos, int grp) -> int {      // consumes the list load
-    if (start + grp * 32 + lane >= end) return -1;
-    if ((unsigned)pos >= (unsigned)t) {
-      atomicOr(p.flags, kFlagBadIndex);
-      return -1;
-    }
-    return pos;
+    return checked_entry(ld, pos, start + grp * 32 + lane, end, t, p.flags);
   };
   const bool paged = p.kv.page_table != nullptr;
   auto page_of = [&](int pos) -> int {                 // issues the page-table load

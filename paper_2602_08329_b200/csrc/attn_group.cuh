@@ -52,23 +52,9 @@ __global__ void __launch_bounds__(kTThreads) gather_group_attn_mma_kernel(AttnPa
 
   // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane; every level is
   // produced one step before it is consumed (see gather_attn_mma_kernel).
-  auto list_pos = [&](int grp) -> int {
-    const int j = start + grp * 32 + lane;
-    if (j >= end) return -1;
-    if (ld.fused) {
-      if (j < ld.s0) return j;
-      if (j < ld.s0 + ld.nmid) return __ldg(ld.list + ld.lo + (j - ld.s0));
-      return ld.wlo + (j - ld.s0 - ld.nmid);
-    }
-    return ld.list ? __ldg(ld.list + j) : j;
-  };
+  auto list_pos = [&](int grp) -> int { return list_entry(ld, start + grp * 32 + lane, end); };
   auto check_pos = [&](int pos, int grp) -> int {
-    if (start + grp * 32 + lane >= end) return -1;
-    if ((unsigned)pos >= (unsigned)t) {
-      atomicOr(p.flags, kFlagBadIndex);
-      return -1;
-    }
-    return pos;
+    return checked_entry(ld, pos, start + grp * 32 + lane, end, t, p.flags);
   };
   const bool paged = p.kv.page_table != nullptr;
   auto page_of = [&](int pos) -> int {

@@ -98,23 +98,9 @@ gather_attn_tma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
   // Row-id pipeline, 32 list entries (two stages) per step, one entry per lane (as in
   // gather_attn_mma_kernel): pos2 = raw list entry of group G + 2, pos1 / pg1 = checked position
   // and page id of group G + 1, rid_a = row id of group G, the one being issued.
-  auto list_pos = [&](int grp) -> int {
-    const int j = start + grp * 32 + lane;
-    if (j >= end) return -1;
-    if (ld.fused) {
-      if (j < ld.s0) return j;
-      if (j < ld.s0 + ld.nmid) return __ldg(ld.list + ld.lo + (j - ld.s0));
-      return ld.wlo + (j - ld.s0 - ld.nmid);
-    }
-    return ld.list ? __ldg(ld.list + j) : j;
-  };
+  auto list_pos = [&](int grp) -> int { return list_entry(ld, start + grp * 32 + lane, end); };
   auto check_pos = [&](int pos, int grp) -> int {
-    if (start + grp * 32 + lane >= end) return -1;
-    if ((unsigned)pos >= (unsigned)t) {
-      atomicOr(p.flags, kFlagBadIndex);
-      return -1;
-    }
-    return pos;
+    return checked_entry(ld, pos, start + grp * 32 + lane, end, t, p.flags);
   };
   const bool paged = p.kv.page_table != nullptr;
   auto page_of = [&](int pos) -> int {

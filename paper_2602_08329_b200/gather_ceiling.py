@@ -63,19 +63,21 @@ def main():
     nbytes = rows * 512
     stream = torch.cuda.current_stream()
 
-    def timed(fn):
+    def timed(fn, rounds=4):
+        """Median time per launch: each sample brackets `rounds` passes over the cache copies with one
+        pair of events (the event clock ticks in steps of about 2 us: a single launch is too short to
+        time on its own), launches back to back, every launch on another copy than the one before."""
         ts = []
         for r in range(args.reps + 1):
-            evs = []
-            for l in range(L):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream)
-                fn(l)
-                b.record(stream)
-                evs.append((a, b))
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(rounds):
+                for l in range(L):
+                    fn(l)
+            b.record(stream)
             torch.cuda.synchronize()
             if r > 0:
-                ts += [a.elapsed_time(b) * 1e3 for a, b in evs]
+                ts.append(a.elapsed_time(b) * 1e3 / (rounds * L))
         return statistics.median(ts)
 
     res = [("gathered attention, list built in the kernel (a sharing step)",
