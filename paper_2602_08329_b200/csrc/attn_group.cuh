@@ -81,11 +81,17 @@ __global__ void __launch_bounds__(kTThreads) gather_group_attn_mma_kernel(AttnPa
   pg1 = page_of(pos1);
   int pos2 = list_pos(2);
 
-  const __nv_bfloat16* src_base = (lane < 16 ? p.kv.k : p.kv.v) + (lane & 15) * 8;
-  const uint32_t dst_tile = (lane < 16 ? 0u : (uint32_t)kTTileBytes);
-  unsigned long long vmask = 0ull;     // 16 validity bits per ring slot
+  // the copy of a row as in gather_attn_mma_kernel: lane p fills position p with source chunk p ^ (r & 7)
+  const __nv_bfloat16* srcx[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) srcx[k] = (lane < 16 ? p.kv.k : p.kv.v) + ((((uint32_t)lane & 15u) ^ (uint32_t)k) << 3);
+  const uint32_t dst_lane = (lane < 16 ? 0u : (uint32_t)kTTileBytes) + (((uint32_t)lane & 15u) << 4);
+  uint32_t vmv[kTStages];              // 16 validity bits per ring slot
+#pragma unroll
+  for (int k = 0; k < kTStages; ++k) vmv[k] = 0u;
 
-  auto issue = [&](int j) {
+  auto issue = [&](int j, auto slot_c) {
+    constexpr int kSlot = decltype(slot_c)::value;
     if (j < nstages) {
       if (j > 0 && (j & 1) == 0) {     // step the row-id pipeline
         const int grp = j >> 1;
@@ -96,41 +102,50 @@ __global__ void __launch_bounds__(kTThreads) gather_group_attn_mma_kernel(AttnPa
         pg1 = page_of(pos1);
         pos2 = list_pos(grp + 2);
       }
-      const int slot_i = j % kTStages;
-      const uint32_t slot = ring + (uint32_t)slot_i * kTStageBytes + dst_tile;
+      const uint32_t rid_cur = __shfl_sync(0xffffffffu, rid_a, (lane + ((j & 1) << 4)) & 31);
+      const uint32_t slot = ring + (uint32_t)kSlot * kTStageBytes + dst_lane;
       const uint32_t vm = (valid_a >> ((j & 1) * kTStageRows)) & 0xffffu;
       if (vm == 0xffffu) {             // the common case: 16 real rows
 #pragma unroll
         for (int r = 0; r < kTStageRows; ++r) {
-          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
-          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
-          cp_async_16_full(dst, src_base + (size_t)rid * kHeadDim);
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_cur, r);
+          cp_async_16_full(slot + r * kRowBytes, srcx[r & 7] + (size_t)rid * kHeadDim);
         }
       } else {
 #pragma unroll
         for (int r = 0; r < kTStageRows; ++r) {
-          const uint32_t rid = __shfl_sync(0xffffffffu, rid_a, (j & 1) * kTStageRows + r);
-          const uint32_t dst = slot + r * kRowBytes + ((((uint32_t)lane & 15u) ^ (r & 7u)) << 4);
-          cp_async_16(dst, src_base + (size_t)rid * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
+          const uint32_t rid = __shfl_sync(0xffffffffu, rid_cur, r);
+          cp_async_16(slot + r * kRowBytes, srcx[r & 7] + (size_t)rid * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
         }
       }
-      vmask = (vmask & ~(0xffffull << (16 * slot_i))) | ((unsigned long long)vm << (16 * slot_i));
+      vmv[kSlot] = vm;
     }
     cp_async_commit();
   };
 
-#pragma unroll
-  for (int j = 0; j < kTStages - 1; ++j) issue(j);
+  issue(0, SlotC<0>{});
+  issue(1, SlotC<1>{});
+  static_assert(kTStages == 3, "the stage loop below is unrolled over three ring slots");
 
-  for (int i = 0; i < nstages; ++i) {
+  auto stage = [&](int i, auto slot_c) {
+    constexpr int kSlot = decltype(slot_c)::value;
     cp_async_wait<kTStages - 2>();
     __syncwarp();
-    const int slot_i = i % kTStages;
-    const uint32_t vm = (uint32_t)(vmask >> (16 * slot_i)) & 0xffffu;
-    issue(i + kTStages - 1);
-    const uint32_t kt = ring + (uint32_t)slot_i * kTStageBytes;
+    const uint32_t vm = vmv[kSlot];
+    issue(i + kTStages - 1, SlotC<(kSlot + kTStages - 1) % kTStages>{});
+    const uint32_t kt = ring + (uint32_t)kSlot * kTStageBytes;
     group_stage(kt, kt + kTTileBytes, aq, (vm >> (2 * tg)) & 1u, (vm >> (2 * tg + 1)) & 1u,
                 (vm >> (8 + 2 * tg)) & 1u, (vm >> (9 + 2 * tg)) & 1u, o, m0, l0, m1, l1, lt0, lt1);
+  };
+  {
+    int i = 0;
+    for (; i + 2 < nstages; i += 3) {
+      stage(i, SlotC<0>{});
+      stage(i + 1, SlotC<1>{});
+      stage(i + 2, SlotC<2>{});
+    }
+    if (i < nstages) stage(i, SlotC<0>{});
+    if (i + 1 < nstages) stage(i + 1, SlotC<1>{});
   }
   cp_async_wait<0>();
   group_epilogue(p, g_smem, b, head0, gq, split, o, m0, l0, m1, l1, lt0, lt1);
