@@ -224,16 +224,18 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
   return best;
 }
 
-// Split count for the scoring kernels: about 4096 key rows (1 MB) per CTA, several waves of CTAs
-// per launch.  Short CTAs finish at different times, so the SMs never run dry together: a grid of
-// one wave of long CTAs measured 3 to 5 % slower (the 32K-context layer at batch 8: 327 us against
-// 317 us; the ragged paged batch of 64: 747 us against 711 us).  A small batch gets at least two
-// CTAs per resident slot, but no CTA fewer than 256 rows.  Contexts of a few thousand keys are
-// bound by latency, not by the stream: they keep the single wave.
-int score_splits(const prhs_ctx* c, int units, int max_t) {
+// Split count for the scoring kernels: a thousand key rows (256 KB) per CTA for a contiguous
+// cache, 4096 for a paged one (whose producer pays a page-table look-up per 16 rows), and so
+// several waves of CTAs per launch.  Short CTAs finish at different times, so the SMs never run
+// dry together: a grid of one wave of long CTAs measured 3 to 5 % slower (the 32K-context layer
+// at batch 8: 327 us against 312 us; the ragged paged batch of 64: 747 us against 711 us).  A
+// small batch gets at least two CTAs per resident slot, but no CTA fewer than 256 rows.  Contexts
+// of a few thousand keys are bound by latency, not by the stream: they keep the single wave.
+int score_splits(const prhs_ctx* c, int units, int max_t, bool paged) {
   if (max_t <= 8192) return pick_splits(c, units, max_t);      // short contexts are bound by latency: one wave
   const int slots = c->sm_count * 2;
-  int s = (max_t + 4095) / 4096;
+  const int rows = paged ? 4096 : 1024;
+  int s = (max_t + rows - 1) / rows;
   const int fill = (2 * slots + units - 1) / std::max(units, 1);
   s = std::max(s, std::min(fill, max_t / 256));
   return std::max(1, std::min(s, kMaxSplits));
@@ -250,7 +252,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.scores = write_scores ? c->scores : nullptr;
   sp.ld = c->ld;
   sp.part_ml = c->part_ml;
-  sp.splits = score_splits(c, batch * c->cfg.num_kv_heads, max_t);
+  sp.splits = score_splits(c, batch * c->cfg.num_kv_heads, max_t, kv.page_table != nullptr);
   sp.num_q_heads = c->cfg.num_q_heads;
   sp.group_size = c->gq;
   sp.need = need;
