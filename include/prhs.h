@@ -85,8 +85,9 @@ typedef struct {
                               default because it measured slower: a tile that ldmatrix reads without
                               bank conflicts needs the 128-byte swizzle, hence two 64-column boxes per
                               row, and at that granularity the copy engine falls behind (a sharing step
-                              of the 32K-context layer: 59.9 us against 51.7 us).  Kept so that the
-                              comparison can be repeated (python -m paper_2602_08329_b200.gather_ceiling). */
+                              of the 32K-context layer at batch 8: 49.0 us against 44.1 us).  Kept so
+                              that the comparison can be repeated
+                              (python -m paper_2602_08329_b200.gather_ceiling). */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at
@@ -246,6 +247,11 @@ prhs_status prhs_dense_decode_attn(prhs_ctx* ctx, const void* q, const prhs_kv_v
  * that need it, cached sets for the rest, attention over valid indices only).
  * Retrieves iff layer % G_L == 0 and step % s == 0; then builds the set and attends.
  * Within a step a group's first layer must be called before its other layers.
+ * With the cosine gate (sim_threshold > -1) the group's first layer decides per head on the
+ * device; unless the diagnostic is on, the attention of the heads that share is then launched on
+ * an internal stream beside the scoring and selection of the heads that retrieve, and `stream`
+ * continues when both branches have finished (event dependencies only; the step can still be
+ * captured into a CUDA graph).
  *   out        device bf16 [batch][Hq][128]
  *   out_delta  device fp32 [batch][Hq] or NULL (used only with PRHS_WANT_DELTA) */
 prhs_status prhs_decode_step(prhs_ctx* ctx, int32_t layer, int32_t step, const prhs_schedule* sched,

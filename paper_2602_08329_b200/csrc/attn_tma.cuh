@@ -15,9 +15,9 @@
 // No multicast.
 //
 // Selected by PRHS_CFG_TMA_GATHER only: it measured SLOWER than the cp.async kernel (a sharing
-// step of the 32K-context layer at batch 8: 59.9 us against 51.7 us; the grouped-query stack at
-// batch 16: 111 us against 91 us).  As a bare copy the row gather ties with cp.async when a row is
-// one 256-byte box (45.6 us against 45.4 us), but a tile that ldmatrix can read without bank
+// step of the 32K-context layer at batch 8: 49.0 us against 44.1 us; the grouped-query stack at
+// batch 16: 92 us against 72 us).  As a bare copy the row gather ties with cp.async when a row is
+// one 256-byte box (44.0 us against 43.0 us), but a tile that ldmatrix can read without bank
 // conflicts needs the 128-byte swizzle, whose boxes are at most 128 bytes wide: two boxes per row,
 // twice the copy instructions, and at that granularity the copy engine is the bottleneck.
 #pragma once
