@@ -75,7 +75,7 @@ typedef struct {
 
 /* Configuration flags */
 #define PRHS_CFG_NO_TMA 1u /* retrieval scoring never uses the tensor-memory-accelerator kernels: the
-                              key stream is staged by the cp.async ring kernel instead, which is what
+                              key stream is staged by the cp.async ring kernel (mma.sync) instead, which is what
                               the library falls back to on its own when the driver does not export
                               cuTensorMapEncodeTiled or the cache spans 2^31 rows or more.  Same
                               results; for testing that path and for comparing the two. */
@@ -88,6 +88,13 @@ typedef struct {
                               of the 32K-context layer at batch 8: 49.0 us against 44.1 us).  Kept so
                               that the comparison can be repeated
                               (python -m paper_2602_08329_b200.gather_ceiling). */
+#define PRHS_CFG_MMA_SYNC_SCORE 4u /* retrieval scoring runs its contraction with mma.sync in eight
+                              consumer warps (score_tma_kernel) instead of on the tcgen05 tensor cores
+                              (score_umma_kernel: 128-key tiles staged by TMA, one thread issues the
+                              MMAs, accumulators in tensor memory), which is the default.  Same results
+                              up to the summation order inside the tensor core; both are bound by the
+                              key stream and measure within 1 % of each other.  For testing that
+                              kernel and for comparing the two. */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at

@@ -24,6 +24,7 @@ PRHS_GROUP_SETS = 4
 PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TIMEOUT = 1, 2, 4, 8
 PRHS_CFG_NO_TMA = 1
 PRHS_CFG_TMA_GATHER = 2
+PRHS_CFG_MMA_SYNC_SCORE = 4
 
 # every symbol include/prhs.h declares
 EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_set",

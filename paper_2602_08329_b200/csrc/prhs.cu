@@ -19,6 +19,7 @@
 #include "common.cuh"
 #include "attn_group.cuh"
 #include "score_tma.cuh"
+#include "score_umma.cuh"
 #include "select.cuh"
 #include "gather_probe.cuh"
 #include "attn_tma.cuh"
@@ -257,7 +258,9 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.group_size = c->gq;
   sp.need = need;
   sp.group_max = (sched && (sched->flags & PRHS_GROUP_SETS) && c->gq > 1) ? 1 : 0;
-  sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + kSTStageRows - 1) & ~(kSTStageRows - 1);
+  const bool umma = !(c->cfg.flags & (PRHS_CFG_MMA_SYNC_SCORE | PRHS_CFG_NO_TMA));
+  const int tile_rows = umma ? kSUTileRows : kSTStageRows;
+  sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + tile_rows - 1) & ~(tile_rows - 1);
   sp.flags = c->flags;
   bool tma_done = false;
   if (c->encode_tiled && !(c->cfg.flags & PRHS_CFG_NO_TMA)) {
@@ -278,7 +281,7 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
       alignas(64) CUtensorMap tm;
       const cuuint64_t gdim[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows_total};
       const cuuint64_t gstr[1] = {(cuuint64_t)kRowBytes};
-      const cuuint32_t box[2] = {64u, paged ? 16u : (cuuint32_t)kSTStageRows};
+      const cuuint32_t box[2] = {64u, paged ? 16u : (cuuint32_t)tile_rows};
       const cuuint32_t estr[2] = {1u, 1u};
       const CUresult cr = reinterpret_cast<EncodeFn>(c->encode_tiled)(
           &tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(kv.k), gdim, gstr, box, estr,
@@ -287,7 +290,9 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
       if (cr == CUDA_SUCCESS) {
         LaunchScope ls(c, PRHS_KIND_SCORE, st);
         const dim3 grid(sp.splits, c->cfg.num_kv_heads, batch);
-        if (paged) score_tma_kernel<true><<<grid, kSTThreads, kSTSmemBytes, st>>>(tm, sp);
+        if (umma && paged) score_umma_kernel<true><<<grid, kSUThreads, kSUSmemBytes, st>>>(tm, sp);
+        else if (umma) score_umma_kernel<false><<<grid, kSUThreads, kSUSmemBytes, st>>>(tm, sp);
+        else if (paged) score_tma_kernel<true><<<grid, kSTThreads, kSTSmemBytes, st>>>(tm, sp);
         else score_tma_kernel<false><<<grid, kSTThreads, kSTSmemBytes, st>>>(tm, sp);
         tma_done = true;
       }
@@ -687,7 +692,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
   if (cfg->max_context > kMaxContext) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context above 2^20");
   if (cfg->max_k > 65536) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_k above 65536");
-  if (cfg->flags & ~(PRHS_CFG_NO_TMA | PRHS_CFG_TMA_GATHER)) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
+  if (cfg->flags & ~(PRHS_CFG_NO_TMA | PRHS_CFG_TMA_GATHER | PRHS_CFG_MMA_SYNC_SCORE)) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
 
   prhs_ctx* c = new (std::nothrow) prhs_ctx();
   if (!c) return fail(nullptr, PRHS_ERR_OOM, "host allocation failed");
@@ -741,6 +746,10 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     e = cudaFuncSetAttribute(score_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSUSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(score_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSUSmemBytes);
   if (e == cudaSuccess) {
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;

@@ -13,8 +13,9 @@ full-size tests are chosen to cover every width at the batch the configuration r
                                            multi-wave grid of every kernel)
   256 threads (two to four units per SM)   test_c3_full_batch_sampled (16 x 32 = 512 units),
                                            test_table3_operator_shapes[16-4096-16]
-Retrieval scoring runs the TMA kernels everywhere except in the test_score_ring_* tests, which
-create their contexts with PRHS_CFG_NO_TMA.
+Retrieval scoring runs the tcgen05 kernel (TMA-staged) everywhere except in the
+test_score_mma_sync_* tests (PRHS_CFG_MMA_SYNC_SCORE: mma.sync consumer warps behind the same TMA
+ring) and the test_score_ring_* tests (PRHS_CFG_NO_TMA: the cp.async ring kernel).
 """
 import math
 
@@ -502,23 +503,96 @@ def test_score_ring_c2_sampled(cuda_device):
     assert st["checked"] == 5 * len(units) and not st["select_fallback"]
 
 
-def test_score_ring_and_tma_logits_agree(cuda_device):
-    # the two scoring kernels on the same inputs: same logits (both within the tolerance of the
-    # oracle, so within twice that of each other) and the same log-sum-exp
+def test_score_kernels_logits_agree(cuda_device):
+    # the three scoring kernels (tcgen05, mma.sync behind TMA, mma.sync behind cp.async) on the same
+    # inputs: same logits (each within the tolerance of the oracle, so within twice that of each
+    # other) and the same log-sum-exp
     w = small(batch=2, q_heads=8, kv_heads=2, context=5000, top_k=64, seed=18)
     k, v = W.make_kv(w, cuda_device)
     q = W.make_queries(w, cuda_device)[0, 0].contiguous()
     view = P.make_view(k, v, W.seq_lens_at(w, 0).to(cuda_device), max_seq_len=w.capacity)
     res = []
-    for flags in (0, P.PRHS_CFG_NO_TMA):
+    for flags in (0, P.PRHS_CFG_MMA_SYNC_SCORE, P.PRHS_CFG_NO_TMA):
         ctx = H.make_ctx(w, flags=flags)
         lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
         ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), w.batch, out_lse_full=lse)
         assert ctx.check() == 0
         res.append((ctx.get_scores(w.batch)[:, :, : w.context + 1], lse.cpu()))
         ctx.close()
-    assert torch.allclose(res[0][0], res[1][0], atol=2 * H.LOGIT_ATOL, rtol=2 * H.LOGIT_RTOL)
-    assert torch.allclose(res[0][1], res[1][1], atol=1e-4)
+    for other in res[1:]:
+        assert torch.allclose(res[0][0], other[0], atol=2 * H.LOGIT_ATOL, rtol=2 * H.LOGIT_RTOL)
+        assert torch.allclose(res[0][1], other[1], atol=1e-4)
+
+
+# ------------------------------------------------ retrieval scoring on the tcgen05 tensor cores
+def test_score_tcgen05_logits_against_oracle(cuda_device):
+    # the default scoring kernel (tcgen05) on the smallest useful case: several 128-key tiles and a
+    # ragged last one per split, grouped-query heads (4 per KV head), logits and log-sum-exp element
+    # by element
+    w = small(batch=2, q_heads=8, kv_heads=2, context=5000, top_k=64, seed=41)
+    k, v = W.make_kv(w, cuda_device)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_host = W.seq_lens_at(w, 0)
+    view = P.make_view(k, v, t_host.to(cuda_device), max_seq_len=w.capacity)
+    ctx = H.make_ctx(w)
+    lse = torch.empty(w.batch, w.q_heads, dtype=torch.float32, device=cuda_device)
+    ctx.score_topk(0, 0, q, view, H.make_sched(w, cuda_device), w.batch, out_lse_full=lse)
+    assert ctx.check() == 0
+    scores = ctx.get_scores(w.batch)
+    kn, qn = k.float().cpu().numpy().astype(np.float64), q.float().cpu().numpy().astype(np.float64)
+    gq = w.q_heads // w.kv_heads
+    for b in range(w.batch):
+        t = int(t_host[b])
+        for h in range(w.q_heads):
+            ref = O.dense_scores(qn[b, h], kn[b, h // gq], t)
+            got = scores[b, h, :t].numpy().astype(np.float64)
+            assert np.allclose(got, ref, atol=H.LOGIT_ATOL, rtol=H.LOGIT_RTOL), (b, h, np.abs(got - ref).max())
+            assert abs(float(lse[b, h]) - O.logsumexp(ref)) < 1e-4
+    ctx.close()
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_score_tcgen05_small_every_unit(cuda_device, paged):
+    w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=3, q_heads=8, kv_heads=2, context=2700,
+              min_context=400 if paged else 0, page_size=16 if paged else 0, seed=42)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged)
+    assert st["checked"] == 2 * 4 * w.batch * w.q_heads
+
+
+def test_score_tcgen05_group_of_sixteen_and_single_head(cuda_device):
+    # the widest group the MMA tile holds (16 heads on its 16 columns) and multi-head attention
+    # (one live column)
+    for q_heads, kv_heads in ((16, 1), (4, 4)):
+        w = small(batch=2, q_heads=q_heads, kv_heads=kv_heads, context=1500, steps=3, refresh=2, seed=43)
+        st = H.run_schedule_parity(w, cuda_device, all_units(w))
+        assert st["checked"] == 3 * w.batch * w.q_heads
+
+
+# ------------------------------------- retrieval scoring with mma.sync consumer warps (an option)
+@pytest.mark.parametrize("paged", [False, True])
+def test_score_mma_sync_small_every_unit(cuda_device, paged):
+    # PRHS_CFG_MMA_SYNC_SCORE: the TMA-staged kernel whose eight consumer warps run m16n8k16 MMAs
+    w = small(layers=2, layer_group=2, steps=4, refresh=2, batch=3, q_heads=8, kv_heads=2, context=2700,
+              min_context=400 if paged else 0, page_size=16 if paged else 0, seed=44)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged,
+                               ctx_over=dict(flags=P.PRHS_CFG_MMA_SYNC_SCORE))
+    assert st["checked"] == 2 * 4 * w.batch * w.q_heads
+
+
+def test_score_mma_sync_c2_sampled(cuda_device):
+    w = W.C2_LLAMA2_7B.scaled(steps=5)
+    units = [(0, 0), (7, 31), (3, 12)]
+    st = H.run_schedule_parity(w, cuda_device, units, ctx_over=dict(flags=P.PRHS_CFG_MMA_SYNC_SCORE))
+    assert st["checked"] == 5 * len(units) and not st["select_fallback"]
+
+
+def test_score_mma_sync_c5_sampled(cuda_device):
+    # paged, ragged, grouped queries at a reduced batch
+    w = W.C5_SERVING.scaled(layers=4, steps=2, batch=6)
+    units = [(0, 0), (5, 31), (2, 9), (3, 16)]
+    st = H.run_schedule_parity(w, cuda_device, units, layers=[0, 1], paged=True,
+                               ctx_over=dict(flags=P.PRHS_CFG_MMA_SYNC_SCORE))
+    assert st["checked"] == 2 * 2 * len(units)
 
 
 # ------------------------------------------ gathered attention with rows by TMA gather (an option)
