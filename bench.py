@@ -47,7 +47,7 @@ UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch (read + write) of the kernels, from the ncu captures summarised under
 # profiles/ (captured at batch 2-4 and scaled to the full batch by the units processed).
-NCU_TRAFFIC_BYTES = {"score": 2.166e9, "attn_sparse": 2.42e8}
+NCU_TRAFFIC_BYTES = {"score": 2.163e9, "attn_sparse": 2.42e8}
 
 
 def load_peaks():

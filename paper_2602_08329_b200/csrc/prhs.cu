@@ -266,8 +266,8 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   if (c->encode_tiled && !(c->cfg.flags & PRHS_CFG_NO_TMA)) {
     // K as a 2-D tensor [rows][128] bf16.  Contiguous cache: rows past the last sequence's max
     // length are out of bounds for the copy engine (zero fill), rows in between belong to the
-    // cache; a copy brings 64 rows.  Paged cache: the rows of the page pool; a copy brings the
-    // 16 rows of one page.
+    // cache; a copy brings the rows of one tile (128 for the tcgen05 kernel, 64 for the mma.sync one).
+    // Paged cache: the rows of the page pool; a copy brings the 16 rows of one page.
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
