@@ -95,6 +95,15 @@ typedef struct {
                               up to the summation order inside the tensor core; both are bound by the
                               key stream and measure within 1 % of each other.  For testing that
                               kernel and for comparing the two. */
+#define PRHS_CFG_GROUP_TCGEN05 8u /* the gathered attention of the group-shared variant (PRHS_GROUP_SETS)
+                              runs on the tcgen05 tensor cores (gather_group_attn_umma_kernel: 128-row
+                              tiles gathered into swizzled shared memory, S and O^T in tensor memory)
+                              instead of mma.sync with register accumulators.  Same results up to
+                              summation order.  Off by default because it measured slower (sharing step
+                              of the variant at 32K, batch 16: 44.6 us against 42.7 us; at 128K, batch 4:
+                              40.4 against 34.3; ragged paged batch of 64: 192 against 122): its ring
+                              leaves room for one CTA per SM, so nothing covers a CTA's set-up and
+                              merge.  Kept for the comparison. */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at

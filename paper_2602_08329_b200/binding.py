@@ -25,6 +25,7 @@ PRHS_FLAG_BAD_INDEX, PRHS_FLAG_BAD_PAGE, PRHS_FLAG_SELECT_FALLBACK, PRHS_FLAG_TI
 PRHS_CFG_NO_TMA = 1
 PRHS_CFG_TMA_GATHER = 2
 PRHS_CFG_MMA_SYNC_SCORE = 4
+PRHS_CFG_GROUP_TCGEN05 = 8
 
 # every symbol include/prhs.h declares
 EXPORTS = ["prhs_create", "prhs_destroy", "prhs_score_topk", "prhs_build_index_set",

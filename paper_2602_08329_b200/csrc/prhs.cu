@@ -23,6 +23,7 @@
 #include "select.cuh"
 #include "gather_probe.cuh"
 #include "attn_tma.cuh"
+#include "attn_group_umma.cuh"
 
 using namespace prhs;
 
@@ -372,10 +373,27 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
     dense_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
   } else if (!idx && fs.share_gq > 1) {
     // group-shared sets: one CTA column per KV head, a gathered row serves the whole group
-    p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
-    dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
     LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
-    gather_group_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
+    if (c->cfg.flags & PRHS_CFG_GROUP_TCGEN05) {
+      // one CTA per SM (a 200 KB ring): the split count that fills whole waves of SMs, tiles of 128 rows
+      const int units = batch * c->cfg.num_kv_heads;
+      int best = 1;
+      double best_cost = 1e30;
+      for (int s = 1; s <= kMaxSplits; ++s) {
+        const int rows = (((max_count + s - 1) / s) + kGUTileRows - 1) & ~(kGUTileRows - 1);
+        if (s > 1 && rows < 2 * kGUTileRows) break;
+        const double waves = (double)(((long long)units * s + c->sm_count - 1) / c->sm_count);
+        const double cost = waves * (rows + 2 * kGUTileRows);
+        if (cost < best_cost * 0.999) { best_cost = cost; best = s; }
+      }
+      p.splits = best;
+      dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
+      gather_group_attn_umma_kernel<<<grid, kGUThreads, kGUSmemBytes, st>>>(p);
+    } else {
+      p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
+      dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
+      gather_group_attn_mma_kernel<<<grid, kTThreads, kTSmemBytes, st>>>(p);
+    }
   } else {
     dim3 grid(p.splits, c->cfg.num_q_heads, batch);
     // rows by 16-byte cp.async copies; by TMA row gather only where the context asks for it
@@ -692,7 +710,7 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (cfg->num_q_heads / cfg->num_kv_heads > 16) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "group size above 16");
   if (cfg->max_context > kMaxContext) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_context above 2^20");
   if (cfg->max_k > 65536) return fail(nullptr, PRHS_ERR_UNSUPPORTED, "max_k above 65536");
-  if (cfg->flags & ~(PRHS_CFG_NO_TMA | PRHS_CFG_TMA_GATHER | PRHS_CFG_MMA_SYNC_SCORE)) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
+  if (cfg->flags & ~(PRHS_CFG_NO_TMA | PRHS_CFG_TMA_GATHER | PRHS_CFG_MMA_SYNC_SCORE | PRHS_CFG_GROUP_TCGEN05)) return fail(nullptr, PRHS_ERR_INVALID_ARG, "prhs_create: unknown configuration flag");
 
   prhs_ctx* c = new (std::nothrow) prhs_ctx();
   if (!c) return fail(nullptr, PRHS_ERR_OOM, "host allocation failed");
@@ -742,6 +760,8 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
     e = cudaFuncSetAttribute(gather_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_group_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_group_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGUSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
   if (e == cudaSuccess)

@@ -866,6 +866,45 @@ def test_group_sets_c3_slice_sampled(cuda_device):
     assert st["checked"] == 4 * 5 * len(units)
 
 
+# ------------------------- the group-shared variant's attention on the tcgen05 tensor cores
+@pytest.mark.gpu
+def test_group_sets_tcgen05_one_small_case(cuda_device):
+    # PRHS_CFG_GROUP_TCGEN05, smallest useful case: lists of a few 128-row tiles with a ragged last
+    # one, four heads per KV head, retrieval and sharing steps
+    w = small(layers=1, steps=3, refresh=2, batch=2, q_heads=8, kv_heads=2, context=2400, top_k=300, seed=51)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), group_sets=True,
+                               ctx_over=dict(flags=P.PRHS_CFG_GROUP_TCGEN05))
+    assert st["checked"] == 3 * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("hq,hkv,paged", [(8, 2, False), (16, 1, False), (12, 4, True), (4, 4, False)])
+def test_group_sets_tcgen05_schedule(cuda_device, hq, hkv, paged):
+    w = small(layers=4, layer_group=2, steps=5, refresh=2, q_heads=hq, kv_heads=hkv, context=2400, seed=52,
+              psaw_layer_start=3, page_size=16 if paged else 0)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=True,
+                               ctx_over=dict(flags=P.PRHS_CFG_GROUP_TCGEN05))
+    assert st["checked"] == 4 * 5 * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
+def test_group_sets_tcgen05_full_shapes_sampled(cuda_device):
+    # the Mistral-shaped stack, the 128K shape (several splits per unit: partials and the merge) and the
+    # ragged paged serving mix
+    over = dict(flags=P.PRHS_CFG_GROUP_TCGEN05)
+    w = W.C3_MISTRAL.scaled(layers=8, steps=5, batch=4)
+    st = H.run_schedule_parity(w, cuda_device, [(0, 0), (0, 3), (2, 21), (3, 31)], layers=[0, 1, 3, 4],
+                               group_sets=True, ctx_over=over)
+    assert st["checked"] == 4 * 5 * 4
+    w = W.C4_LLAMA3_128K.scaled(steps=5)
+    st = H.run_schedule_parity(w, cuda_device, [(0, 0), (1, 13), (3, 31)], group_sets=True, ctx_over=over)
+    assert st["checked"] == 5 * 3 and not st["select_fallback"]
+    w = W.C5_SERVING.scaled(layers=4, steps=5, batch=6)
+    st = H.run_schedule_parity(w, cuda_device, [(0, 0), (2, 9), (5, 31), (3, 16)], layers=[0, 1, 3], paged=True,
+                               group_sets=True, ctx_over=over)
+    assert st["checked"] == 5 * 3 * 4
+
+
 # ------------------------------------------- selection kernel: the rarely taken configurations
 @pytest.mark.gpu
 @pytest.mark.parametrize("case", ["large_k_bitonic", "one_bitmap", "k_above_candidates", "list_everything"])
