@@ -247,6 +247,44 @@ def test_bad_index_is_flagged_not_faulted(cuda_device):
     ctx.close()
 
 
+@pytest.mark.parametrize("flags,group_sets", [(0, False), (P.PRHS_CFG_MMA_SYNC_SCORE, False), (P.PRHS_CFG_NO_TMA, False),
+                                              (P.PRHS_CFG_TMA_GATHER, False), (0, True),
+                                              (P.PRHS_CFG_GROUP_TCGEN05, True)])
+def test_bad_page_id_is_flagged_not_dereferenced(cuda_device, flags, group_sets):
+    # page ids outside the pool in one sequence's table: every kernel that looks pages up (the three
+    # scoring kernels, the gathered attention kernels, the dense baseline) checks the id before it
+    # forms an address, skips the page and records the anomaly; the other sequence is untouched
+    w = small(batch=2, q_heads=8, kv_heads=2, context=1500, top_k=64, page_size=16, seed=61)
+    table, pool = W.make_page_table(w)
+    k, v = W.make_kv(w, cuda_device)
+    kp, vp = W.to_paged(w, k, table, pool), W.to_paged(w, v, table, pool)
+    q = W.make_queries(w, cuda_device)[0, 0].contiguous()
+    t_dev = W.seq_lens_at(w, 0).to(cuda_device)
+    bad = table.clone()
+    bad[1, 5] = pool + 3
+    bad[1, 9] = -1
+    sched = H.make_sched(w, cuda_device, flags=P.PRHS_GROUP_SETS if group_sets else 0)
+    outs = []
+    for tab in (table, bad):
+        ctx = H.make_ctx(w, flags=flags)
+        view = P.make_view(kp, vp, t_dev, page_table=tab.to(cuda_device), max_seq_len=w.capacity)
+        out = torch.empty(w.batch, w.q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+        dense = torch.empty_like(out)
+        ctx.decode_step(0, 0, sched, q, view, w.batch, out)
+        ctx.dense_decode_attn(q, view, w.batch, dense)
+        if tab is table:
+            assert ctx.check() == 0
+        else:
+            with pytest.raises(P.PrhsError) as e:
+                ctx.check()
+            assert e.value.status == 7 and int(str(e.value).split("0x")[1], 16) & P.PRHS_FLAG_BAD_PAGE
+            assert ctx.check() == 0
+        outs.append((out.cpu(), dense.cpu()))
+        ctx.close()
+    assert torch.equal(outs[0][0][0], outs[1][0][0]) and torch.equal(outs[0][1][0], outs[1][1][0])
+    assert torch.isfinite(outs[1][1][1].float()).all()
+
+
 def test_results_are_deterministic(cuda_device):
     w = small(context=2500)
     outs = []
