@@ -1114,6 +1114,25 @@ def test_random_schedules(cuda_device, seed):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("seed", list(range(100, 112)))
+def test_random_schedules_kernel_options(cuda_device, seed):
+    """The same random shapes through the optional kernels, in turn: scoring with mma.sync behind the TMA
+    ring, scoring behind the cp.async ring, the TMA row-gather attention, and the group-shared variant's
+    attention on tcgen05."""
+    w, paged, group_sets = _random_workload(seed)
+    flags = [P.PRHS_CFG_MMA_SYNC_SCORE, P.PRHS_CFG_NO_TMA, P.PRHS_CFG_TMA_GATHER, P.PRHS_CFG_GROUP_TCGEN05][seed % 4]
+    if flags == P.PRHS_CFG_GROUP_TCGEN05:
+        group_sets = True
+        if w.q_heads == w.kv_heads:
+            w = w.scaled(q_heads=2 * w.q_heads)
+    elif flags == P.PRHS_CFG_TMA_GATHER:
+        group_sets = False
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=group_sets,
+                               ctx_over=dict(flags=flags))
+    assert st["checked"] == w.layers * w.steps * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
 def test_group_sets_stage_calls(cuda_device):
     """The stage-by-stage entry points with group-shared sets: prhs_score_topk hands every head
     of a group the group's S* (ranked by the group maximum), prhs_build_index_set the group's
