@@ -59,7 +59,7 @@ def time_workload(w: W.Workload, dev, copies: int = 4, reps: int = 6, group_sets
     kps = W.top_k_per_seq(w)
     max_k = max(w.top_k, int(w.k_frac * w.context))
     ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
-                    page_size=w.page_size)
+                    page_size=w.page_size, flags=CTX_FLAGS)
     sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=w.refresh, dilate_r=w.dilate_r,
                             top_k_per_seq=None if kps is None else kps.to(dev),
                             flags=P.PRHS_GROUP_SETS if group_sets else 0)
@@ -133,7 +133,7 @@ def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6, grou
     kps = W.top_k_per_seq(w)
     max_k = max(w.top_k, int(w.k_frac * w.context))
     ctx = P.Context(copies, B, Hq, w.kv_heads, w.capacity, max_k, w.window, w.sinks, max_dilate_r=w.dilate_r,
-                    page_size=w.page_size)
+                    page_size=w.page_size, flags=CTX_FLAGS)
     sched = P.make_schedule(w.top_k, w.window, w.sinks, refresh_interval=s, dilate_r=w.dilate_r,
                             top_k_per_seq=None if kps is None else kps.to(dev),
                             flags=P.PRHS_GROUP_SETS if group_sets else 0)
@@ -176,6 +176,9 @@ def time_blocks(w: W.Workload, dev, s: int, copies: int = 4, reps: int = 6, grou
     assert ctx.check() == 0
     ctx.close()
     return res
+
+
+CTX_FLAGS = 0      # PRHS_CFG_* flags every context of this module is created with (--ctx-flags)
 
 
 def _make_caches(w: W.Workload, dev):
@@ -225,7 +228,7 @@ def config_summary(w: W.Workload, dev, reps: int = 7, copies: int = 4, group_set
     kps = W.top_k_per_seq(ws)
     max_k = max(ws.top_k, int(ws.k_frac * ws.context))
     ctx = P.Context(NL, B, Hq, ws.kv_heads, ws.capacity, max_k, ws.window, ws.sinks, max_dilate_r=ws.dilate_r,
-                    page_size=ws.page_size, min_layer_group=ws.layer_group)
+                    page_size=ws.page_size, min_layer_group=ws.layer_group, flags=CTX_FLAGS)
     sched = P.make_schedule(ws.top_k, ws.window, ws.sinks, refresh_interval=s, layer_group=ws.layer_group,
                             dilate_r=ws.dilate_r, top_k_per_seq=None if kps is None else kps.to(dev),
                             flags=P.PRHS_GROUP_SETS if group_sets else 0)
@@ -360,7 +363,7 @@ def gated_summary(w: W.Workload, dev, tau: float = 0.8, sigma: float = 0.7, s: i
     def run(sim_threshold, refresh):
         ctx = P.Context(copies, B, Hq, ws.kv_heads, ws.capacity, ws.top_k, ws.window, ws.sinks,
                         max_dilate_r=ws.dilate_r, page_size=ws.page_size,
-                        max_block_sets=refresh if sim_threshold is not None else 1)
+                        max_block_sets=refresh if sim_threshold is not None else 1, flags=CTX_FLAGS)
         sched = P.make_schedule(ws.top_k, ws.window, ws.sinks, refresh_interval=refresh, dilate_r=ws.dilate_r,
                                 sim_threshold=-1.0 if sim_threshold is None else sim_threshold)
         retrieved = 0
@@ -495,6 +498,8 @@ def main():
     ap.add_argument("--sigmas", default="0.6,0.7,0.75", help="with --gated: query drifts to time")
     ap.add_argument("--only", default=None, help="with --configs: time this configuration alone (its name)")
     ap.add_argument("--batch", type=int, default=0, help="with --configs: override the batch size (profiler captures)")
+    ap.add_argument("--ctx-flags", type=int, default=0,
+                    help="PRHS_CFG_* flags for every context (4: mma.sync scoring, 8: tcgen05 group attention, ...)")
     ap.add_argument("--group-sets", action="store_true",
                     help="with --configs: the labelled variant with one index set per KV head (not in the paper)")
     args = ap.parse_args()
@@ -502,6 +507,8 @@ def main():
         raise SystemExit("needs a CUDA device")
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
+    global CTX_FLAGS
+    CTX_FLAGS = args.ctx_flags
     if args.gated:
         import json
         w = W.CONFIGS[args.only] if args.only else W.C2_LLAMA2_7B
