@@ -94,7 +94,9 @@ typedef struct {
                               MMAs, accumulators in tensor memory), which is the default.  Same results
                               up to the summation order inside the tensor core; both are bound by the
                               key stream and measure within 1 % of each other.  For testing that
-                              kernel and for comparing the two. */
+                              kernel and for comparing the two.  Cosine-gated steps use this kernel
+                              whatever the flag says: most of their CTAs return at once, and an empty CTA
+                              of a kernel that uses tensor memory is several times as expensive. */
 #define PRHS_CFG_GROUP_TCGEN05 8u /* the gathered attention of the group-shared variant (PRHS_GROUP_SETS)
                               runs on the tcgen05 tensor cores (gather_group_attn_umma_kernel: 128-row
                               tiles gathered into swizzled shared memory, S and O^T in tensor memory)

@@ -233,10 +233,12 @@ int pick_splits(const prhs_ctx* c, int units, int max_count) {
 // at batch 8: 327 us against 312 us; the ragged paged batch of 64: 747 us against 711 us).  A
 // small batch gets at least two CTAs per resident slot, but no CTA fewer than 256 rows.  Contexts
 // of a few thousand keys are bound by latency, not by the stream: they keep the single wave.
-int score_splits(const prhs_ctx* c, int units, int max_t, bool paged) {
+int score_splits(const prhs_ctx* c, int units, int max_t, bool paged, bool gated) {
   if (max_t <= 8192) return pick_splits(c, units, max_t);      // short contexts are bound by latency: one wave
   const int slots = c->sm_count * 2;
-  const int rows = paged ? 4096 : 1024;
+  // a cosine-gated step launches the CTAs of every unit and those of the units that share return at
+  // once: four times fewer CTAs there (7 us of empty CTAs per step at 8448, 2 us at 2304)
+  const int rows = (paged || gated) ? 4096 : 1024;
   int s = (max_t + rows - 1) / rows;
   const int fill = (2 * slots + units - 1) / std::max(units, 1);
   s = std::max(s, std::min(fill, max_t / 256));
@@ -254,12 +256,16 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.scores = write_scores ? c->scores : nullptr;
   sp.ld = c->ld;
   sp.part_ml = c->part_ml;
-  sp.splits = score_splits(c, batch * c->cfg.num_kv_heads, max_t, kv.page_table != nullptr);
+  sp.splits = score_splits(c, batch * c->cfg.num_kv_heads, max_t, kv.page_table != nullptr, need != nullptr);
   sp.num_q_heads = c->cfg.num_q_heads;
   sp.group_size = c->gq;
   sp.need = need;
   sp.group_max = (sched && (sched->flags & PRHS_GROUP_SETS) && c->gq > 1) ? 1 : 0;
-  const bool umma = !(c->cfg.flags & (PRHS_CFG_MMA_SYNC_SCORE | PRHS_CFG_NO_TMA));
+  // A cosine-gated step launches the grid for every unit and the CTAs of the units that share return at
+  // once.  A CTA of a kernel that uses tensor memory costs about half a microsecond to launch and retire
+  // even then (8448 empty CTAs: 28 us against 7 us for the mma.sync kernel), so gated steps score with
+  // the mma.sync kernel.
+  const bool umma = !(c->cfg.flags & (PRHS_CFG_MMA_SYNC_SCORE | PRHS_CFG_NO_TMA)) && need == nullptr;
   const int tile_rows = umma ? kSUTileRows : kSTStageRows;
   sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + tile_rows - 1) & ~(tile_rows - 1);
   sp.flags = c->flags;

@@ -13,7 +13,9 @@
 // CTA instead of nine, and two accumulators in tensor memory let the MMAs of tile j + 1 run while
 // tile j is read out.  The kernel is bound by the key stream exactly like score_tma_kernel (the two
 // measure within 1 % of each other on every benchmark shape, this one ahead); it is the default
-// because it leaves the SM's issue slots and registers nearly idle.
+// because it leaves the SM's issue slots and registers nearly idle.  Not for cosine-gated steps, whose
+// CTAs mostly return at once: a CTA of this kernel costs about half a microsecond to launch and retire
+// even then.
 //
 // Warp roles: 0 = TMA producer, 1 = tensor-memory allocation + MMA issue, 2..5 = epilogue (tensor
 // memory lanes 32 (warp mod 4) .. + 31).  Every mbarrier wait is bounded like score_tma_kernel's;
