@@ -262,9 +262,9 @@ prhs_status launch_score(prhs_ctx* c, const void* q, const KvDev& kv, int batch,
   sp.need = need;
   sp.group_max = (sched && (sched->flags & PRHS_GROUP_SETS) && c->gq > 1) ? 1 : 0;
   // A cosine-gated step launches the grid for every unit and the CTAs of the units that share return at
-  // once.  A CTA of a kernel that uses tensor memory costs about half a microsecond to launch and retire
-  // even then (8448 empty CTAs: 28 us against 7 us for the mma.sync kernel), so gated steps score with
-  // the mma.sync kernel.
+  // once.  CTAs of a kernel that uses tensor memory are several times slower to launch and retire even
+  // then (8448 empty CTAs: 28 us against 7 us for the mma.sync kernel), so gated steps score with the
+  // mma.sync kernel.
   const bool umma = !(c->cfg.flags & (PRHS_CFG_MMA_SYNC_SCORE | PRHS_CFG_NO_TMA)) && need == nullptr;
   const int tile_rows = umma ? kSUTileRows : kSTStageRows;
   sp.chunk_rows = (((max_t + sp.splits - 1) / sp.splits) + tile_rows - 1) & ~(tile_rows - 1);
