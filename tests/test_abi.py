@@ -27,6 +27,23 @@ def test_header_and_binding_agree():
     assert declared_symbols() == sorted(P.EXPORTS)
 
 
+def test_header_constants_and_binding_agree(lib):
+    # every PRHS_* integer constant the header defines has the same value in the binding, and a
+    # configuration flag the header does not define is rejected at creation
+    text = open(os.path.join(ROOT, "include", "prhs.h")).read()
+    defs = dict(re.findall(r"#define\s+(PRHS_(?:CFG|FLAG)_[A-Z0-9_]+)\s+(\d+)u?", text))
+    assert {"PRHS_CFG_NO_TMA", "PRHS_CFG_TMA_GATHER", "PRHS_CFG_MMA_SYNC_SCORE", "PRHS_CFG_GROUP_TCGEN05"} <= set(defs)
+    for name, value in defs.items():
+        assert getattr(P, name) == int(value), name
+    known = 0
+    for name, value in defs.items():
+        if name.startswith("PRHS_CFG_"):
+            known |= int(value)
+    h = ctypes.c_void_p()
+    bad = P.Config(1, 1, 4, 2, 128, 1000, 0, 16, 16, 4, 1, -1, 1, 1, (known + 1) & ~known)
+    assert lib.prhs_create(ctypes.byref(bad), ctypes.byref(h)) == 1 and not h.value
+
+
 def test_library_exports_every_declared_symbol(lib):
     for name in declared_symbols():
         assert hasattr(lib, name), name
