@@ -102,10 +102,11 @@ typedef struct {
                               tiles gathered into swizzled shared memory, S and O^T in tensor memory)
                               instead of mma.sync with register accumulators.  Same results up to
                               summation order.  Off by default because it measured slower (sharing step
-                              of the variant at 32K, batch 16: 44.6 us against 42.7 us; at 128K, batch 4:
-                              40.4 against 34.3; ragged paged batch of 64: 192 against 122): its ring
-                              leaves room for one CTA per SM, so nothing covers a CTA's set-up and
-                              merge.  Kept for the comparison. */
+                              of the variant at 32K, batch 16: 44.5 us against 42.6 us; at 128K, batch 4:
+                              40.3 against 34.3; ragged paged batch of 64: 128 against 120): its rings
+                              of 128-row tiles leave room for one deep or two shallow CTAs per SM,
+                              where the mma.sync kernel pipelines 16-row stages per warp.  Kept for the
+                              comparison. */
 
 /* A view of one layer's KV cache (device memory, bf16, caller-owned).
  *   contiguous (page_table == NULL): row i of (b, kvh) is at

@@ -23,14 +23,18 @@
 // outputs and delta are per query head, as in the mma.sync kernel.  Every mbarrier wait is bounded;
 // tensor memory is freed on every path.
 //
+// The kernel is a template over the shape of a CTA (GUShape below): two softmax groups and two loader sets
+// as described (18 warps, a 205 KB ring, one CTA per SM), or one of each (10 warps, 109 KB, two CTAs per
+// SM); the library launches the second where there are more units than SMs.
+//
 // Selected by PRHS_CFG_GROUP_TCGEN05 only.  Measured against the mma.sync kernel (sharing step of the
-// group-shared variant, us): 32K contexts at batch 16: 44.6 against 42.7; 128K at batch 4: 40.4 against
-// 34.3; the ragged paged batch of 64: 192 against 122.  Its 200 KB ring allows one CTA per SM, so the
-// per-CTA set-up and merge (about 7 us: list description, tensor-memory allocation, Q tile; partials,
-// ticket) is not covered by a second CTA as it is for the mma.sync kernel, which costs most where a
-// launch is several waves of CTAs; and a tile passes through four agents (loader set, S issue, softmax
-// group, O issue), so a stage stays occupied for about 3 us.  Deeper variants measured slower (three
-// loader sets with three K and three V stages: 52.6 us at the first shape).
+// group-shared variant, us): 32K contexts at batch 16: 44.5 against 42.6; 128K at batch 4: 40.3 against
+// 34.3; the ragged paged batch of 64: 128 against 120.  With one CTA per SM the per-CTA set-up and merge
+// (about 7 us: list description, tensor-memory allocation, Q tile; partials, ticket) is not covered by a
+// second CTA as it is for the mma.sync kernel; with two per SM each has room for one K tile and two V
+// tiles only, and a tile passes through four agents (loader set, S issue, softmax group, O issue), so a
+// stage stays occupied for about 3 us.  Other arrangements measured slower (three loader sets with three
+// K and three V stages: 52.6 us at the first shape; two sets with three and three: 46.5).
 #pragma once
 #include "attn.cuh"
 #include "score_umma.cuh"
@@ -38,12 +42,20 @@
 namespace prhs {
 
 constexpr int kGUTileRows = 128;
-constexpr int kGUKStages = 2, kGUVStages = 4;            // K tiles, V tiles in flight
 constexpr int kGUHalfBytes = kGUTileRows * 128;          // [128 rows][64 columns] bf16
 constexpr int kGUTileBytes = 2 * kGUHalfBytes;           // one K or V tile: 32 KB
 constexpr int kGUQBytes = 2 * kSUHeads * 128;            // Q tile, and each of the two P tiles: 4 KB
-constexpr int kGUSmemBytes = (kGUKStages + kGUVStages) * kGUTileBytes + 3 * kGUQBytes + 1024;
-constexpr int kGUThreads = 18 * 32;                      // 2 x 4 softmax warps, 2 x 4 loader warps, 2 MMA warps
+// Shape of a CTA: G softmax groups (1 or 2), SETS loader sets (1 or 2); K stages = SETS (one per set), V
+// stages = 2 SETS.  (2, 2): 18 warps and a 205 KB ring, one CTA per SM.  (1, 1): 10 warps and 109 KB, two CTAs
+// per SM, each with a shallower pipeline, covering each other's set-up and merge.
+template <int G, int SETS>
+struct GUShape {
+  static constexpr int kKStages = SETS, kVStages = 2 * SETS;
+  static constexpr int kLoaderWarp0 = 4 * G, kQKWarp = 4 * G + 4 * SETS, kPVWarp = kQKWarp + 1;
+  static constexpr int kThreads = (kPVWarp + 1) * 32;
+  static constexpr int kSmemBytes = (kKStages + kVStages) * kGUTileBytes + 3 * kGUQBytes + 1024;
+  static constexpr int kCtasPerSm = (G == 1 && SETS == 1) ? 2 : 1;
+};
 constexpr int kGUTmemCols = 64;                          // S0, S1, O0, O1: 16 fp32 columns each
 constexpr uint32_t kGUIdescQK = kSUIdesc;                // A = K tile (K-major), B = Q tile (K-major)
 constexpr uint32_t kGUIdescPV = kSUIdesc | (1u << 15);   // A = V tile read MN-major, B = P tile (K-major)
@@ -67,10 +79,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
 }
 // named barriers: 1 and 2 = the softmax groups (128 threads each), 3 = both groups
 __device__ __forceinline__ void group_bar(int g) { asm volatile("bar.sync %0, 128;" ::"r"(g + 1) : "memory"); }
-__device__ __forceinline__ void groups_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+__device__ __forceinline__ void groups_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }   // G = 2 only
 
-// grid (splits, Hkv, B), 576 threads.
-__global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(AttnParams p) {
+// grid (splits, Hkv, B), GUShape<G, SETS>::kThreads threads.
+template <int G, int SETS>
+__global__ void __launch_bounds__(GUShape<G, SETS>::kThreads, GUShape<G, SETS>::kCtasPerSm)
+gather_group_attn_umma_kernel(AttnParams p) {
+  using Shape = GUShape<G, SETS>;
+  constexpr int kGUKStages = Shape::kKStages, kGUVStages = Shape::kVStages, kGUThreads = Shape::kThreads;
   extern __shared__ unsigned char gu_smem_raw[];
   // full[0..4), k_empty[4..6), v_empty[6..10), s_full[10..12), s_empty[12..14), p_full[14..16), p_empty[16..18),
   // o_done[18], drain[19..21).  A wait names a phase by its parity, which is only sound for a waiter that
@@ -134,7 +150,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (warp == 16) {
+  if (warp == Shape::kQKWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"((uint32_t)__cvta_generic_to_shared(&tmem_slot)), "r"((uint32_t)kGUTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -144,13 +160,12 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
   tc_fence_after();
   const uint32_t tmem0 = *(volatile uint32_t*)&tmem_slot;
 
-  if (warp < 8) {
+  if (warp < Shape::kLoaderWarp0) {
     // ---------------- softmax groups: group g takes the tiles j = g, g + 2, ...; a thread is key
     // row `row` of each of them, and dimension `row` of the group's O^T
-    const int g = warp >> 2;
+    const int g = G == 2 ? warp >> 2 : 0;
     const int row = tid & 127;
     const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
-    const uint32_t tmem_s = tmem0 + (uint32_t)(g * kSUHeads) + lane_base;
     const uint32_t tmem_o = tmem0 + (uint32_t)((2 + g) * kSUHeads) + lane_base;
     float m_run[kSUHeads], l_run[kSUHeads], lt_run[kSUHeads];
 #pragma unroll
@@ -158,12 +173,14 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
     // A warp whose wait runs out sets `aborted` and keeps looping without touching anything, so that
     // the four warps of a group execute the same number of named barriers whatever happens.
     bool aborted = false;
-    for (int j = g, i = 0; j < ntiles; j += 2, ++i) {
+    for (int j = g, i = 0; j < ntiles; j += G, ++i) {
       const int stage = j % kGUVStages;
+      const int a = j & 1, ua = j >> 1;          // S and P buffer of the tile, and which use of them this is
+      const uint32_t tmem_s = tmem0 + (uint32_t)(a * kSUHeads) + lane_base;
       float s[16];
       bool exceed = false;
       if (!aborted) {
-        bool ok = mbar_wait(bar_sfull + 8 * g, i & 1, &sh_abort);
+        bool ok = mbar_wait(bar_sfull + 8 * a, ua & 1, &sh_abort);
         if (ok) ok = mbar_wait(bar_full + 8 * stage, (j / kGUVStages) & 1, &sh_abort);
         aborted = !__all_sync(0xffffffffu, ok);
       }
@@ -172,7 +189,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         tmem_ld16(tmem_s, s);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_sempty + 8 * g);
+        if (lane == 0) mbar_arrive(bar_sempty + 8 * a);
         const bool valid = ((vmask[stage][warp & 3] >> lane) & 1u) != 0u && start + j * kGUTileRows + row < end;
         // logits in the log2 domain; does any exceed its head's running maximum by more than the gap?
 #pragma unroll
@@ -223,8 +240,14 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         group_bar(g);                                      // red_max may be rewritten by the next raise
       }
       if (aborted) continue;
-      // the group's previous tile: its P tile has been consumed and its MMAs into O have landed
-      if (i >= 1 && !__all_sync(0xffffffffu, mbar_wait(bar_pempty + 8 * g, (i - 1) & 1, &sh_abort))) {
+      // the P buffer's previous tile has been consumed; with two groups that is the group's previous tile,
+      // whose MMAs into O have then landed too; a single group asks for its previous tile's separately
+      if (ua >= 1 && !__all_sync(0xffffffffu, mbar_wait(bar_pempty + 8 * a, (ua - 1) & 1, &sh_abort))) {
+        aborted = true;
+        continue;
+      }
+      if (G == 1 && raise && j >= 1 &&
+          !__all_sync(0xffffffffu, mbar_wait(bar_pempty + 8 * (a ^ 1), ((j - 1) >> 1) & 1, &sh_abort))) {
         aborted = true;
         continue;
       }
@@ -239,7 +262,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         tmem_st16(tmem_o, o);
         tc_fence_before();
       }
-      const uint32_t pdst = p_smem + g * kGUQBytes + (row >> 6) * (kSUHeads * 128) + (row & 7) * 2;
+      const uint32_t pdst = p_smem + a * kGUQBytes + (row >> 6) * (kSUHeads * 128) + (row & 7) * 2;
       const int pc = (row & 63) >> 3;
 #pragma unroll
       for (int h = 0; h < kSUHeads; ++h) {
@@ -253,7 +276,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_pfull + 8 * g);
+      if (lane == 0) mbar_arrive(bar_pfull + 8 * a);
     }
     if (aborted && lane == 0) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; }
     // ---- the group's result: O^T[row][head], the sums over its keys
@@ -285,7 +308,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
     }
     // ---- the odd tiles' group hands its result to the even tiles' group through the (free) ring
     float* xo = reinterpret_cast<float*>(gu_smem_raw + (smem0 - (uint32_t)__cvta_generic_to_shared(gu_smem_raw)));
-    if (g == 1) {
+    if (G == 2 && g == 1) {
 #pragma unroll
       for (int h = 0; h < kSUHeads; ++h)
         if (h < gq) xo[h * kGUTileRows + row] = o[h];
@@ -295,7 +318,8 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
           if (h < gq) other_m[h] = m_run[h];
       }
     }
-    groups_bar();
+    if (G == 2) groups_bar();
+    else group_bar(0);
     if (g == 0) {
       float M[kSUHeads], L[kSUHeads], Lt[kSUHeads];
 #pragma unroll
@@ -303,15 +327,15 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         if (h < gq) {
           const float l0 = red_l[0][0][h] + red_l[0][1][h] + red_l[0][2][h] + red_l[0][3][h];
           const float t0 = red_lt[0][0][h] + red_lt[0][1][h] + red_lt[0][2][h] + red_lt[0][3][h];
-          const float l1 = red_l[1][0][h] + red_l[1][1][h] + red_l[1][2][h] + red_l[1][3][h];
-          const float t1 = red_lt[1][0][h] + red_lt[1][1][h] + red_lt[1][2][h] + red_lt[1][3][h];
-          const float m1 = other_m[h];
+          const float l1 = G == 2 ? red_l[1][0][h] + red_l[1][1][h] + red_l[1][2][h] + red_l[1][3][h] : 0.f;
+          const float t1 = G == 2 ? red_lt[1][0][h] + red_lt[1][1][h] + red_lt[1][2][h] + red_lt[1][3][h] : 0.f;
+          const float m1 = G == 2 ? other_m[h] : -INFINITY;
           const float mm = fmaxf(m_run[h], m1);
           const float f0 = mm > -INFINITY ? exp2f(m_run[h] - mm) : 0.f, f1 = mm > -INFINITY ? exp2f(m1 - mm) : 0.f;
           M[h] = mm;
           L[h] = l0 * f0 + l1 * f1;
           Lt[h] = t0 * f0 + t1 * f1;
-          o[h] = o[h] * f0 + xo[h * kGUTileRows + row] * f1;
+          o[h] = o[h] * f0 + (G == 2 ? xo[h * kGUTileRows + row] * f1 : 0.f);
         }
       }
       auto finish = [&](int unit, float acc, float Mx, float Lx, float Ltx) {
@@ -365,11 +389,11 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         }
       }
     }
-  } else if (warp < 16) {
-    // ---------------- loader warps: set ls brings the tiles j = ls, ls + 2, ... (K stage ls, V stage j mod 4),
+  } else if (warp < Shape::kQKWarp) {
+    // ---------------- loader warps: set ls brings the tiles j = ls, ls + SETS, ... (K stage ls, V stage j mod 2 SETS),
     // warp `band` of the set the rows 32 band .. + 31 of each; lanes 0-15 copy a K row, lanes 16-31 the V
     // row of the same entry
-    const int ls = (warp - 8) >> 2, band = (warp - 8) & 3;
+    const int ls = (warp - Shape::kLoaderWarp0) >> 2, band = (warp - Shape::kLoaderWarp0) & 3;
     const bool paged = p.kv.page_table != nullptr;
     const uint32_t outer_rows = (uint32_t)(p.kv.stride_outer >> 7), head_rows = (uint32_t)(p.kv.stride_head >> 7);
     const int c = lane & 15;
@@ -378,11 +402,11 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
     const int jl0 = start + band * 32 + lane;
     int pos_next = list_entry(ld, jl0 + ls * kGUTileRows, end);
     bool aborted = false;
-    for (int j = ls, i = 0; j < ntiles; j += 2, ++i) {
+    for (int j = ls, i = 0; j < ntiles; j += SETS, ++i) {
       const int stage = j % kGUVStages;
       const int jl = jl0 + j * kGUTileRows;
       const int pos = checked_entry(ld, pos_next, jl, end, t, p.flags);
-      if (j + 2 < ntiles) pos_next = list_entry(ld, jl + 2 * kGUTileRows, end);
+      if (j + SETS < ntiles) pos_next = list_entry(ld, jl + SETS * kGUTileRows, end);
       uint32_t rid = kBadRow;
       if (pos >= 0) {
         if (paged) {
@@ -395,7 +419,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
       }
       const uint32_t vm = __ballot_sync(0xffffffffu, rid != kBadRow);
       if (rid == kBadRow) rid = 0u;
-      // the set's K stage was last read by the S of tile j - 2, the V stage by the O of tile j - 4
+      // the set's K stage was last read by the S of the set's previous tile, the V stage by the O of the one before
       bool ok = true;
       if (i >= 1) ok = mbar_wait(bar_kempty + 8 * ls, (i - 1) & 1, &sh_abort);
       if (ok && j >= kGUVStages) ok = mbar_wait(bar_vempty + 8 * stage, ((j / kGUVStages) - 1) & 1, &sh_abort);
@@ -419,7 +443,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
       if (lane == 0) mbar_arrive(bar_full + 8 * stage);
     }
     if (aborted && lane == 0) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; }
-  } else if (warp == 16) {
+  } else if (warp == Shape::kQKWarp) {
     // ---------------- S = K Q^T: one thread, one tile ahead of the softmax groups
     if (lane == 0) {
       const uint64_t qd = umma_desc(q_smem);
@@ -430,7 +454,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         if (ok) ok = mbar_wait(bar_full + 8 * (j % kGUVStages), (j / kGUVStages) & 1, &sh_abort);
         if (!ok) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; break; }
         tc_fence_after();
-        const uint64_t kd = umma_desc(smem0 + (uint32_t)a * kGUTileBytes);
+        const uint64_t kd = umma_desc(smem0 + (uint32_t)(j % kGUKStages) * kGUTileBytes);
         const uint32_t d = tmem0 + (uint32_t)(a * kSUHeads);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
@@ -438,7 +462,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
           const uint64_t qb = qd + (uint64_t)((ks >> 2) * ((kSUHeads * 128) >> 4) + (ks & 3) * 2);
           umma_bf16(d, ka, qb, kGUIdescQK, ks > 0 ? 1u : 0u);
         }
-        umma_commit(bar_kempty + 8 * a);       // the K stage may be refilled
+        umma_commit(bar_kempty + 8 * (j % kGUKStages));   // the K stage may be refilled
         umma_commit(bar_sfull + 8 * a);
       }
     }
@@ -453,13 +477,13 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
         tc_fence_after();
         const uint64_t vd = umma_desc_mn(v_ring + (uint32_t)stage * kGUTileBytes);
         const uint64_t pd = umma_desc(p_smem + a * kGUQBytes);
-        const uint32_t d = tmem0 + (uint32_t)((2 + a) * kSUHeads);
+        const uint32_t d = tmem0 + (uint32_t)((2 + (G == 2 ? a : 0)) * kSUHeads);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           // 16 keys further: sixteen 128-byte rows of the V tile, 32 bytes along a row of the P tile
           const uint64_t va = vd + (uint64_t)(ks * ((16 * 128) >> 4));
           const uint64_t pb = pd + (uint64_t)((ks >> 2) * ((kSUHeads * 128) >> 4) + (ks & 3) * 2);
-          umma_bf16(d, va, pb, kGUIdescPV, (j >= 2 || ks > 0) ? 1u : 0u);
+          umma_bf16(d, va, pb, kGUIdescPV, (j >= G || ks > 0) ? 1u : 0u);
         }
         umma_commit(bar_vempty + 8 * stage);   // the V stage may be refilled
         umma_commit(bar_pempty + 8 * a);       // and the group's P tile
@@ -473,8 +497,8 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
   if (sh_abort) {
     // MMAs may still be in flight: a bounded wait on a last commit of each issuing thread before the
     // tensor memory goes back
-    if (tid == 16 * 32 || tid == 17 * 32) {
-      const uint32_t bar = bar_drain + 8 * (warp - 16);
+    if (tid == Shape::kQKWarp * 32 || tid == Shape::kPVWarp * 32) {
+      const uint32_t bar = bar_drain + 8 * (warp - Shape::kQKWarp);
       umma_commit(bar);
       const long long t0 = clock64();
       while (!mbar_try_wait(bar, 0))
@@ -482,7 +506,7 @@ __global__ void __launch_bounds__(kGUThreads, 1) gather_group_attn_umma_kernel(A
     }
     __syncthreads();
   }
-  if (warp == 16) {
+  if (warp == Shape::kQKWarp) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem0), "r"((uint32_t)kGUTmemCols) : "memory");

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -381,20 +382,27 @@ prhs_status launch_attn(prhs_ctx* c, const void* q, const KvDev& kv, const int* 
     // group-shared sets: one CTA column per KV head, a gathered row serves the whole group
     LaunchScope ls(c, PRHS_KIND_ATTN_SPARSE, st);
     if (c->cfg.flags & PRHS_CFG_GROUP_TCGEN05) {
-      // one CTA per SM (a 200 KB ring): the split count that fills whole waves of SMs, tiles of 128 rows
+      // Two shapes of CTA: 18 warps with a 205 KB ring (one per SM: the deeper pipeline), or 10 warps with
+      // 109 KB (two per SM, which cover each other's set-up and merge).  The second where there are more
+      // units than SMs and a launch is several waves (the ragged paged batch of 64: 128 us against 192 us
+      // per sharing step; at 128 units the first: 44.5 against 56.5).  Then the split count that fills
+      // whole waves of CTA slots, in tiles of 128 rows.
       const int units = batch * c->cfg.num_kv_heads;
+      const bool light = units > c->sm_count;
+      const int slots = c->sm_count * (light ? 2 : 1);
       int best = 1;
       double best_cost = 1e30;
       for (int s = 1; s <= kMaxSplits; ++s) {
         const int rows = (((max_count + s - 1) / s) + kGUTileRows - 1) & ~(kGUTileRows - 1);
         if (s > 1 && rows < 2 * kGUTileRows) break;
-        const double waves = (double)(((long long)units * s + c->sm_count - 1) / c->sm_count);
+        const double waves = (double)(((long long)units * s + slots - 1) / slots);
         const double cost = waves * (rows + 2 * kGUTileRows);
         if (cost < best_cost * 0.999) { best_cost = cost; best = s; }
       }
       p.splits = best;
       dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
-      gather_group_attn_umma_kernel<<<grid, kGUThreads, kGUSmemBytes, st>>>(p);
+      if (light) gather_group_attn_umma_kernel<1, 1><<<grid, GUShape<1, 1>::kThreads, GUShape<1, 1>::kSmemBytes, st>>>(p);
+      else gather_group_attn_umma_kernel<2, 2><<<grid, GUShape<2, 2>::kThreads, GUShape<2, 2>::kSmemBytes, st>>>(p);
     } else {
       p.splits = pick_splits(c, batch * c->cfg.num_kv_heads, max_count);
       dim3 grid(p.splits, c->cfg.num_kv_heads, batch);
@@ -767,7 +775,9 @@ prhs_status prhs_create(const prhs_config* cfg, prhs_ctx** out) {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gather_group_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTSmemBytes);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(gather_group_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGUSmemBytes);
+    e = cudaFuncSetAttribute(gather_group_attn_umma_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GUShape<2, 2>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gather_group_attn_umma_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, GUShape<1, 1>::kSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(score_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSTSmemBytes);
   if (e == cudaSuccess)

@@ -926,6 +926,18 @@ def test_group_sets_tcgen05_schedule(cuda_device, hq, hkv, paged):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("paged", [False, True])
+def test_group_sets_tcgen05_more_units_than_sms(cuda_device, paged):
+    # more (sequence, KV head) units than the GPU has SMs: the library launches the kernel in its second
+    # shape (one softmax group and one loader set per CTA, two CTAs per SM)
+    w = small(layers=1, steps=3, refresh=2, batch=24, q_heads=16, kv_heads=8, context=900, top_k=200,
+              min_context=300, page_size=16 if paged else 0, seed=53)
+    st = H.run_schedule_parity(w, cuda_device, all_units(w), paged=paged, group_sets=True,
+                               ctx_over=dict(flags=P.PRHS_CFG_GROUP_TCGEN05))
+    assert st["checked"] == 3 * w.batch * w.q_heads
+
+
+@pytest.mark.gpu
 def test_group_sets_tcgen05_full_shapes_sampled(cuda_device):
     # the Mistral-shaped stack, the 128K shape (several splits per unit: partials and the merge) and the
     # ragged paged serving mix
