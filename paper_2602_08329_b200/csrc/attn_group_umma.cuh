@@ -401,13 +401,13 @@ gather_group_attn_umma_kernel(AttnParams p) {
     const uint32_t dst_lane = (uint32_t)(c >> 3) * kGUHalfBytes;
     const int jl0 = start + band * 32 + lane;
     int pos_next = list_entry(ld, jl0 + ls * kGUTileRows, end);
-    bool aborted = false;
-    for (int j = ls, i = 0; j < ntiles; j += SETS, ++i) {
-      const int stage = j % kGUVStages;
+    // row id of this lane's entry of tile j (0 and a cleared bit of vm if it is masked); also starts the load
+    // of the entry of the set's next tile
+    auto lookup = [&](int j, uint32_t& rid, uint32_t& vm) {
       const int jl = jl0 + j * kGUTileRows;
       const int pos = checked_entry(ld, pos_next, jl, end, t, p.flags);
       if (j + SETS < ntiles) pos_next = list_entry(ld, jl + SETS * kGUTileRows, end);
-      uint32_t rid = kBadRow;
+      rid = kBadRow;
       if (pos >= 0) {
         if (paged) {
           const int page = __ldg(p.kv.page_table + (long long)b * p.kv.page_table_stride + (pos >> kPageShift));
@@ -417,8 +417,14 @@ gather_group_attn_umma_kernel(AttnParams p) {
           rid = (uint32_t)b * outer_rows + (uint32_t)kvh * head_rows + (uint32_t)pos;
         }
       }
-      const uint32_t vm = __ballot_sync(0xffffffffu, rid != kBadRow);
+      vm = __ballot_sync(0xffffffffu, rid != kBadRow);
       if (rid == kBadRow) rid = 0u;
+    };
+    uint32_t rid = 0u, vm = 0u;
+    if (ls < ntiles) lookup(ls, rid, vm);
+    bool aborted = false;
+    for (int j = ls, i = 0; j < ntiles; j += SETS, ++i) {
+      const int stage = j % kGUVStages;
       // the set's K stage was last read by the S of the set's previous tile, the V stage by the O of the one before
       bool ok = true;
       if (i >= 1) ok = mbar_wait(bar_kempty + 8 * ls, (i - 1) & 1, &sh_abort);
@@ -436,11 +442,16 @@ gather_group_attn_umma_kernel(AttnParams p) {
         cp_async_16(tile + trow * 128 + (((c & 7) ^ (trow & 7)) << 4), src + (size_t)rr * kHeadDim, ((vm >> r) & 1u) ? 16 : 0);
       }
       cp_async_commit();
+      // while the rows are on their way: the row ids of the set's next tile
+      uint32_t rid_n = 0u, vm_n = 0u;
+      if (j + SETS < ntiles) lookup(j + SETS, rid_n, vm_n);
       // the rows have landed: made visible to the tensor core, then signalled
       cp_async_wait<0>();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_full + 8 * stage);
+      rid = rid_n;
+      vm = vm_n;
     }
     if (aborted && lane == 0) { atomicOr(p.flags, kFlagTimeout); sh_abort = 1; }
   } else if (warp == Shape::kQKWarp) {
